@@ -1,0 +1,226 @@
+/*
+ * sbnn.h — C interface of libsbnn: group-sparse convolution for NVIDIA B200 (sm_100a).
+ *
+ * The library computes convolutions whose weights are fine-grained group-sparse:
+ * G consecutive output channels (one "group") share one 0/1 mask over the input
+ * channels, so a "unit" — the G weights (1x1 kernel) or 9*G weights (3x3 kernel)
+ * that connect one input channel to one group — is either kept or removed as a
+ * whole (the paper's connectivity group pruning, Section 3.2 and Eq. 2, with an
+ * input-channel group size of 1).  The result is by definition the ordinary
+ * convolution with W~ = W (.) M (Section 3.1); the kernels reach it by visiting
+ * kept units only (Algorithm 1).
+ *
+ * Conventions that hold for every entry point
+ *   - Tensors: activations [N][H][W][C] fp32 (NHWC), weights [Cout][KH][KW][Cin]
+ *     fp32, as in Algorithm 1's data declaration.  Zero padding (K-1)/2,
+ *     cross-correlation (no kernel flip), bias added before the optional ReLU.
+ *   - "_host" pointers are ordinary host memory, "_dev" pointers are device
+ *     memory of the current CUDA device, 16-byte aligned, owned by the caller.
+ *     Input and output buffers must not overlap.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Compute calls only enqueue kernels on it and return; they never
+ *     synchronise.  Calls that create, pack or free objects may synchronise.
+ *   - Every function returns an sbnn_status; nothing throws, aborts or exits.
+ *     On error no kernel is launched.  sbnn_last_error() gives a thread-local
+ *     one-line explanation of the most recent failure.
+ *   - There is no CPU fallback: compute calls need a B200-class device
+ *     (compute capability 10.x) and fail with SBNN_ERR_ARCH / SBNN_ERR_CUDA
+ *     otherwise.  Packing is host-side and works without a device.
+ */
+#ifndef SBNN_H_
+#define SBNN_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SBNN_API __attribute__((visibility("default")))
+#else
+#define SBNN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SBNN_OK = 0,
+    SBNN_ERR_NULL = 1,                   /* a required pointer is NULL */
+    SBNN_ERR_SHAPE = 2,                  /* a dimension is negative, zero where it may not be, or inconsistent */
+    SBNN_ERR_GROUP = 3,                  /* G not in {1,2,4,8,16} or Cout % G != 0 */
+    SBNN_ERR_MASK_NOT_GROUP_UNIFORM = 4, /* mask differs inside a group's rows or taps, or holds a value > 1 */
+    SBNN_ERR_ALIGN = 5,                  /* a device pointer is not 16-byte aligned */
+    SBNN_ERR_UNSUPPORTED = 6,            /* valid request outside what the kernels implement */
+    SBNN_ERR_ARCH = 7,                   /* current device is not compute capability 10.x */
+    SBNN_ERR_ALLOC = 8,                  /* host or device allocation failed */
+    SBNN_ERR_CUDA = 9,                   /* a CUDA runtime call failed or no device is present */
+    SBNN_ERR_TIMEOUT = 10                /* a bounded device-side wait gave up (reported by sbnn_get_async_status) */
+} sbnn_status;
+
+/* Static name of a status code ("SBNN_OK", ...). Never NULL. */
+SBNN_API const char* sbnn_status_str(sbnn_status s);
+/* Detail of the calling thread's most recent failing call; "" if none.  Valid until that thread's next call. */
+SBNN_API const char* sbnn_last_error(void);
+
+/* ------------------------------------------------------------------------------------------------
+ * Packing (Section 3.5: the conversion step that produces the engine's sparse weight format;
+ * Algorithm 1's "sparse info SD" is the per-group list of kept input channels).
+ * ------------------------------------------------------------------------------------------------ */
+
+/* Opaque packed layer.  Owns a host copy and, if a device was present at pack time, device copies. */
+typedef struct sbnn_packed sbnn_packed;
+
+/*
+ * Build the group-compressed form of one layer.
+ *   W_host    [Cout][KH][KW][Cin] fp32 dense weights (values under a zero mask entry are ignored)
+ *   mask_host [Cout][KH][KW][Cin] uint8, 1 = kept.  Must be identical for the G rows of a group and
+ *             for all KH*KW taps (a unit is kept or removed as a whole), else
+ *             SBNN_ERR_MASK_NOT_GROUP_UNIFORM.
+ *   bias_host [Cout] or NULL (= zeros)
+ *   KH = KW = 1 or 3.  G in {1,2,4,8,16}, Cout % G == 0.
+ * Canonical layout produced (all little-endian host arrays, also uploaded to the device):
+ *   group_ptr int32 [Cout/G + 1]   prefix sums of kept units per group
+ *   idx       int32 [nnz_units]    kept input channels, ascending inside each group
+ *   val       fp32  [nnz_units][KH*KW][G]   weights of a unit: taps outer, the group's channels inner
+ *   bias      fp32  [Cout]
+ * A kept weight that is numerically zero stays stored (packing follows the mask, not the values).
+ * On success *out owns everything; release it with sbnn_packed_free.  If no CUDA device is present the
+ * object is host-only (view / unpack work, compute calls return SBNN_ERR_CUDA).
+ */
+SBNN_API sbnn_status sbnn_pack_weights(const float* W_host, const uint8_t* mask_host, const float* bias_host,
+                                       int Cout, int KH, int KW, int Cin, int G, sbnn_packed** out);
+
+typedef struct {
+    int Cout, KH, KW, Cin, G, ngroups;
+    int64_t nnz_units;
+    const int32_t* group_ptr; /* host, borrowed from the sbnn_packed */
+    const int32_t* idx;       /* host, borrowed */
+    const float* val;         /* host, borrowed */
+    const float* bias;        /* host, borrowed */
+} sbnn_packed_view;
+
+/* Borrow the canonical host arrays; they stay valid until sbnn_packed_free. */
+SBNN_API sbnn_status sbnn_packed_get(const sbnn_packed* p, sbnn_packed_view* view);
+/* Inverse of packing: writes W (.) M and M (either pointer may be NULL), each [Cout][KH][KW][Cin]. */
+SBNN_API sbnn_status sbnn_unpack_weights(const sbnn_packed* p, float* W_host_out, uint8_t* mask_host_out);
+/* Frees host and device copies.  NULL is accepted. */
+SBNN_API sbnn_status sbnn_packed_free(sbnn_packed* p);
+
+/* ------------------------------------------------------------------------------------------------
+ * Group-sparse convolutions (Algorithm 1 for the 1x1 case; Section 3.2's connectivity group
+ * pruning of whole 3x3 kernels for the 3x3 case).
+ * ------------------------------------------------------------------------------------------------ */
+
+enum {
+    SBNN_RELU = 1,    /* apply max(.,0) after the bias */
+    SBNN_BF16_TC = 2  /* 1x1 only: round activations and weights to bf16 and contract on tensor cores, fp32 accumulate */
+};
+
+/*
+ * Y[n][y][x][g*G + r] = act( bias[g*G + r] + sum_j val[g][j][r] * X[n][y][x][idx[g][j]] )
+ *   w      packed 1x1 layer (KH = KW = 1)
+ *   x_dev  [N][H][W][Cin] fp32, y_dev [N][H][W][Cout] fp32
+ * Cin must be a multiple of 4 (else SBNN_ERR_UNSUPPORTED).  N*H*W == 0 returns SBNN_OK without a launch.
+ */
+SBNN_API sbnn_status sbnn_conv1x1_gs(const sbnn_packed* w, const float* x_dev, float* y_dev,
+                                     int N, int H, int W, int flags, void* cuda_stream);
+
+/*
+ * Same operation with an explicit tile shape, for tuning and for testing every compiled kernel
+ * instance: P pixels per lane, GPW groups per warp, NW warps per CTA, KC input channels per
+ * pipeline step.  Combinations that were not compiled return SBNN_ERR_UNSUPPORTED.  The first call
+ * with a new combination builds a private re-layout of the weights (allocates and copies
+ * synchronously); later calls only enqueue.  SBNN_BF16_TC is not accepted here.
+ */
+SBNN_API sbnn_status sbnn_conv1x1_gs_tuned(const sbnn_packed* w, const float* x_dev, float* y_dev,
+                                           int N, int H, int W, int flags, int P, int GPW, int NW, int KC,
+                                           void* cuda_stream);
+
+/*
+ * 3x3, stride 1, pad 1:
+ * Y[n][y][x][g*G + r] = act( bias + sum_j sum_{kh,kw} val[g][j][kh*3+kw][r] * X[n][y+kh-1][x+kw-1][idx[g][j]] ),
+ * X taken as zero outside the image.  Shapes as above with KH = KW = 3.  SBNN_BF16_TC is not accepted.
+ */
+SBNN_API sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev, float* y_dev,
+                                     int N, int H, int W, int flags, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Dense supporting layers of MobileNet-v1 (Section 3.2 names the operators; they stay dense here).
+ * ------------------------------------------------------------------------------------------------ */
+
+/*
+ * Depthwise 3x3, pad 1, stride 1 or 2:
+ * Y[n][y][x][c] = act( b[c] + sum_{kh,kw} w[kh][kw][c] * X[n][s*y+kh-1][s*x+kw-1][c] ).
+ *   w_dev [3][3][C], b_dev [C] or NULL, x_dev [N][H][W][C], y_dev [N][Ho][Wo][C], Ho = (H-1)/s + 1.
+ * C must be a multiple of 4.
+ */
+SBNN_API sbnn_status sbnn_dwconv3x3(const float* w_dev, const float* b_dev, const float* x_dev, float* y_dev,
+                                    int N, int H, int W, int C, int stride, int flags, void* cuda_stream);
+
+/*
+ * Dense 3x3, pad 1, stride 1 or 2, for thin inputs (the network's first layer, Cin = 3):
+ *   w_dev [Cout][3][3][Cin], b_dev [Cout] or NULL, x_dev [N][H][W][Cin], y_dev [N][Ho][Wo][Cout].
+ * Cin <= 4 and Cout a multiple of 8 and <= 64; other shapes return SBNN_ERR_UNSUPPORTED.
+ * x_dev needs 4-byte alignment only.
+ */
+SBNN_API sbnn_status sbnn_conv3x3_dense(const float* w_dev, const float* b_dev, const float* x_dev, float* y_dev,
+                                        int N, int H, int W, int Cin, int Cout, int stride, int flags,
+                                        void* cuda_stream);
+
+/* Global average pool: x_dev [N][HW][C] -> y_dev [N][C], C a multiple of 4. */
+SBNN_API sbnn_status sbnn_avgpool(const float* x_dev, float* y_dev, int N, int HW, int C, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * MobileNet-v1 (width 1.0, 224x224x3) forward chain (Section 3.5: the sparse inference engine's
+ * forward pass; Tables 3 and 4 prune the 13 pointwise layers only).
+ * ------------------------------------------------------------------------------------------------ */
+
+typedef struct sbnn_mbv1 sbnn_mbv1;
+
+#define SBNN_MBV1_NUM_BLOCKS 13
+#define SBNN_MBV1_NUM_LAYERS 29 /* conv0, 13 x (dw, pw), pool, fc */
+
+/*
+ * Bind weights and allocate the two ping-pong activation workspaces for up to max_batch images.
+ *   pw[13]        packed pointwise layers, in network order (borrowed; must outlive the network)
+ *   fc            packed classifier, 1000 x 1024, any G dividing 1000 (normally a full mask)
+ *   dw_w_dev[13]  depthwise weights [3][3][C]; dw_b_dev[13] their biases [C]  (device, borrowed)
+ *   conv0_w_dev   [32][3][3][3], conv0_b_dev [32]                               (device, borrowed)
+ * Shapes are checked against the network's layer table.
+ */
+SBNN_API sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, const sbnn_packed* fc,
+                                              const float* const* dw_w_dev, const float* const* dw_b_dev,
+                                              const float* conv0_w_dev, const float* conv0_b_dev,
+                                              int max_batch, sbnn_mbv1** out);
+
+/*
+ * Enqueue the whole forward pass for N <= max_batch images on one stream:
+ * conv0 -> 13 x (depthwise 3x3 -> group-sparse 1x1) -> average pool -> classifier.
+ *   x_dev [N][224][224][3] fp32 (4-byte aligned is enough), logits_dev [N][1000] fp32.
+ * Every conv but the classifier applies ReLU.  No host synchronisation.
+ */
+SBNN_API sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_dev, float* logits_dev,
+                                               int N, void* cuda_stream);
+
+/*
+ * Run a single layer of the chain on caller-provided input (for layer-isolated checks):
+ * layer 0 = conv0, 2i-1 = dw_i, 2i = pw_i (i = 1..13), 27 = pool, 28 = fc.
+ * in_dev / out_dev are NHWC buffers of that layer's input / output shape for N images.
+ */
+SBNN_API sbnn_status sbnn_mobilenet_v1_run_layer(sbnn_mbv1* net, int layer, const float* in_dev, float* out_dev,
+                                                 int N, void* cuda_stream);
+
+/* Shape of a layer of the chain: input side, input channels, output side, output channels. */
+SBNN_API sbnn_status sbnn_mobilenet_v1_layer_shape(int layer, int* Hin, int* Cin, int* Hout, int* Cout);
+
+SBNN_API sbnn_status sbnn_mobilenet_v1_free(sbnn_mbv1* net);
+
+/*
+ * Synchronise the stream and report device-side trouble: SBNN_ERR_CUDA if a kernel failed,
+ * SBNN_ERR_TIMEOUT if a bounded wait inside a kernel expired, else SBNN_OK.
+ */
+SBNN_API sbnn_status sbnn_get_async_status(void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SBNN_H_ */
