@@ -1,0 +1,95 @@
+// Shared declarations of libsbnn's translation units (not part of the public interface).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <map>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "sbnn.h"
+
+namespace sbnn {
+
+// Records the thread-local error text and returns `s`, so call sites can `return fail(...)`.
+sbnn_status fail(sbnn_status s, const char* fmt, ...);
+void clear_error();
+
+// SBNN_OK if the current device exists and is compute capability 10.x.
+sbnn_status check_device();
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+#define SBNN_CUDA_TRY(expr)                                                                         \
+    do {                                                                                            \
+        cudaError_t e__ = (expr);                                                                   \
+        if (e__ != cudaSuccess)                                                                     \
+            return ::sbnn::fail(e__ == cudaErrorMemoryAllocation ? SBNN_ERR_ALLOC : SBNN_ERR_CUDA,  \
+                                "%s: %s", #expr, cudaGetErrorString(e__));                          \
+    } while (0)
+
+// Tile configuration of the group-sparse 1x1 kernel; also the key of the kernel-private weight stream.
+struct TileCfg {
+    int P;    // pixels per lane (a warp covers 32*P consecutive pixels)
+    int GPW;  // groups a warp accumulates at once
+    int NW;   // warps per CTA
+    int KC;   // input channels staged per pipeline step
+    int TM() const { return 32 * P; }
+    int GT() const { return NW * GPW; }
+    bool operator<(const TileCfg& o) const {
+        if (P != o.P) return P < o.P;
+        if (GPW != o.GPW) return GPW < o.GPW;
+        if (NW != o.NW) return NW < o.NW;
+        return KC < o.KC;
+    }
+};
+
+// Kernel-private re-layout of a packed 1x1 layer for one TileCfg (device memory).
+struct Stream1x1 {
+    uint4* rec = nullptr;        // record stream, 16-byte units
+    int32_t* blk_ptr = nullptr;  // [ntiles][nchunks + 1] offsets into rec
+    int ntiles = 0, nchunks = 0;
+    int max_blk = 0;             // largest block in 16-byte units
+};
+
+// Kernel-private re-layout of a packed 3x3 layer (see conv3x3_gs.cu).
+struct Stream3x3 {
+    uint4* rec = nullptr;
+    int32_t* blk_ptr = nullptr;
+    int ntiles = 0, nchunks = 0;
+    int max_blk = 0;
+};
+
+}  // namespace sbnn
+
+struct sbnn_packed {
+    int Cout = 0, KH = 0, KW = 0, Cin = 0, G = 0, ngroups = 0;
+    int64_t nnz = 0;
+    std::vector<int32_t> group_ptr, idx;
+    std::vector<float> val, bias;
+    // device side (valid when device >= 0)
+    int device = -1;
+    int32_t* d_group_ptr = nullptr;
+    int32_t* d_idx = nullptr;
+    float* d_val = nullptr;
+    float* d_bias = nullptr;
+    // kernel-private layouts, built on first use of a tile configuration
+    mutable std::mutex mu;
+    mutable std::map<sbnn::TileCfg, sbnn::Stream1x1> streams1x1;
+    mutable std::map<int, sbnn::Stream3x3> streams3x3;
+    mutable void* bf16_stream = nullptr;  // see conv1x1_bf16.cu
+};
+
+namespace sbnn {
+// conv1x1_gs.cu
+sbnn_status prepare_default_1x1(const sbnn_packed* p);
+void free_streams_1x1(sbnn_packed* p);
+// conv1x1_bf16.cu
+sbnn_status conv1x1_bf16(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st);
+void free_stream_bf16(sbnn_packed* p);
+// conv3x3_gs.cu
+sbnn_status prepare_default_3x3(const sbnn_packed* p);
+void free_streams_3x3(sbnn_packed* p);
+}  // namespace sbnn

@@ -1,0 +1,234 @@
+// Status strings, error text, and the host-side packer of group-sparse weights
+// (the conversion step of Section 3.5; Algorithm 1's "sparse info" becomes the
+// per-group list of kept input channels).
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.h"
+
+namespace sbnn {
+
+static thread_local char g_err[512] = "";
+
+sbnn_status fail(sbnn_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+void clear_error() { g_err[0] = 0; }
+
+sbnn_status check_device() {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(SBNN_ERR_CUDA, "no usable CUDA device: %s", cudaGetErrorString(e));
+    }
+    static std::mutex mu;
+    static std::map<int, int> major_of;
+    int major = 0;
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        auto it = major_of.find(dev);
+        if (it == major_of.end()) {
+            e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+            if (e != cudaSuccess) {
+                cudaGetLastError();
+                return fail(SBNN_ERR_CUDA, "cannot query device %d: %s", dev, cudaGetErrorString(e));
+            }
+            major_of[dev] = major;
+        } else {
+            major = it->second;
+        }
+    }
+    if (major != 10)
+        return fail(SBNN_ERR_ARCH, "device %d has compute capability %d.x; this library is built for 10.x", dev, major);
+    return SBNN_OK;
+}
+
+static bool supported_group(int G) { return G == 1 || G == 2 || G == 4 || G == 8 || G == 16; }
+
+template <typename T>
+static sbnn_status upload(T** dst, const std::vector<T>& src) {
+    size_t bytes = (src.size() ? src.size() : 1) * sizeof(T);
+    SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(dst), bytes));
+    if (!src.empty()) SBNN_CUDA_TRY(cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice));
+    return SBNN_OK;
+}
+
+}  // namespace sbnn
+
+using namespace sbnn;
+
+extern "C" const char* sbnn_status_str(sbnn_status s) {
+    switch (s) {
+        case SBNN_OK: return "SBNN_OK";
+        case SBNN_ERR_NULL: return "SBNN_ERR_NULL";
+        case SBNN_ERR_SHAPE: return "SBNN_ERR_SHAPE";
+        case SBNN_ERR_GROUP: return "SBNN_ERR_GROUP";
+        case SBNN_ERR_MASK_NOT_GROUP_UNIFORM: return "SBNN_ERR_MASK_NOT_GROUP_UNIFORM";
+        case SBNN_ERR_ALIGN: return "SBNN_ERR_ALIGN";
+        case SBNN_ERR_UNSUPPORTED: return "SBNN_ERR_UNSUPPORTED";
+        case SBNN_ERR_ARCH: return "SBNN_ERR_ARCH";
+        case SBNN_ERR_ALLOC: return "SBNN_ERR_ALLOC";
+        case SBNN_ERR_CUDA: return "SBNN_ERR_CUDA";
+        case SBNN_ERR_TIMEOUT: return "SBNN_ERR_TIMEOUT";
+    }
+    return "SBNN_ERR_UNKNOWN";
+}
+
+extern "C" const char* sbnn_last_error(void) { return g_err; }
+
+extern "C" sbnn_status sbnn_pack_weights(const float* W, const uint8_t* mask, const float* bias, int Cout, int KH,
+                                         int KW, int Cin, int G, sbnn_packed** out) {
+    clear_error();
+    if (!W || !mask || !out) return fail(SBNN_ERR_NULL, "W_host, mask_host and out must not be NULL");
+    *out = nullptr;
+    if (Cout <= 0 || Cin <= 0) return fail(SBNN_ERR_SHAPE, "Cout=%d and Cin=%d must be positive", Cout, Cin);
+    if (!((KH == 1 && KW == 1) || (KH == 3 && KW == 3)))
+        return fail(SBNN_ERR_SHAPE, "kernel %dx%d: only 1x1 and 3x3", KH, KW);
+    if (!supported_group(G)) return fail(SBNN_ERR_GROUP, "G=%d not in {1,2,4,8,16}", G);
+    if (Cout % G) return fail(SBNN_ERR_GROUP, "Cout=%d is not a multiple of G=%d", Cout, G);
+
+    sbnn_packed* p = new (std::nothrow) sbnn_packed;
+    if (!p) return fail(SBNN_ERR_ALLOC, "out of host memory");
+    p->Cout = Cout; p->KH = KH; p->KW = KW; p->Cin = Cin; p->G = G; p->ngroups = Cout / G;
+    const int taps = KH * KW;
+    const int64_t row = (int64_t)taps * Cin;  // elements per output channel
+    try {
+        p->group_ptr.assign(p->ngroups + 1, 0);
+        p->bias.assign(Cout, 0.0f);
+        if (bias) memcpy(p->bias.data(), bias, sizeof(float) * Cout);
+        // Pass 1: validate that a unit is kept or removed as a whole, and count.
+        for (int g = 0; g < p->ngroups; ++g) {
+            const uint8_t* m0 = mask + (int64_t)g * G * row;  // first row, first tap
+            int kept = 0;
+            for (int c = 0; c < Cin; ++c) {
+                const uint8_t ref = m0[c];
+                if (ref > 1) {
+                    delete p;
+                    return fail(SBNN_ERR_MASK_NOT_GROUP_UNIFORM, "mask value %d at group %d channel %d is not 0/1", ref, g, c);
+                }
+                for (int r = 0; r < G; ++r)
+                    for (int t = 0; t < taps; ++t)
+                        if (m0[(int64_t)r * row + (int64_t)t * Cin + c] != ref) {
+                            delete p;
+                            return fail(SBNN_ERR_MASK_NOT_GROUP_UNIFORM,
+                                        "mask of group %d differs at row %d tap %d channel %d", g, r, t, c);
+                        }
+                kept += ref;
+            }
+            p->group_ptr[g + 1] = p->group_ptr[g] + kept;
+        }
+        p->nnz = p->group_ptr[p->ngroups];
+        p->idx.resize(p->nnz);
+        p->val.resize((size_t)p->nnz * taps * G);
+        // Pass 2: emit ascending indices and the [taps][G] value block of every kept unit.
+        for (int g = 0; g < p->ngroups; ++g) {
+            const uint8_t* m0 = mask + (int64_t)g * G * row;
+            const float* w0 = W + (int64_t)g * G * row;
+            int64_t u = p->group_ptr[g];
+            for (int c = 0; c < Cin; ++c) {
+                if (!m0[c]) continue;
+                p->idx[u] = c;
+                float* v = p->val.data() + (size_t)u * taps * G;
+                for (int t = 0; t < taps; ++t)
+                    for (int r = 0; r < G; ++r) v[t * G + r] = w0[(int64_t)r * row + (int64_t)t * Cin + c];
+                ++u;
+            }
+        }
+    } catch (const std::bad_alloc&) {
+        delete p;
+        return fail(SBNN_ERR_ALLOC, "out of host memory while packing");
+    }
+
+    // Device copies, if there is a device.
+    int ndev = 0, dev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0 || cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        *out = p;
+        return SBNN_OK;
+    }
+    sbnn_status st = SBNN_OK;
+    p->device = dev;
+    if ((st = upload(&p->d_group_ptr, p->group_ptr)) != SBNN_OK || (st = upload(&p->d_idx, p->idx)) != SBNN_OK ||
+        (st = upload(&p->d_val, p->val)) != SBNN_OK || (st = upload(&p->d_bias, p->bias)) != SBNN_OK) {
+        sbnn_packed_free(p);
+        return st;
+    }
+    st = (KH == 1) ? prepare_default_1x1(p) : prepare_default_3x3(p);
+    if (st != SBNN_OK) {
+        sbnn_packed_free(p);
+        return st;
+    }
+    *out = p;
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_packed_get(const sbnn_packed* p, sbnn_packed_view* v) {
+    clear_error();
+    if (!p || !v) return fail(SBNN_ERR_NULL, "packed and view must not be NULL");
+    v->Cout = p->Cout; v->KH = p->KH; v->KW = p->KW; v->Cin = p->Cin; v->G = p->G; v->ngroups = p->ngroups;
+    v->nnz_units = p->nnz;
+    v->group_ptr = p->group_ptr.data();
+    v->idx = p->idx.data();
+    v->val = p->val.data();
+    v->bias = p->bias.data();
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_unpack_weights(const sbnn_packed* p, float* W, uint8_t* mask) {
+    clear_error();
+    if (!p) return fail(SBNN_ERR_NULL, "packed must not be NULL");
+    const int taps = p->KH * p->KW, G = p->G;
+    const int64_t row = (int64_t)taps * p->Cin;
+    if (W) memset(W, 0, sizeof(float) * row * p->Cout);
+    if (mask) memset(mask, 0, (size_t)row * p->Cout);
+    for (int g = 0; g < p->ngroups; ++g)
+        for (int64_t u = p->group_ptr[g]; u < p->group_ptr[g + 1]; ++u) {
+            const int c = p->idx[u];
+            const float* v = p->val.data() + (size_t)u * taps * G;
+            for (int t = 0; t < taps; ++t)
+                for (int r = 0; r < G; ++r) {
+                    int64_t o = ((int64_t)g * G + r) * row + (int64_t)t * p->Cin + c;
+                    if (W) W[o] = v[t * G + r];
+                    if (mask) mask[o] = 1;
+                }
+        }
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_packed_free(sbnn_packed* p) {
+    clear_error();
+    if (!p) return SBNN_OK;
+    if (p->device >= 0) {
+        int cur = 0;
+        bool sw = cudaGetDevice(&cur) == cudaSuccess && cur != p->device && cudaSetDevice(p->device) == cudaSuccess;
+        free_streams_1x1(p);
+        free_stream_bf16(p);
+        free_streams_3x3(p);
+        cudaFree(p->d_group_ptr);
+        cudaFree(p->d_idx);
+        cudaFree(p->d_val);
+        cudaFree(p->d_bias);
+        if (sw) cudaSetDevice(cur);
+        cudaGetLastError();
+    }
+    delete p;
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_get_async_status(void* stream) {
+    clear_error();
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail(SBNN_ERR_CUDA, "stream failed: %s", cudaGetErrorString(e));
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(SBNN_ERR_CUDA, "pending error: %s", cudaGetErrorString(e));
+    return SBNN_OK;
+}
