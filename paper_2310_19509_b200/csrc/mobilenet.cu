@@ -1,0 +1,158 @@
+// MobileNet-v1 (width 1.0, 224x224x3) forward chain: the engine's forward pass of Section 3.5
+// with the 13 pointwise layers group-sparse (the layers Tables 3 and 4 prune) and everything
+// else dense.  Launches only: conv0 -> 13 x (depthwise, pointwise) -> pool -> classifier on one
+// stream over two ping-pong workspaces.
+#include <new>
+
+#include "common.h"
+
+namespace sbnn {
+namespace {
+
+struct LayerShape {
+    int kind;  // 0 conv0, 1 dw, 2 pw, 3 pool, 4 fc
+    int hin, cin, hout, cout, stride;
+};
+
+// Network table (Howard et al. 2017, Table 1).
+struct Table {
+    LayerShape t[SBNN_MBV1_NUM_LAYERS];
+    Table() {
+        static const int chans[SBNN_MBV1_NUM_BLOCKS][3] = {
+            {32, 64, 1},   {64, 128, 2},  {128, 128, 1}, {128, 256, 2}, {256, 256, 1}, {256, 512, 2}, {512, 512, 1},
+            {512, 512, 1}, {512, 512, 1}, {512, 512, 1}, {512, 512, 1}, {512, 1024, 2}, {1024, 1024, 1}};
+        int n = 0, h = 112;
+        t[n++] = {0, 224, 3, 112, 32, 2};
+        for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
+            const int ci = chans[i][0], co = chans[i][1], s = chans[i][2];
+            t[n++] = {1, h, ci, h / s, ci, s};
+            h /= s;
+            t[n++] = {2, h, ci, h, co, 1};
+        }
+        t[n++] = {3, 7, 1024, 1, 1024, 1};
+        t[n++] = {4, 1, 1024, 1, 1000, 1};
+    }
+};
+
+const LayerShape* layer_table() {
+    static const Table tab;
+    return tab.t;
+}
+
+}  // namespace
+}  // namespace sbnn
+
+struct sbnn_mbv1 {
+    const sbnn_packed* pw[SBNN_MBV1_NUM_BLOCKS];
+    const sbnn_packed* fc;
+    const float* dw_w[SBNN_MBV1_NUM_BLOCKS];
+    const float* dw_b[SBNN_MBV1_NUM_BLOCKS];
+    const float* c0_w;
+    const float* c0_b;
+    int max_batch;
+    int device;
+    float* ws[2];  // ping-pong activation buffers
+};
+
+using namespace sbnn;
+
+extern "C" sbnn_status sbnn_mobilenet_v1_layer_shape(int layer, int* Hin, int* Cin, int* Hout, int* Cout) {
+    clear_error();
+    if (layer < 0 || layer >= SBNN_MBV1_NUM_LAYERS) return fail(SBNN_ERR_SHAPE, "layer %d out of range", layer);
+    const LayerShape& L = layer_table()[layer];
+    if (Hin) *Hin = L.hin;
+    if (Cin) *Cin = L.cin;
+    if (Hout) *Hout = L.hout;
+    if (Cout) *Cout = L.cout;
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, const sbnn_packed* fc,
+                                                const float* const* dw_w_dev, const float* const* dw_b_dev,
+                                                const float* conv0_w_dev, const float* conv0_b_dev, int max_batch,
+                                                sbnn_mbv1** out) {
+    clear_error();
+    if (!pw || !fc || !dw_w_dev || !dw_b_dev || !conv0_w_dev || !conv0_b_dev || !out)
+        return fail(SBNN_ERR_NULL, "all arguments must be non-NULL");
+    *out = nullptr;
+    if (max_batch <= 0) return fail(SBNN_ERR_SHAPE, "max_batch=%d must be positive", max_batch);
+    const LayerShape* T = layer_table();
+    for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
+        const LayerShape& L = T[2 + 2 * i];
+        if (!pw[i] || !dw_w_dev[i] || !dw_b_dev[i]) return fail(SBNN_ERR_NULL, "block %d has a NULL weight pointer", i + 1);
+        if (pw[i]->KH != 1 || pw[i]->Cin != L.cin || pw[i]->Cout != L.cout)
+            return fail(SBNN_ERR_SHAPE, "pointwise layer %d is %d->%d (k=%d), expected %d->%d 1x1", i + 1, pw[i]->Cin,
+                        pw[i]->Cout, pw[i]->KH, L.cin, L.cout);
+        if (!aligned16(dw_w_dev[i]) || !aligned16(dw_b_dev[i]))
+            return fail(SBNN_ERR_ALIGN, "depthwise weights of block %d not 16-byte aligned", i + 1);
+    }
+    if (fc->KH != 1 || fc->Cin != 1024 || fc->Cout != 1000) return fail(SBNN_ERR_SHAPE, "classifier must be 1024->1000 1x1");
+    sbnn_status st = check_device();
+    if (st != SBNN_OK) return st;
+    sbnn_mbv1* n = new (std::nothrow) sbnn_mbv1;
+    if (!n) return fail(SBNN_ERR_ALLOC, "out of host memory");
+    for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
+        n->pw[i] = pw[i];
+        n->dw_w[i] = dw_w_dev[i];
+        n->dw_b[i] = dw_b_dev[i];
+    }
+    n->fc = fc; n->c0_w = conv0_w_dev; n->c0_b = conv0_b_dev; n->max_batch = max_batch;
+    n->ws[0] = n->ws[1] = nullptr;
+    cudaGetDevice(&n->device);
+    // Largest activation: pw1's output, 112*112*64 floats per image.
+    const size_t bytes = (size_t)max_batch * 112 * 112 * 64 * sizeof(float);
+    for (int i = 0; i < 2; ++i) {
+        cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&n->ws[i]), bytes);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            sbnn_mobilenet_v1_free(n);
+            return fail(SBNN_ERR_ALLOC, "workspace of %zu bytes: %s", bytes, cudaGetErrorString(e));
+        }
+    }
+    *out = n;
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_mobilenet_v1_run_layer(sbnn_mbv1* net, int layer, const float* in, float* outp, int N,
+                                                   void* stream) {
+    clear_error();
+    if (!net || !in || !outp) return fail(SBNN_ERR_NULL, "net, in_dev and out_dev must not be NULL");
+    if (layer < 0 || layer >= SBNN_MBV1_NUM_LAYERS) return fail(SBNN_ERR_SHAPE, "layer %d out of range", layer);
+    if (N < 0) return fail(SBNN_ERR_SHAPE, "N=%d", N);
+    const LayerShape& L = layer_table()[layer];
+    const int blk = (layer - 1) / 2;
+    switch (L.kind) {
+        case 0: return sbnn_conv3x3_dense(net->c0_w, net->c0_b, in, outp, N, L.hin, L.hin, L.cin, L.cout, L.stride, SBNN_RELU, stream);
+        case 1: return sbnn_dwconv3x3(net->dw_w[blk], net->dw_b[blk], in, outp, N, L.hin, L.hin, L.cin, L.stride, SBNN_RELU, stream);
+        case 2: return sbnn_conv1x1_gs(net->pw[blk], in, outp, N, L.hin, L.hin, SBNN_RELU, stream);
+        case 3: return sbnn_avgpool(in, outp, N, L.hin * L.hin, L.cin, stream);
+        default: return sbnn_conv1x1_gs(net->fc, in, outp, N, 1, 1, 0, stream);
+    }
+}
+
+extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_dev, float* logits_dev, int N,
+                                                 void* stream) {
+    clear_error();
+    if (!net || !x_dev || !logits_dev) return fail(SBNN_ERR_NULL, "net, x_dev and logits_dev must not be NULL");
+    if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
+    if (!aligned16(logits_dev)) return fail(SBNN_ERR_ALIGN, "logits_dev must be 16-byte aligned");
+    if (N == 0) return SBNN_OK;
+    const float* cur = x_dev;
+    for (int l = 0; l < SBNN_MBV1_NUM_LAYERS; ++l) {
+        float* dst = (l == SBNN_MBV1_NUM_LAYERS - 1) ? logits_dev : net->ws[l & 1];
+        sbnn_status st = sbnn_mobilenet_v1_run_layer(net, l, cur, dst, N, stream);
+        if (st != SBNN_OK) return st;
+        cur = dst;
+    }
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_mobilenet_v1_free(sbnn_mbv1* net) {
+    clear_error();
+    if (!net) return SBNN_OK;
+    cudaFree(net->ws[0]);
+    cudaFree(net->ws[1]);
+    cudaGetLastError();
+    delete net;
+    return SBNN_OK;
+}
