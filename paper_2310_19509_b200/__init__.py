@@ -1,0 +1,26 @@
+"""Group-sparse convolution for NVIDIA B200: thin ctypes binding over libsbnn.so.
+
+Every function here only marshals arguments into the C interface declared in
+include/sbnn.h; all arithmetic runs in the library's CUDA kernels.  There is
+no CPU fallback: if the shared library is missing, importing the binding's
+functions raises.
+"""
+from .binding import (  # noqa: F401
+    SBNN_BF16_TC,
+    SBNN_RELU,
+    MobileNetV1,
+    Packed,
+    SbnnError,
+    avgpool,
+    conv1x1_gs,
+    conv1x1_gs_tuned,
+    conv3x3_dense,
+    conv3x3_gs,
+    dwconv3x3,
+    get_async_status,
+    lib,
+    lib_path,
+    mobilenet_v1_layer_shape,
+    pack_weights,
+    status_str,
+)
