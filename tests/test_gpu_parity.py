@@ -1,0 +1,185 @@
+"""GPU parity: every CUDA entry point against the CPU oracle on the same seeded inputs.
+
+Tolerance (fp32 path): |gpu - ref| <= 1e-5 * S per output, S = |b| + sum |w*x| from the oracle.
+Packed indices are compared bit for bit in test_abi_cpu.py.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2310_19509_b200 as sbnn
+from oracle import reference as R
+from sbnn_inputs import workloads as WL
+from sbnn_inputs import mobilenet_v1_inputs
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def assert_within(y_gpu, ref, s, tol=TOL, what=""):
+    y = y_gpu.astype(np.float64)
+    assert y.shape == ref.shape, (y.shape, ref.shape)
+    assert np.all(np.isfinite(y)), what
+    ratio = np.abs(y - ref) / np.maximum(tol * s, 1e-300)
+    bad = np.abs(y - ref) > tol * s
+    assert not bad.any(), f"{what}: {bad.sum()} outputs outside tolerance, worst ratio {ratio[bad].max():.3g}"
+    return float(np.max(np.where(s > 0, np.abs(y - ref) / np.maximum(tol * s, 1e-300), 0.0)))
+
+
+def run_1x1(d, flags=sbnn.SBNN_RELU, cfg=None):
+    x = d["x"]
+    n, h, w, cin = x.shape
+    cout = d["w"].shape[0]
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], d["g"])
+    xd = dev(x)
+    yd = torch.full((n, h, w, cout), float("nan"), device="cuda", dtype=torch.float32)
+    if cfg is None:
+        sbnn.conv1x1_gs(p, xd, yd, n, h, w, flags)
+    else:
+        sbnn.conv1x1_gs_tuned(p, xd, yd, n, h, w, flags, *cfg)
+    sbnn.get_async_status()
+    y = yd.cpu().numpy()
+    p.free()
+    return y
+
+
+def test_config1_single_pointwise_layer():
+    d = WL.config1()
+    y = run_1x1(d)
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    worst = assert_within(y, ref, s, what="config 1")
+    assert worst < 0.5       # fp32 accumulation error is far inside the bound on these inputs
+
+
+CFGS = {1: [(8, 4, 8, 64)], 2: [(8, 2, 8, 64)],
+        4: [(8, 1, 16, 64), (8, 2, 8, 64), (8, 2, 16, 32), (4, 1, 8, 64), (4, 2, 8, 64)],
+        8: [(8, 1, 16, 32), (8, 1, 8, 64), (4, 1, 8, 64)], 16: [(4, 1, 8, 64)]}
+
+
+@pytest.mark.parametrize("g", [1, 2, 4, 8, 16])
+def test_every_kernel_instance_on_ragged_shapes(g):
+    """Several pixel tiles with a ragged tail, several channel steps with a ragged tail, a ragged group tile."""
+    for cfg in CFGS[g]:
+        tm = 32 * cfg[0]
+        d = WL.single_conv_inputs(1, 1, 2 * tm + 37, 148, 16 * 11, 1, g, 50, seed=3, mask_mode="layer_global")
+        for relu in (True, False):
+            y = run_1x1(d, sbnn.SBNN_RELU if relu else 0, cfg)
+            ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
+            assert_within(y, ref, s, what=f"G={g} cfg={cfg} relu={relu}")
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1, 4, 4), (1, 7, 7, 12, 8), (2, 3, 5, 32, 64), (1, 1, 300, 8, 1000)])
+def test_small_and_odd_shapes(shape):
+    n, h, w, cin, cout = shape
+    for sp in (0, 50, 100):
+        d = WL.single_conv_inputs(n, h, w, cin, cout, 1, 4, sp, seed=5)
+        y = run_1x1(d)
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+        assert_within(y, ref, s, what=f"{shape} sp={sp}")
+
+
+def test_group_without_kept_units_and_zero_bias_gives_exact_zero():
+    d = WL.single_conv_inputs(1, 5, 5, 16, 16, 1, 4, 50, seed=2)
+    d["mask"][4:8] = 0
+    d["bias"][4:8] = 0.0
+    y = run_1x1(d, 0)
+    assert not y[..., 4:8].any()
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=False)
+    assert_within(y, ref, s)
+
+
+def test_paper_style_4x4_blocks_and_magnitude_masks():
+    for mode, gi in (("balanced", 4), ("magnitude", 1)):
+        d = WL.single_conv_inputs(1, 9, 13, 64, 64, 1, 4, 30, seed=9, mask_mode=mode, gi=gi)
+        y = run_1x1(d)
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+        assert_within(y, ref, s, what=mode)
+
+
+def test_empty_batch_is_ok():
+    d = WL.single_conv_inputs(1, 1, 1, 8, 8, 1, 4, 50)
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    x = torch.zeros(16, device="cuda")
+    sbnn.conv1x1_gs(p, x, x, 0, 5, 5)
+
+
+@pytest.mark.parametrize("stride", [1, 2])
+@pytest.mark.parametrize("shape", [(2, 9, 11, 32), (1, 14, 14, 512), (1, 1, 1, 4), (1, 7, 7, 8)])
+def test_depthwise(stride, shape):
+    n, h, w, c = shape
+    rng = np.random.default_rng(11)
+    x = rng.random((n, h, w, c), dtype=np.float32)
+    wt = rng.standard_normal((3, 3, c)).astype(np.float32)
+    b = rng.standard_normal(c).astype(np.float32)
+    ho, wo = (h - 1) // stride + 1, (w - 1) // stride + 1
+    yd = torch.full((n, ho, wo, c), float("nan"), device="cuda")
+    sbnn.dwconv3x3(dev(wt), dev(b), dev(x), yd, n, h, w, c, stride)
+    sbnn.get_async_status()
+    ref, s = R.dwconv3x3(x, wt, b, stride=stride, relu=True)
+    assert_within(yd.cpu().numpy(), ref, s, what=f"dw {shape} s{stride}")
+
+
+@pytest.mark.parametrize("stride,shape", [(2, (2, 32, 32, 3, 32)), (1, (1, 9, 7, 3, 32)), (2, (1, 15, 17, 4, 8))])
+def test_thin_dense_conv(stride, shape):
+    n, h, w, cin, cout = shape
+    rng = np.random.default_rng(12)
+    x = rng.random((n, h, w, cin), dtype=np.float32)
+    wt = rng.standard_normal((cout, 3, 3, cin)).astype(np.float32)
+    b = rng.standard_normal(cout).astype(np.float32)
+    ho, wo = (h - 1) // stride + 1, (w - 1) // stride + 1
+    yd = torch.full((n, ho, wo, cout), float("nan"), device="cuda")
+    sbnn.conv3x3_dense(dev(wt), dev(b), dev(x), yd, n, h, w, cin, cout, stride)
+    sbnn.get_async_status()
+    ref, s = R.conv2d(x, wt, np.ones_like(wt, dtype=np.uint8), b, stride=stride, relu=True)
+    assert_within(yd.cpu().numpy(), ref, s, what=f"conv0 {shape}")
+
+
+def test_avgpool():
+    rng = np.random.default_rng(13)
+    x = rng.standard_normal((3, 7, 7, 64)).astype(np.float32)
+    yd = torch.full((3, 64), float("nan"), device="cuda")
+    sbnn.avgpool(dev(x), yd, 3, 49, 64)
+    ref, s = R.avgpool(x)
+    assert_within(yd.cpu().numpy(), ref, s, what="avgpool")
+
+
+def build_net(layers, max_batch):
+    pw = [sbnn.pack_weights(L["w"], L["mask"], L["bias"], L["g"]) for L in layers if L["kind"] == "pw"]
+    fcL = [L for L in layers if L["kind"] == "fc"][0]
+    fc = sbnn.pack_weights(fcL["w"], fcL["mask"], fcL["bias"], fcL["g"])
+    dw_w = [dev(L["w"]) for L in layers if L["kind"] == "dw"]
+    dw_b = [dev(L["bias"]) for L in layers if L["kind"] == "dw"]
+    c0 = layers[0]
+    return sbnn.MobileNetV1(pw, fc, dw_w, dw_b, dev(c0["w"]), dev(c0["bias"]), max_batch)
+
+
+@pytest.mark.parametrize("sparsity", [30])
+def test_mobilenet_v1_batch1_layer_isolated_and_end_to_end(sparsity):
+    x, layers = mobilenet_v1_inputs(1, sparsity, 4, seed=0)
+    outs = R.mobilenet_v1_forward(x, layers)
+    net = build_net(layers, 2)
+    # (i) every layer alone, fed the oracle's fp32 input of that layer
+    for li, rec in enumerate(outs):
+        ref, s = rec["ref"], rec["S"]
+        yd = torch.full(ref.shape, float("nan"), device="cuda", dtype=torch.float32)
+        net.run_layer(li, dev(rec["in"]), yd, 1)
+        sbnn.get_async_status()
+        assert_within(yd.cpu().numpy(), ref, s, what=f"layer {li} {rec['name']}")
+    # (ii) the chain, against the propagated first-order bound
+    logits = torch.full((1, 1000), float("nan"), device="cuda")
+    net.forward(dev(x), logits, 1)
+    sbnn.get_async_status()
+    y = logits.cpu().numpy().astype(np.float64).reshape(outs[-1]["ref"].shape)
+    err = np.abs(y - outs[-1]["ref"])
+    assert np.all(err <= outs[-1]["E"]), f"worst ratio {np.max(err / outs[-1]['E'])}"
+    # two images in one call give the single-image result twice
+    x2 = np.concatenate([x, x])
+    l2 = torch.full((2, 1000), float("nan"), device="cuda")
+    net.forward(dev(x2), l2, 2)
+    sbnn.get_async_status()
+    assert torch.equal(l2[0], l2[1]) and torch.equal(l2[0], logits[0])
+    net.free()
