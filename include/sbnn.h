@@ -139,6 +139,8 @@ SBNN_API sbnn_status sbnn_conv1x1_gs_tuned(const sbnn_packed* w, const float* x_
  * 3x3, stride 1, pad 1:
  * Y[n][y][x][g*G + r] = act( bias + sum_j sum_{kh,kw} val[g][j][kh*3+kw][r] * X[n][y+kh-1][x+kw-1][idx[g][j]] ),
  * X taken as zero outside the image.  Shapes as above with KH = KW = 3.  SBNN_BF16_TC is not accepted.
+ * W <= 256 and Cin a multiple of 4, else SBNN_ERR_UNSUPPORTED.  The first call with a new image width
+ * builds a private re-layout of the weights (allocates and copies synchronously); later calls only enqueue.
  */
 SBNN_API sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev, float* y_dev,
                                      int N, int H, int W, int flags, void* cuda_stream);

@@ -1,11 +1,366 @@
-// Group-sparse 3x3 convolution (placeholder until the kernel lands).
+// Group-sparse 3x3 convolution, stride 1, pad 1, fp32: whole 3x3 kernels of one input channel are
+// kept or removed jointly for a group of G output channels (connectivity group pruning, Section 3.2).
+//
+//   Y[n][y][x][g*G+r] = act( b + sum_j sum_{kh,kw} val[g][j][kh*3+kw][r] * X[n][y+kh-1][x+kw-1][idx[g][j]] )
+//
+// Work decomposition
+//   * Image rows of the whole batch are numbered f = n*H + y.  A CTA owns R consecutive rows f and GT
+//     consecutive groups, and walks the input channels in steps of KC.
+//   * Per step the rows f0-1 .. f0+R of KC channels are staged in shared memory as one plane per
+//     channel ([row][column], column = x + 1, so that x = -1 and x = W are zero columns).  Row 0 of
+//     every plane is an all-zero row: a lane whose image row is the first (last) of its image reads
+//     that row instead of the row above (below), which gives the vertical padding without branches
+//     and lets a CTA's rows span several images.
+//   * A lane owns CW consecutive output columns of one row (CW = 7 or 8, chosen so that the lanes of
+//     a row tile the width with least waste; ImageNet-style maps have W = 7 * 2^k), a warp owns 32/LPR
+//     rows (LPR lanes per row), and keeps CW x G x GPW partial sums in registers.  Per kept unit and
+//     kernel row a lane reads CW+2 activations and feeds 3*CW*G FMAs; the 9*G weights of the unit are
+//     broadcast reads.  The plane pitch is picked on the host so that the 32 lanes of a warp hit 32
+//     different banks.
+#include <string.h>
+
+#include <algorithm>
+
 #include "common.h"
+
 namespace sbnn {
-sbnn_status prepare_default_3x3(const sbnn_packed*) { return SBNN_OK; }
-void free_streams_3x3(sbnn_packed*) {}
+namespace {
+
+struct Geo3 {
+    int N, H, W, Cin, Cout, ngroups;
+    int LPR, RPW, R;        // lanes per row, rows per warp, rows per CTA
+    int pitch, plane;       // floats
+    int nchunks;
+    int dpp_row, dpp_x;     // how (row, x) advance when a thread's staged pixel index grows by its stride
+};
+
+template <int G_, int CW_, int GPW_, int NPW_, int NGW_, int KC_>
+struct K3 {
+    static constexpr int G = G_, CW = CW_, GPW = GPW_, NPW = NPW_, NGW = NGW_, KC = KC_;
+    static constexpr int NW = NPW * NGW, NT = NW * 32, GT = NGW * GPW;
+    static constexpr int UNIT = 1 + (9 * G + 3) / 4;   // record of one kept unit, 16-byte units
+    static constexpr int HDR = (GT * 2 + 3) / 4;
+    static constexpr int WS_U4 = HDR + GT * KC * UNIT;
+    static_assert(KC % 4 == 0, "KC");
+};
+
+template <class C>
+__global__ void __launch_bounds__(C::NT, 1)
+conv3x3_gs_kernel(const float* __restrict__ X, float* __restrict__ Y, const float* __restrict__ bias,
+                  const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, Geo3 geo, int relu) {
+    constexpr int G = C::G, CW = C::CW, GPW = C::GPW, KC = C::KC;
+    extern __shared__ __align__(16) unsigned char smem[];
+    float* xs = reinterpret_cast<float*>(smem);                                  // [KC][plane]
+    uint4* ws = reinterpret_cast<uint4*>(smem + (size_t)KC * geo.plane * 4);     // weight block
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pw = warp % C::NPW, gw = warp / C::NPW;
+    const int f0 = blockIdx.x * geo.R;
+    const int tile = blockIdx.y;
+    const int NH = geo.N * geo.H, W = geo.W, Cin = geo.Cin;
+    const int32_t* bp = blk_ptr + (size_t)tile * (geo.nchunks + 1);
+
+    // zero the planes once: zero rows, zero columns and rows outside the batch stay zero for good
+    for (int i = tid; i < KC * geo.plane; i += C::NT) xs[i] = 0.0f;
+
+    // this lane's pixels
+    const int lrow = pw * geo.RPW + lane / geo.LPR;   // row inside the CTA tile
+    const int lx = (lane % geo.LPR) * CW;             // first output column
+    const int f = f0 + lrow;
+    const int y = f % geo.H;
+    // plane row r holds image row f0 - 2 + r  (r = 0 is the zero row)
+    int rowoff[3];
+    rowoff[0] = (y > 0) ? (lrow + 1) * geo.pitch : 0;
+    rowoff[1] = (lrow + 2) * geo.pitch;
+    rowoff[2] = (y < geo.H - 1) ? (lrow + 3) * geo.pitch : 0;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) rowoff[k] += lx;
+
+    float acc[GPW][CW][G];
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * C::GT + gw * GPW + q;
+#pragma unroll
+        for (int r = 0; r < G; ++r) {
+            const float b = (g < geo.ngroups) ? bias[g * G + r] : 0.0f;
+#pragma unroll
+            for (int p = 0; p < CW; ++p) acc[q][p][r] = b;
+        }
+    }
+
+    // staging: a thread owns channel quad (tid % (KC/4)) of pixels tid/(KC/4) + j*stride
+    constexpr int QPP = KC / 4;                 // float4 loads per pixel and step
+    constexpr int PSTRIDE = C::NT / QPP;        // pixel stride between a thread's loads
+    static_assert(C::NT % QPP == 0, "staging split");
+    const int cq = tid % QPP;
+    const int npix = (geo.R + 2) * W;           // pixels of rows f0-1 .. f0+R
+    const long long pix0 = (long long)(f0 - 1) * W;   // global pixel index of the first staged pixel
+
+    for (int k = 0; k < geo.nchunks; ++k) {
+        __syncthreads();   // previous step's reads are done (and the zero fill, first time)
+        {
+            const int beg = bp[k], n = bp[k + 1] - beg;
+            for (int i = tid; i < n; i += C::NT) ws[i] = rec[beg + i];
+            const int c = k * KC + cq * 4;
+            int pp = tid / QPP;
+            int prow = pp / W, px = pp - prow * W;
+            for (; pp < npix; pp += PSTRIDE) {
+                const long long gp = pix0 + pp;
+                if (c < Cin && gp >= 0 && gp < (long long)NH * W) {
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(X + (size_t)gp * Cin + c));
+                    float* d = xs + (size_t)(cq * 4) * geo.plane + (prow + 1) * geo.pitch + px + 1;
+                    d[0] = v.x;
+                    d[geo.plane] = v.y;
+                    d[2 * geo.plane] = v.z;
+                    d[3 * geo.plane] = v.w;
+                }
+                prow += geo.dpp_row;
+                px += geo.dpp_x;
+                if (px >= W) { px -= W; ++prow; }
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < GPW; ++q) {
+            const int2 hd = reinterpret_cast<const int2*>(ws)[gw * GPW + q];   // (start, units)
+            const uint4* r = ws + hd.x;
+            for (int it = 0; it < hd.y; ++it, r += C::UNIT) {
+                const float* plane = xs + r[0].x;                 // plane offset in floats
+                const float* wq = reinterpret_cast<const float*>(r + 1);   // [9][G]
+#pragma unroll
+                for (int kh = 0; kh < 3; ++kh) {
+                    const float* arow = plane + rowoff[kh];
+                    float a[CW + 2];
+#pragma unroll
+                    for (int i = 0; i < CW + 2; ++i) a[i] = arow[i];
+#pragma unroll
+                    for (int kw = 0; kw < 3; ++kw) {
+                        float w[G];
+                        if constexpr (G % 4 == 0) {
+#pragma unroll
+                            for (int v = 0; v < G / 4; ++v) {
+                                const float4 t = reinterpret_cast<const float4*>(wq + (kh * 3 + kw) * G)[v];
+                                w[4 * v] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int rr = 0; rr < G; ++rr) w[rr] = wq[(kh * 3 + kw) * G + rr];
+                        }
+#pragma unroll
+                        for (int p = 0; p < CW; ++p)
+#pragma unroll
+                            for (int rr = 0; rr < G; ++rr) acc[q][p][rr] = fmaf(a[p + kw], w[rr], acc[q][p][rr]);
+                    }
+                }
+            }
+        }
+    }
+
+    if (f >= NH || lrow >= geo.R) return;
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * C::GT + gw * GPW + q;
+        if (g >= geo.ngroups) continue;
+#pragma unroll
+        for (int p = 0; p < CW; ++p) {
+            const int x = lx + p;
+            if (x >= W) continue;
+            float* yp = Y + ((size_t)f * W + x) * geo.Cout + g * G;
+            float v[G];
+#pragma unroll
+            for (int rr = 0; rr < G; ++rr) v[rr] = relu ? fmaxf(acc[q][p][rr], 0.0f) : acc[q][p][rr];
+            if constexpr (G >= 4) {
+#pragma unroll
+                for (int vv = 0; vv < G / 4; ++vv)
+                    reinterpret_cast<float4*>(yp)[vv] = make_float4(v[4 * vv], v[4 * vv + 1], v[4 * vv + 2], v[4 * vv + 3]);
+            } else if constexpr (G == 2) {
+                *reinterpret_cast<float2*>(yp) = make_float2(v[0], v[1]);
+            } else {
+                yp[0] = v[0];
+            }
+        }
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------
+
+int pow2_ceil(int v) {
+    int p = 1;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+// Lanes per row for a column width; 0 if the image is too wide for one warp row.
+int lanes_per_row(int W, int CW) {
+    const int l = pow2_ceil((W + CW - 1) / CW);
+    return l <= 32 ? l : 0;
+}
+
+// Smallest pitch >= LPR*CW+2 for which the first reads of the 32 lanes fall into 32 distinct banks.
+int pick_pitch(int LPR, int CW) {
+    const int lo = LPR * CW + 2;
+    for (int p = lo; p < lo + 64; ++p) {
+        unsigned used = 0;
+        bool ok = true;
+        for (int l = 0; l < 32 && ok; ++l) {
+            const int b = ((l / LPR) * p + (l % LPR) * CW) & 31;
+            ok = !((used >> b) & 1u);
+            used |= 1u << b;
+        }
+        if (ok) return p;
+    }
+    return lo;
+}
+
+// Record stream: block (tile t, step k) = GT (start, units) pairs, then per group its units:
+// one 16-byte word whose first lane is the plane offset in floats, then the 9*G weights.
+sbnn_status build_stream3(const sbnn_packed* p, int GT, int KC, int plane, Stream3x3* out) {
+    const int G = p->G;
+    const int ntiles = (p->ngroups + GT - 1) / GT, nchunks = (p->Cin + KC - 1) / KC;
+    const int HDR = (GT * 2 + 3) / 4, UNIT = 1 + (9 * G + 3) / 4;
+    std::vector<int32_t> blk((size_t)ntiles * (nchunks + 1));
+    std::vector<uint32_t> rec;
+    int max_blk = 0;
+    try {
+        for (int t = 0; t < ntiles; ++t) {
+            for (int k = 0; k < nchunks; ++k) {
+                const size_t blk_beg = rec.size() / 4;
+                blk[(size_t)t * (nchunks + 1) + k] = (int32_t)blk_beg;
+                rec.resize(rec.size() + (size_t)HDR * 4, 0u);
+                for (int s = 0; s < GT; ++s) {
+                    const int g = t * GT + s;
+                    int lo = 0, hi = 0;
+                    if (g < p->ngroups) {
+                        const int32_t* b = p->idx.data() + p->group_ptr[g];
+                        const int32_t* e = p->idx.data() + p->group_ptr[g + 1];
+                        lo = (int)(std::lower_bound(b, e, k * KC) - p->idx.data());
+                        hi = (int)(std::lower_bound(b, e, (k + 1) * KC) - p->idx.data());
+                    }
+                    rec[blk_beg * 4 + 2 * s + 0] = (uint32_t)(rec.size() / 4 - blk_beg);
+                    rec[blk_beg * 4 + 2 * s + 1] = (uint32_t)(hi - lo);
+                    for (int j = lo; j < hi; ++j) {
+                        const size_t base = rec.size();
+                        rec.resize(base + (size_t)UNIT * 4, 0u);
+                        rec[base] = (uint32_t)((p->idx[j] - k * KC) * plane);
+                        memcpy(&rec[base + 4], &p->val[(size_t)j * 9 * G], sizeof(float) * 9 * G);
+                    }
+                }
+                max_blk = std::max(max_blk, (int)(rec.size() / 4 - blk_beg));
+            }
+            blk[(size_t)t * (nchunks + 1) + nchunks] = (int32_t)(rec.size() / 4);
+        }
+    } catch (const std::bad_alloc&) {
+        return fail(SBNN_ERR_ALLOC, "out of host memory building the 3x3 weight stream");
+    }
+    Stream3x3 s;
+    s.ntiles = ntiles; s.nchunks = nchunks; s.max_blk = max_blk;
+    SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&s.rec), std::max<size_t>(rec.size() * 4, 16)));
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s.blk_ptr), blk.size() * 4);
+    if (e == cudaSuccess && !rec.empty()) e = cudaMemcpy(s.rec, rec.data(), rec.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(s.blk_ptr, blk.data(), blk.size() * 4, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(s.rec);
+        cudaFree(s.blk_ptr);
+        cudaGetLastError();
+        return fail(SBNN_ERR_CUDA, "uploading the 3x3 weight stream: %s", cudaGetErrorString(e));
+    }
+    *out = s;
+    return SBNN_OK;
+}
+
+template <class C>
+sbnn_status launch3(const sbnn_packed* p, const float* x, float* y, int N, int H, int W, int relu, cudaStream_t st) {
+    Geo3 g;
+    g.N = N; g.H = H; g.W = W; g.Cin = p->Cin; g.Cout = p->Cout; g.ngroups = p->ngroups;
+    g.LPR = lanes_per_row(W, C::CW);
+    g.RPW = 32 / g.LPR;
+    g.R = C::NPW * g.RPW;
+    g.pitch = pick_pitch(g.LPR, C::CW);
+    int plane = (g.R + 3) * g.pitch;
+    plane = (plane + 7) / 8 * 8 + 4;   // multiple of 4 floats, and 4 (mod 8) to spread the staging stores over banks
+    g.plane = plane;
+    g.nchunks = (p->Cin + C::KC - 1) / C::KC;
+    constexpr int PSTRIDE = C::NT / (C::KC / 4);
+    g.dpp_row = PSTRIDE / W;
+    g.dpp_x = PSTRIDE % W;
+    const size_t smem = (size_t)C::KC * plane * 4 + (size_t)C::WS_U4 * 16;
+    if (smem > 227 * 1024) return fail(SBNN_ERR_UNSUPPORTED, "3x3 tile for W=%d needs %zu bytes of shared memory", W, smem);
+
+    // the stream's plane offsets depend on the plane size, hence on (W, tile shape)
+    Stream3x3 s;
+    {
+        std::lock_guard<std::mutex> lk(p->mu);
+        const int key = (plane << 8) | (C::GT << 4) | (C::KC / 4);
+        auto it = p->streams3x3.find(key);
+        if (it == p->streams3x3.end()) {
+            sbnn_status r = build_stream3(p, C::GT, C::KC, plane, &s);
+            if (r != SBNN_OK) return r;
+            p->streams3x3[key] = s;
+        } else {
+            s = it->second;
+        }
+    }
+    if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
+    SBNN_CUDA_TRY(cudaFuncSetAttribute(conv3x3_gs_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const long long NH = (long long)N * H;
+    dim3 grid((unsigned)((NH + g.R - 1) / g.R), s.ntiles);
+    conv3x3_gs_kernel<C><<<grid, C::NT, smem, st>>>(x, y, p->d_bias, s.rec, s.blk_ptr, g, relu);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    return SBNN_OK;
+}
+
+// Column width per lane: the one that tiles the row with least waste (ties go to 8).
+int choose_cw(int W) {
+    const int l7 = lanes_per_row(W, 7), l8 = lanes_per_row(W, 8);
+    if (!l7 && !l8) return 0;
+    if (!l7) return 8;
+    if (!l8) return 7;
+    return (l7 * 7 < l8 * 8) ? 7 : 8;
+}
+
+template <int CW>
+sbnn_status dispatch3(const sbnn_packed* p, const float* x, float* y, int N, int H, int W, int relu, cudaStream_t st) {
+    switch (p->G) {
+        case 1: return launch3<K3<1, CW, 4, 7, 2, 8>>(p, x, y, N, H, W, relu, st);
+        case 2: return launch3<K3<2, CW, 4, 7, 2, 8>>(p, x, y, N, H, W, relu, st);
+        case 4: return launch3<K3<4, CW, 2, 7, 2, 8>>(p, x, y, N, H, W, relu, st);
+        case 8: return launch3<K3<8, CW, 1, 7, 2, 8>>(p, x, y, N, H, W, relu, st);
+        default: return launch3<K3<16, CW, 1, 7, 1, 8>>(p, x, y, N, H, W, relu, st);
+    }
+}
+}  // namespace
+
+sbnn_status prepare_default_3x3(const sbnn_packed*) { return SBNN_OK; }  // the re-layout depends on the image width
+
+void free_streams_3x3(sbnn_packed* p) {
+    for (auto& kv : p->streams3x3) {
+        cudaFree(kv.second.rec);
+        cudaFree(kv.second.blk_ptr);
+    }
+    p->streams3x3.clear();
+}
+
 }  // namespace sbnn
+
 using namespace sbnn;
-extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed*, const float*, float*, int, int, int, int, void*) {
+
+extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev, float* y_dev, int N, int H, int W,
+                                       int flags, void* cuda_stream) {
     clear_error();
-    return fail(SBNN_ERR_UNSUPPORTED, "3x3 kernel not built yet");
+    if (!w || !x_dev || !y_dev) return fail(SBNN_ERR_NULL, "packed weights, x_dev and y_dev must not be NULL");
+    if (w->KH != 3 || w->KW != 3) return fail(SBNN_ERR_SHAPE, "packed layer is %dx%d, expected 3x3", w->KH, w->KW);
+    if (N < 0 || H < 0 || W < 0) return fail(SBNN_ERR_SHAPE, "negative activation shape %dx%dx%d", N, H, W);
+    if ((int64_t)N * H * W > 0x7fffffff) return fail(SBNN_ERR_SHAPE, "N*H*W exceeds 2^31-1");
+    if (flags & ~SBNN_RELU) return fail(SBNN_ERR_UNSUPPORTED, "flag bits 0x%x not accepted by the 3x3 kernel", flags);
+    if (!aligned16(x_dev) || !aligned16(y_dev)) return fail(SBNN_ERR_ALIGN, "x_dev and y_dev must be 16-byte aligned");
+    if (w->Cin % 4) return fail(SBNN_ERR_UNSUPPORTED, "Cin=%d is not a multiple of 4", w->Cin);
+    if (w->device < 0) return fail(SBNN_ERR_CUDA, "packed weights have no device copy (packed without a CUDA device)");
+    if ((int64_t)N * H * W == 0) return SBNN_OK;
+    const int cw = choose_cw(W);
+    if (!cw) return fail(SBNN_ERR_UNSUPPORTED, "W=%d: the 3x3 kernel handles rows of at most 256 pixels", W);
+    sbnn_status st = check_device();
+    if (st != SBNN_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    return cw == 7 ? dispatch3<7>(w, x_dev, y_dev, N, H, W, flags & SBNN_RELU, s)
+                   : dispatch3<8>(w, x_dev, y_dev, N, H, W, flags & SBNN_RELU, s);
 }

@@ -183,3 +183,45 @@ def test_mobilenet_v1_batch1_layer_isolated_and_end_to_end(sparsity):
     sbnn.get_async_status()
     assert torch.equal(l2[0], l2[1]) and torch.equal(l2[0], logits[0])
     net.free()
+
+
+def run_3x3(d, flags=sbnn.SBNN_RELU):
+    x = d["x"]
+    n, h, w, cin = x.shape
+    cout = d["w"].shape[0]
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], d["g"])
+    yd = torch.full((n, h, w, cout), float("nan"), device="cuda", dtype=torch.float32)
+    sbnn.conv3x3_gs(p, dev(x), yd, n, h, w, flags)
+    sbnn.get_async_status()
+    y = yd.cpu().numpy()
+    p.free()
+    return y
+
+
+def test_config4_group_sparse_3x3_reduced_batch():
+    """Config 4's layer (28x28, 256 -> 256, G=4, half of the kernels removed) on 3 images: the CTA tiles of
+    56 image rows span image boundaries, with a ragged last tile."""
+    d = WL.config4(n=3)
+    y = run_3x3(d)
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    worst = assert_within(y, ref, s, what="config 4 (n=3)")
+    assert worst < 0.5
+
+
+@pytest.mark.parametrize("g", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("hw", [(5, 5), (9, 13), (14, 14), (7, 32), (3, 57), (6, 100)])
+def test_3x3_shapes_and_groups(g, hw):
+    h, w = hw
+    d = WL.single_conv_inputs(2, h, w, 20, 48, 3, g, 50, seed=4, w_sigma=0.1, mask_mode="layer_global")
+    for relu in (True, False):
+        y = run_3x3(d, sbnn.SBNN_RELU if relu else 0)
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
+        assert_within(y, ref, s, what=f"3x3 G={g} {hw} relu={relu}")
+
+
+def test_3x3_dense_and_empty_masks():
+    for sp in (0, 100):
+        d = WL.single_conv_inputs(1, 8, 8, 8, 8, 3, 4, sp, seed=6)
+        y = run_3x3(d)
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+        assert_within(y, ref, s, what=f"3x3 sp={sp}")
