@@ -217,6 +217,33 @@ SBNN_API sbnn_status sbnn_mobilenet_v1_layer_shape(int layer, int* Hin, int* Cin
 SBNN_API sbnn_status sbnn_mobilenet_v1_free(sbnn_mbv1* net);
 
 /*
+ * Classifier head without any allocation: logits = classifier(mean over HW of x).
+ * (The paper has no counterpart; this entry point exists for deployment only.)
+ *
+ * Who needs it: callers that may not allocate device memory at the point where they run the head --
+ * a serving loop with a latency budget that a cudaMalloc (an implicit device synchronisation) would
+ * break, a plug-in living inside another framework's capped memory pool, an application that has
+ * frozen its device memory map after start-up.  The ordinary route (sbnn_avgpool, then
+ * sbnn_conv1x1_gs) needs a pooled [N][Cin] buffer from the caller; here that buffer is a fixed
+ * array of SBNN_HEAD_NOALLOC_MAX_FLOATS floats (256 KiB) inside the library image, resident on every
+ * GPU that loads the library until the process exits.
+ *
+ *   fc          packed 1x1 classifier (any Cout; Cin a multiple of 4), packed while a device was present
+ *   x_dev       [N][HW][Cin] fp32, logits_dev [N][Cout] fp32; no ReLU
+ *   N * Cin must not exceed SBNN_HEAD_NOALLOC_MAX_FLOATS (e.g. 64 images x 1024 channels), else
+ *   SBNN_ERR_SHAPE and nothing is launched.
+ * The call uses no cudaMalloc/cudaFree and no allocating library routine; it enqueues two kernels.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, once per
+ * device): make that first call outside of any stream capture.  All calls on a device share the one
+ * array, which keeps the previous call's values (every element read is rewritten first, nothing
+ * needs to start at zero): two calls whose kernels may overlap on the GPU (different streams) race
+ * on it -- keep calls on one stream or order them with events.
+ */
+#define SBNN_HEAD_NOALLOC_MAX_FLOATS 65536
+SBNN_API sbnn_status sbnn_head_noalloc(const sbnn_packed* fc, const float* x_dev, float* logits_dev,
+                                       int N, int HW, void* cuda_stream);
+
+/*
  * Synchronise the stream and report device-side trouble: SBNN_ERR_CUDA if a kernel failed,
  * SBNN_ERR_TIMEOUT if a bounded wait inside a kernel expired, else SBNN_OK.
  */

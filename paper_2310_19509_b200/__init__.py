@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     conv3x3_gs,
     dwconv3x3,
     get_async_status,
+    head_noalloc,
     lib,
     lib_path,
     mobilenet_v1_layer_shape,

@@ -55,6 +55,7 @@ def lib():
         "sbnn_mobilenet_v1_layer_shape": [I, P, P, P, P],
         "sbnn_mobilenet_v1_free": [P],
         "sbnn_get_async_status": [P],
+        "sbnn_head_noalloc": [P, P, P, I, I, P],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -176,6 +177,11 @@ def conv3x3_dense(w, b, x, y, n, h, wd, cin, cout, stride, flags=SBNN_RELU, stre
 
 def avgpool(x, y, n, hw, c, stream=None):
     _check(lib().sbnn_avgpool(_ptr(x), _ptr(y), n, hw, c, _stream(stream)))
+
+
+def head_noalloc(fc: Packed, x, logits, n, hw, stream=None):
+    """Average pool + classifier through the library's fixed scratch array; allocates nothing."""
+    _check(lib().sbnn_head_noalloc(fc.handle, _ptr(x), _ptr(logits), n, hw, _stream(stream)))
 
 
 def get_async_status(stream=None):
