@@ -112,7 +112,8 @@ SBNN_API sbnn_status sbnn_packed_free(sbnn_packed* p);
 
 enum {
     SBNN_RELU = 1,    /* apply max(.,0) after the bias */
-    SBNN_BF16_TC = 2  /* 1x1 only: round activations and weights to bf16 and contract on tensor cores, fp32 accumulate */
+    SBNN_BF16_TC = 2, /* 1x1 only: round activations and weights to bf16 and contract on tensor cores, fp32 accumulate */
+    SBNN_OUT_CM = 4   /* sbnn_conv1x1_gs_cm only: write the output channel-major, [Cout][ldy] */
 };
 
 /*
@@ -134,6 +135,23 @@ SBNN_API sbnn_status sbnn_conv1x1_gs(const sbnn_packed* w, const float* x_dev, f
 SBNN_API sbnn_status sbnn_conv1x1_gs_tuned(const sbnn_packed* w, const float* x_dev, float* y_dev,
                                            int N, int H, int W, int flags, int P, int GPW, int NW, int KC,
                                            void* cuda_stream);
+
+/*
+ * Channel-major variant of the 1x1 convolution (same arithmetic as sbnn_conv1x1_gs): the activations
+ * are given as xt_dev [Cin][ldx] with the M = N*H*W pixels of a channel contiguous (ldx >= M, a multiple
+ * of 4; the padding need not be initialised).  In this layout the kernel's shared-memory tiles are
+ * filled by bulk asynchronous copies, which is the fast path for layers bound by arithmetic.
+ *   output: y_dev [M][ldy] (pixel-major rows of ldy >= Cout floats), or, with SBNN_OUT_CM, [Cout][ldy]
+ *   with ldy >= M; ldy a multiple of 4 in both cases.
+ *   P, GPW, NW, KC: tile shape as in sbnn_conv1x1_gs_tuned, or all 0 for the default of the layer.
+ * sbnn_conv1x1_gs itself takes this path for wide layers (Cin >= 128, M >= 4096): it first copies X
+ * into a channel-major scratch buffer kept per device, which it allocates or grows (synchronously) the
+ * first time a size is seen.
+ * sbnn_to_channel_major converts x_dev [M][C] to xt_dev [C][ld].
+ */
+SBNN_API sbnn_status sbnn_conv1x1_gs_cm(const sbnn_packed* w, const float* xt_dev, int ldx, float* y_dev, int ldy,
+                                        int M, int flags, int P, int GPW, int NW, int KC, void* cuda_stream);
+SBNN_API sbnn_status sbnn_to_channel_major(const float* x_dev, float* xt_dev, int M, int C, int ld, void* cuda_stream);
 
 /*
  * 3x3, stride 1, pad 1:

@@ -7,12 +7,14 @@ functions raises.
 """
 from .binding import (  # noqa: F401
     SBNN_BF16_TC,
+    SBNN_OUT_CM,
     SBNN_RELU,
     MobileNetV1,
     Packed,
     SbnnError,
     avgpool,
     conv1x1_gs,
+    conv1x1_gs_cm,
     conv1x1_gs_tuned,
     conv3x3_dense,
     conv3x3_gs,
@@ -24,4 +26,5 @@ from .binding import (  # noqa: F401
     mobilenet_v1_layer_shape,
     pack_weights,
     status_str,
+    to_channel_major,
 )

@@ -7,7 +7,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-SBNN_RELU, SBNN_BF16_TC = 1, 2
+SBNN_RELU, SBNN_BF16_TC, SBNN_OUT_CM = 1, 2, 4
 _lib = None
 
 
@@ -46,6 +46,8 @@ def lib():
         "sbnn_conv1x1_gs": [P, P, P, I, I, I, I, P],
         "sbnn_conv1x1_gs_tuned": [P, P, P, I, I, I, I, I, I, I, I, P],
         "sbnn_conv3x3_gs": [P, P, P, I, I, I, I, P],
+        "sbnn_conv1x1_gs_cm": [P, P, I, P, I, I, I, I, I, I, I, P],
+        "sbnn_to_channel_major": [P, P, I, I, I, P],
         "sbnn_dwconv3x3": [P, P, P, P, I, I, I, I, I, I, P],
         "sbnn_conv3x3_dense": [P, P, P, P, I, I, I, I, I, I, I, P],
         "sbnn_avgpool": [P, P, I, I, I, P],
@@ -160,6 +162,14 @@ def conv1x1_gs(w: Packed, x, y, n, h, wd, flags=SBNN_RELU, stream=None):
 
 def conv1x1_gs_tuned(w: Packed, x, y, n, h, wd, flags, p, gpw, nw, kc, stream=None):
     _check(lib().sbnn_conv1x1_gs_tuned(w.handle, _ptr(x), _ptr(y), n, h, wd, flags, p, gpw, nw, kc, _stream(stream)))
+
+
+def conv1x1_gs_cm(w: Packed, xt, ldx, y, ldy, m, flags=SBNN_RELU, tile=(0, 0, 0, 0), stream=None):
+    _check(lib().sbnn_conv1x1_gs_cm(w.handle, _ptr(xt), ldx, _ptr(y), ldy, m, flags, *tile, _stream(stream)))
+
+
+def to_channel_major(x, xt, m, c, ld, stream=None):
+    _check(lib().sbnn_to_channel_major(_ptr(x), _ptr(xt), m, c, ld, _stream(stream)))
 
 
 def conv3x3_gs(w: Packed, x, y, n, h, wd, flags=SBNN_RELU, stream=None):

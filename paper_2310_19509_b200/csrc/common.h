@@ -78,6 +78,7 @@ struct sbnn_packed {
     // kernel-private layouts, built on first use of a tile configuration
     mutable std::mutex mu;
     mutable std::map<sbnn::TileCfg, sbnn::Stream1x1> streams1x1;
+    mutable std::map<sbnn::TileCfg, sbnn::Stream1x1> streams_cm;   // channel-major kernel, see conv1x1_cm.cu
     mutable std::map<int, sbnn::Stream3x3> streams3x3;
     mutable void* bf16_stream = nullptr;  // see conv1x1_bf16.cu
 };
@@ -86,6 +87,12 @@ namespace sbnn {
 // conv1x1_gs.cu
 sbnn_status prepare_default_1x1(const sbnn_packed* p);
 void free_streams_1x1(sbnn_packed* p);
+// conv1x1_cm.cu
+sbnn_status prepare_default_cm(const sbnn_packed* p);
+void free_streams_cm(sbnn_packed* p);
+// Runs the NHWC call through the channel-major kernel if the shape profits; *done tells whether it did.
+sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st, bool* done);
+sbnn_status read_async_status(int* value);
 // conv1x1_bf16.cu
 sbnn_status conv1x1_bf16(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st);
 void free_stream_bf16(sbnn_packed* p);

@@ -1,0 +1,521 @@
+// Group-sparse 1x1 convolution on channel-major activations, fp32 (Algorithm 1 re-thought for sm_100a).
+//
+//   Y[m][g*G + r] = act( bias[g*G + r] + sum_j val[g][j][r] * X[idx[g][j]][m] ),   X given as [Cin][ldx]
+//
+// With the pixels of one input channel contiguous in global memory, the [channel][pixel] shared
+// memory tile that the compute warps want is a set of plain row copies, so the staging is done by
+// the copy engine and costs the SM no instructions:
+//   * warp NW (the producer) issues, per channel step, one bulk asynchronous copy per channel row
+//     and one for the step's weight block; their bytes complete a "full" mbarrier of the stage;
+//   * the NW compute warps wait on "full", run their kept units out of the stage, and each
+//     releases it by arriving on the stage's "empty" mbarrier; STAGES stages are in flight, so warps
+//     whose groups keep more units in a step are not waited for until STAGES steps later
+//     (balanced masks give every group the same total), and no CTA-wide barrier sits in the loop;
+//   * every wait has an iteration cap; a wait that expires records SBNN_ERR_TIMEOUT in a device
+//     status word, raises the CTA's abort flag, and the CTA drains its copies and returns.
+// Compute warps: a lane owns P consecutive-by-4 pixels (LDS.128 along the row) and G x GPW output
+// channels, accumulators packed in pairs of pixels and updated with fma.rn.f32x2.
+#include <string.h>
+
+#include <algorithm>
+
+#include "common.h"
+#include "pipeline.cuh"
+
+namespace sbnn {
+namespace {
+
+// Device status word: 0, or the sbnn_status of the first bounded wait that gave up.
+__device__ int g_async_status;
+
+template <int G_, int P_, int GPW_, int NW_, int KC_, int STAGES_>
+struct K2 {
+    static constexpr int G = G_, P = P_, GPW = GPW_, NW = NW_, KC = KC_, STAGES = STAGES_;
+    static constexpr int TM = 32 * P, GT = NW * GPW, NT = (NW + 1) * 32;
+    static constexpr int ROW_BYTES = TM * 4;
+    static constexpr int XS_BYTES = KC * ROW_BYTES;
+    static constexpr int HDR = (GT * 2 + 3) / 4;   // 16-byte units
+    static constexpr int QUAD = 1 + G;             // 4 row offsets + 4*G weights
+    static constexpr int WS_U4 = HDR + GT * (KC / 4) * QUAD;
+    static constexpr int WS_BYTES = (WS_U4 + QUAD) * 16;   // + slack: the loop reads one quad ahead
+    static constexpr size_t SMEM = (size_t)STAGES * (XS_BYTES + WS_BYTES) + 2 * STAGES * 8 + 16;
+    static_assert(P % 4 == 0 && KC % 4 == 0, "tile shape");
+    static_assert(SMEM <= 227 * 1024, "shared memory");
+};
+
+template <int G>
+__device__ __forceinline__ void unit_weights(const float* wq, int u, float (&w)[G]) {
+    if constexpr (G >= 4) {
+#pragma unroll
+        for (int v = 0; v < G / 4; ++v) {
+            const float4 t = reinterpret_cast<const float4*>(wq)[u * (G / 4) + v];
+            w[4 * v + 0] = t.x; w[4 * v + 1] = t.y; w[4 * v + 2] = t.z; w[4 * v + 3] = t.w;
+        }
+    } else if constexpr (G == 2) {
+        const float2 t = reinterpret_cast<const float2*>(wq)[u];
+        w[0] = t.x; w[1] = t.y;
+    } else {
+        w[0] = wq[u];
+    }
+}
+
+template <class C, bool OUT_CM>
+__global__ void __launch_bounds__(C::NT, 1)
+conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, int ldy,
+                  const float* __restrict__ bias, const uint4* __restrict__ rec,
+                  const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout, int ngroups, int nchunks,
+                  int relu, int* status) {
+    constexpr int G = C::G, P = C::P, GPW = C::GPW, NW = C::NW, KC = C::KC, S = C::STAGES;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* xs0 = smem;
+    unsigned char* ws0 = smem + (size_t)S * C::XS_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(ws0 + (size_t)S * C::WS_BYTES);
+    uint64_t* empty = full + S;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + S);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m0 = blockIdx.x * C::TM;
+    const int tile = blockIdx.y;
+    const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, NW);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == NW) {
+        // ---------------- producer warp ----------------
+        const uint32_t row_bytes = (uint32_t)min(C::TM, ldx - m0) * 4u;
+        int issued = 0;
+        bool ok = true;
+        for (int k = 0; k < nchunks && ok; ++k) {
+            const int s = k % S;
+            if (k >= S) ok = mbar_wait(empty + s, ((k / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+            if (!ok) break;
+            const int rows = min(KC, Cin - k * KC);
+            const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
+            if (lane == 0) mbar_arrive_expect_tx(full + s, (uint32_t)rows * row_bytes + (uint32_t)wn * 16u);
+            __syncwarp();
+            unsigned char* xs = xs0 + (size_t)s * C::XS_BYTES;
+            for (int r = lane; r < rows; r += 32)
+                bulk_g2s(xs + (size_t)r * C::ROW_BYTES, X + (size_t)(k * KC + r) * ldx + m0, row_bytes, full + s);
+            if (lane == 0) bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, full + s);
+            ++issued;
+        }
+        if (!ok) {
+            // gave up: let the copies already issued land before the CTA's shared memory is released
+            for (int k = max(0, issued - S); k < issued; ++k) {
+                bool landed = false;
+                for (uint32_t i = 0; i < kWaitLimit && !landed; ++i) landed = mbar_try_wait(full + k % S, (k / S) & 1);
+            }
+        }
+        return;
+    }
+
+    // ---------------- compute warps ----------------
+    f32x2 acc[GPW][P / 2][G];   // acc[q][p2][r]: pixels (2*p2, 2*p2+1) of the lane, channel r of group q
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * C::GT + warp * GPW + q;
+#pragma unroll
+        for (int r = 0; r < G; ++r) {
+            const float b = (g < ngroups) ? bias[g * G + r] : 0.0f;
+#pragma unroll
+            for (int p = 0; p < P / 2; ++p) acc[q][p][r] = pack2(b, b);
+        }
+    }
+
+    const unsigned lane_off = lane * 16;
+    bool ok = true;
+    for (int k = 0; k < nchunks; ++k) {
+        const int s = k % S;
+        ok = mbar_wait(full + s, (k / S) & 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+        if (!ok) break;
+        const unsigned char* xs = xs0 + (size_t)s * C::XS_BYTES + lane_off;
+        const uint4* ws = reinterpret_cast<const uint4*>(ws0 + (size_t)s * C::WS_BYTES);
+#pragma unroll
+        for (int q = 0; q < GPW; ++q) {
+            const int2 hd = reinterpret_cast<const int2*>(ws)[warp * GPW + q];   // (start, kept units)
+            const uint4* r = ws + hd.x;
+            uint4 off = r[0];
+            for (int j = 0; j < hd.y; j += 4, r += C::QUAD) {
+                const uint4 off_next = r[C::QUAD];   // one quad ahead (slack keeps it in bounds)
+                const float* wq = reinterpret_cast<const float*>(r + 1);
+                const unsigned offs[4] = {off.x, off.y, off.z, off.w};
+                const int left = hd.y - j;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (u < left) {   // warp-uniform: only the last quad of a list is short
+                        const unsigned char* ap = xs + offs[u];
+                        ulonglong2 a[P / 4];
+#pragma unroll
+                        for (int i = 0; i < P / 4; ++i) a[i] = *reinterpret_cast<const ulonglong2*>(ap + i * 512);
+                        float w[G];
+                        unit_weights<G>(wq, u, w);
+#pragma unroll
+                        for (int rr = 0; rr < G; ++rr) {
+                            const f32x2 ww = pack2(w[rr], w[rr]);
+#pragma unroll
+                            for (int i = 0; i < P / 4; ++i) {
+                                fma2(acc[q][2 * i][rr], a[i].x, ww);
+                                fma2(acc[q][2 * i + 1][rr], a[i].y, ww);
+                            }
+                        }
+                    }
+                }
+                off = off_next;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty + s);
+    }
+    if (!ok) return;
+
+    // epilogue
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * C::GT + warp * GPW + q;
+        if (g >= ngroups) continue;
+#pragma unroll
+        for (int i = 0; i < P / 4; ++i) {
+            const int mb = m0 + i * 128 + lane * 4;
+            float v[4][G];
+#pragma unroll
+            for (int rr = 0; rr < G; ++rr) {
+                unpack2(acc[q][2 * i][rr], v[0][rr], v[1][rr]);
+                unpack2(acc[q][2 * i + 1][rr], v[2][rr], v[3][rr]);
+            }
+            if (relu) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int rr = 0; rr < G; ++rr) v[e][rr] = fmaxf(v[e][rr], 0.0f);
+            }
+            if constexpr (OUT_CM) {
+#pragma unroll
+                for (int rr = 0; rr < G; ++rr) {
+                    float* yp = Y + (size_t)(g * G + rr) * ldy + mb;
+                    if (mb + 3 < M) {
+                        *reinterpret_cast<float4*>(yp) = make_float4(v[0][rr], v[1][rr], v[2][rr], v[3][rr]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (mb + e < M) yp[e] = v[e][rr];
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (mb + e >= M) continue;
+                    float* yp = Y + (size_t)(mb + e) * ldy + g * G;
+                    if constexpr (G >= 4) {
+#pragma unroll
+                        for (int vv = 0; vv < G / 4; ++vv)
+                            reinterpret_cast<float4*>(yp)[vv] =
+                                make_float4(v[e][4 * vv], v[e][4 * vv + 1], v[e][4 * vv + 2], v[e][4 * vv + 3]);
+                    } else if constexpr (G == 2) {
+                        *reinterpret_cast<float2*>(yp) = make_float2(v[e][0], v[e][1]);
+                    } else {
+                        yp[0] = v[e][0];
+                    }
+                }
+            }
+        }
+    }
+}
+
+// X [M][C] (row-major, C contiguous) -> Xt [C][ld]: 32 x 32 tiles through padded shared memory.
+__global__ void __launch_bounds__(256)
+to_channel_major_kernel(const float* __restrict__ x, float* __restrict__ xt, int M, int C, int ld) {
+    __shared__ float t[32][33];
+    const int m0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty + 8 * i, c = c0 + tx;
+        if (m < M && c < C) t[ty + 8 * i][tx] = x[(size_t)m * C + c];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = c0 + ty + 8 * i, m = m0 + tx;
+        if (m < M && c < C) xt[(size_t)c * ld + m] = t[tx][ty + 8 * i];
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------
+
+// Record stream for one tile shape: block (tile t, step k) = GT (start, kept units) pairs, then per
+// group its quads (4 byte offsets of the units' shared-memory rows, then 4*G weights); the last quad
+// of a list is zero-padded and the kernel skips the padding.
+sbnn_status build_stream_cm(const sbnn_packed* p, const TileCfg& c, Stream1x1* out) {
+    const int G = p->G, GT = c.GT(), KC = c.KC, TM = c.TM();
+    const int ntiles = (p->ngroups + GT - 1) / GT, nchunks = (p->Cin + KC - 1) / KC;
+    const int HDR = (GT * 2 + 3) / 4, QUAD = 1 + G;
+    std::vector<int32_t> blk((size_t)ntiles * (nchunks + 1));
+    std::vector<uint32_t> rec;
+    int max_blk = 0;
+    try {
+        rec.reserve(((size_t)p->nnz / 4 + (size_t)ntiles * nchunks * (GT + HDR)) * QUAD * 4);
+        for (int t = 0; t < ntiles; ++t) {
+            for (int k = 0; k < nchunks; ++k) {
+                const size_t blk_beg = rec.size() / 4;
+                blk[(size_t)t * (nchunks + 1) + k] = (int32_t)blk_beg;
+                rec.resize(rec.size() + (size_t)HDR * 4, 0u);
+                for (int s = 0; s < GT; ++s) {
+                    const int g = t * GT + s;
+                    int lo = 0, hi = 0;
+                    if (g < p->ngroups) {
+                        const int32_t* b = p->idx.data() + p->group_ptr[g];
+                        const int32_t* e = p->idx.data() + p->group_ptr[g + 1];
+                        lo = (int)(std::lower_bound(b, e, k * KC) - p->idx.data());
+                        hi = (int)(std::lower_bound(b, e, (k + 1) * KC) - p->idx.data());
+                    }
+                    const int n = hi - lo, nq = (n + 3) / 4;
+                    rec[blk_beg * 4 + 2 * s + 0] = (uint32_t)(rec.size() / 4 - blk_beg);
+                    rec[blk_beg * 4 + 2 * s + 1] = (uint32_t)n;
+                    for (int qd = 0; qd < nq; ++qd) {
+                        const size_t base = rec.size();
+                        rec.resize(base + (size_t)QUAD * 4, 0u);
+                        for (int u = 0; u < 4; ++u) {
+                            const int j = lo + qd * 4 + u;
+                            if (j >= hi) break;
+                            rec[base + u] = (uint32_t)(p->idx[j] - k * KC) * (uint32_t)(TM * 4);
+                            memcpy(&rec[base + 4 + u * G], &p->val[(size_t)j * G], sizeof(float) * G);
+                        }
+                    }
+                }
+                max_blk = std::max(max_blk, (int)(rec.size() / 4 - blk_beg));
+            }
+            blk[(size_t)t * (nchunks + 1) + nchunks] = (int32_t)(rec.size() / 4);
+        }
+    } catch (const std::bad_alloc&) {
+        return fail(SBNN_ERR_ALLOC, "out of host memory building the channel-major weight stream");
+    }
+    if (rec.size() / 4 > 0x7fffffffull) return fail(SBNN_ERR_UNSUPPORTED, "weight stream too large");
+    Stream1x1 s;
+    s.ntiles = ntiles; s.nchunks = nchunks; s.max_blk = max_blk;
+    SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&s.rec), std::max<size_t>(rec.size() * 4, 16)));
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s.blk_ptr), blk.size() * 4);
+    if (e == cudaSuccess && !rec.empty()) e = cudaMemcpy(s.rec, rec.data(), rec.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(s.blk_ptr, blk.data(), blk.size() * 4, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(s.rec);
+        cudaFree(s.blk_ptr);
+        cudaGetLastError();
+        return fail(SBNN_ERR_CUDA, "uploading the channel-major weight stream: %s", cudaGetErrorString(e));
+    }
+    *out = s;
+    return SBNN_OK;
+}
+
+sbnn_status get_stream_cm(const sbnn_packed* p, const TileCfg& c, Stream1x1* out) {
+    std::lock_guard<std::mutex> lk(p->mu);
+    auto it = p->streams_cm.find(c);
+    if (it != p->streams_cm.end()) {
+        *out = it->second;
+        return SBNN_OK;
+    }
+    sbnn_status st = build_stream_cm(p, c, out);
+    if (st == SBNN_OK) p->streams_cm[c] = *out;
+    return st;
+}
+
+// Address of the device status word on the current device.
+sbnn_status status_word(int** out) {
+    static std::mutex mu;
+    static std::map<int, int*> addr;
+    int dev = 0;
+    SBNN_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = addr.find(dev);
+    if (it == addr.end()) {
+        int* p = nullptr;
+        SBNN_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_async_status));
+        it = addr.emplace(dev, p).first;
+    }
+    *out = it->second;
+    return SBNN_OK;
+}
+
+template <class C>
+sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, int ldx, float* y, int ldy, int M,
+                      int relu, bool out_cm, cudaStream_t st) {
+    static std::mutex mu;
+    static std::map<int, bool> configured;
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (!configured[dev]) {
+            SBNN_CUDA_TRY(cudaFuncSetAttribute(conv1x1_cm_kernel<C, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
+            SBNN_CUDA_TRY(cudaFuncSetAttribute(conv1x1_cm_kernel<C, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
+            configured[dev] = true;
+        }
+    }
+    if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
+    int* status = nullptr;
+    sbnn_status r = status_word(&status);
+    if (r != SBNN_OK) return r;
+    dim3 grid((M + C::TM - 1) / C::TM, s.ntiles);
+    if (out_cm)
+        conv1x1_cm_kernel<C, true><<<grid, C::NT, C::SMEM, st>>>(x, ldx, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
+                                                                 p->ngroups, s.nchunks, relu, status);
+    else
+        conv1x1_cm_kernel<C, false><<<grid, C::NT, C::SMEM, st>>>(x, ldx, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
+                                                                  p->ngroups, s.nchunks, relu, status);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    return SBNN_OK;
+}
+
+// Instantiated shapes: (G, P, GPW, NW, KC, STAGES).
+#define SBNN_K2_CONFIGS(X) \
+    X(1, 8, 4, 8, 32, 4)   \
+    X(2, 8, 2, 8, 32, 4)   \
+    X(4, 8, 1, 16, 32, 4)  \
+    X(4, 8, 2, 8, 32, 4)   \
+    X(4, 8, 2, 16, 32, 3)  \
+    X(4, 4, 1, 8, 32, 4)   \
+    X(8, 8, 1, 8, 32, 4)   \
+    X(8, 8, 1, 16, 32, 4)  \
+    X(8, 4, 1, 16, 32, 4)  \
+    X(16, 4, 1, 8, 32, 4)
+
+int stages_of(int G, const TileCfg& c) {
+#define SBNN_ST(g, pp, gpw, nw, kc, st) \
+    if (G == g && c.P == pp && c.GPW == gpw && c.NW == nw && c.KC == kc) return st;
+    SBNN_K2_CONFIGS(SBNN_ST)
+#undef SBNN_ST
+    return 0;
+}
+
+sbnn_status dispatch_cm(const sbnn_packed* p, const TileCfg& c, const float* x, int ldx, float* y, int ldy, int M,
+                        int relu, bool out_cm, cudaStream_t st) {
+    Stream1x1 s;
+#define SBNN_TRY(g, pp, gpw, nw, kc, stg)                                                        \
+    if (p->G == g && c.P == pp && c.GPW == gpw && c.NW == nw && c.KC == kc) {                    \
+        sbnn_status r = get_stream_cm(p, c, &s);                                                 \
+        if (r != SBNN_OK) return r;                                                              \
+        return launch_cm<K2<g, pp, gpw, nw, kc, stg>>(p, s, x, ldx, y, ldy, M, relu, out_cm, st); \
+    }
+    SBNN_K2_CONFIGS(SBNN_TRY)
+#undef SBNN_TRY
+    return fail(SBNN_ERR_UNSUPPORTED, "no channel-major 1x1 kernel instance for G=%d P=%d GPW=%d NW=%d KC=%d", p->G,
+                c.P, c.GPW, c.NW, c.KC);
+}
+
+TileCfg default_cfg_cm(const sbnn_packed* p) {
+    switch (p->G) {
+        case 1: return {8, 4, 8, 32};
+        case 2: return {8, 2, 8, 32};
+        case 4: return {8, 1, 16, 32};
+        case 8: return {8, 1, 8, 32};
+        default: return {4, 1, 8, 32};
+    }
+}
+
+// Per-device scratch for the channel-major copy of X made on behalf of NHWC callers.  Grows on demand
+// (synchronously) and is kept until the process exits.
+struct Workspace {
+    float* ptr = nullptr;
+    size_t bytes = 0;
+};
+sbnn_status workspace(size_t bytes, float** out) {
+    static std::mutex mu;
+    static std::map<int, Workspace> ws;
+    int dev = 0;
+    SBNN_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(mu);
+    Workspace& w = ws[dev];
+    if (w.bytes < bytes) {
+        if (w.ptr) SBNN_CUDA_TRY(cudaFree(w.ptr));   // cudaFree waits for the launches that still use it
+        w.ptr = nullptr;
+        w.bytes = 0;
+        SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&w.ptr), bytes));
+        w.bytes = bytes;
+    }
+    *out = w.ptr;
+    return SBNN_OK;
+}
+
+}  // namespace
+
+sbnn_status prepare_default_cm(const sbnn_packed* p) {
+    Stream1x1 s;
+    return get_stream_cm(p, default_cfg_cm(p), &s);
+}
+
+void free_streams_cm(sbnn_packed* p) {
+    for (auto& kv : p->streams_cm) {
+        cudaFree(kv.second.rec);
+        cudaFree(kv.second.blk_ptr);
+    }
+    p->streams_cm.clear();
+}
+
+sbnn_status read_async_status(int* value) {
+    int* w = nullptr;
+    sbnn_status r = status_word(&w);
+    if (r != SBNN_OK) return r;
+    SBNN_CUDA_TRY(cudaMemcpy(value, w, sizeof(int), cudaMemcpyDeviceToHost));
+    if (*value) SBNN_CUDA_TRY(cudaMemset(w, 0, sizeof(int)));
+    return SBNN_OK;
+}
+
+sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st, bool* done) {
+    *done = false;
+    // worth the extra transposition pass only where the layer is bound by arithmetic
+    if (w->Cin < 128 || w->Cout < 64 || M < 4096) return SBNN_OK;
+    const int ld = (M + 3) / 4 * 4;
+    float* xt = nullptr;
+    sbnn_status r = workspace((size_t)w->Cin * ld * sizeof(float), &xt);
+    if (r != SBNN_OK) return r;
+    dim3 grid((M + 31) / 32, (w->Cin + 31) / 32);
+    to_channel_major_kernel<<<grid, 256, 0, st>>>(x, xt, M, w->Cin, ld);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    r = dispatch_cm(w, default_cfg_cm(w), xt, ld, y, w->Cout, M, relu, false, st);
+    if (r == SBNN_OK) *done = true;
+    return r;
+}
+
+}  // namespace sbnn
+
+using namespace sbnn;
+
+extern "C" sbnn_status sbnn_to_channel_major(const float* x_dev, float* xt_dev, int M, int C, int ld, void* cuda_stream) {
+    clear_error();
+    if (!x_dev || !xt_dev) return fail(SBNN_ERR_NULL, "x_dev and xt_dev must not be NULL");
+    if (M < 0 || C <= 0 || ld < M || ld % 4) return fail(SBNN_ERR_SHAPE, "bad shape M=%d C=%d ld=%d (ld >= M, ld %% 4 == 0)", M, C, ld);
+    if (M == 0) return SBNN_OK;
+    sbnn_status st = check_device();
+    if (st != SBNN_OK) return st;
+    dim3 grid((M + 31) / 32, (C + 31) / 32);
+    if (grid.y > 65535) return fail(SBNN_ERR_SHAPE, "C too large");
+    to_channel_major_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(x_dev, xt_dev, M, C, ld);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_conv1x1_gs_cm(const sbnn_packed* w, const float* xt_dev, int ldx, float* y_dev, int ldy, int M,
+                                          int flags, int P, int GPW, int NW, int KC, void* cuda_stream) {
+    clear_error();
+    if (!w || !xt_dev || !y_dev) return fail(SBNN_ERR_NULL, "packed weights, xt_dev and y_dev must not be NULL");
+    if (w->KH != 1 || w->KW != 1) return fail(SBNN_ERR_SHAPE, "packed layer is %dx%d, expected 1x1", w->KH, w->KW);
+    if (flags & ~(SBNN_RELU | SBNN_OUT_CM)) return fail(SBNN_ERR_UNSUPPORTED, "flag bits 0x%x not accepted here", flags);
+    const bool out_cm = (flags & SBNN_OUT_CM) != 0;
+    if (M < 0 || ldx < M || ldx % 4) return fail(SBNN_ERR_SHAPE, "ldx=%d must be >= M=%d and a multiple of 4", ldx, M);
+    if (out_cm ? (ldy < M || ldy % 4) : (ldy < w->Cout || ldy % 4))
+        return fail(SBNN_ERR_SHAPE, "ldy=%d does not fit the output layout", ldy);
+    if (!aligned16(xt_dev) || !aligned16(y_dev)) return fail(SBNN_ERR_ALIGN, "xt_dev and y_dev must be 16-byte aligned");
+    if (w->device < 0) return fail(SBNN_ERR_CUDA, "packed weights have no device copy (packed without a CUDA device)");
+    if (M == 0) return SBNN_OK;
+    sbnn_status st = check_device();
+    if (st != SBNN_OK) return st;
+    const TileCfg c = (P | GPW | NW | KC) ? TileCfg{P, GPW, NW, KC} : default_cfg_cm(w);
+    return dispatch_cm(w, c, xt_dev, ldx, y_dev, ldy, M, flags & SBNN_RELU, out_cm, static_cast<cudaStream_t>(cuda_stream));
+}

@@ -37,6 +37,21 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
 
+// Packed pair of fp32 values in one 64-bit register; fma2 is two independent fp32 FMAs (round to
+// nearest even each) issued as one instruction, which halves the issue slots the FMAs take.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma2(f32x2& d, f32x2 a, f32x2 b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
+}
+
 template <int G_, int P_, int GPW_, int NW_, int KC_>
 struct K1 {
     static constexpr int G = G_, P = P_, GPW = GPW_, NW = NW_, KC = KC_;
@@ -85,7 +100,8 @@ conv1x1_gs_kernel(const float* __restrict__ X, float* __restrict__ Y, const floa
     const int tile = blockIdx.y;
     const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
 
-    float acc[GPW][P][G];
+    // acc[q][p2][r] holds pixels (2*p2, 2*p2+1) of the lane for output channel r of group q
+    f32x2 acc[GPW][P / 2][G];
 #pragma unroll
     for (int q = 0; q < GPW; ++q) {
         const int g = tile * C::GT + warp * GPW + q;
@@ -93,7 +109,7 @@ conv1x1_gs_kernel(const float* __restrict__ X, float* __restrict__ Y, const floa
         for (int r = 0; r < G; ++r) {
             const float b = (g < ngroups) ? bias[g * G + r] : 0.0f;
 #pragma unroll
-            for (int p = 0; p < P; ++p) acc[q][p][r] = b;
+            for (int p = 0; p < P / 2; ++p) acc[q][p][r] = pack2(b, b);
         }
     }
 
@@ -156,19 +172,19 @@ conv1x1_gs_kernel(const float* __restrict__ X, float* __restrict__ Y, const floa
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const unsigned char* ap = xs + (offs[u] ^ lane_xor);
-                    float4 a[P / 4];
+                    ulonglong2 a[P / 4];   // four consecutive pixels = two packed pairs
 #pragma unroll
-                    for (int i = 0; i < P / 4; ++i) a[i] = *reinterpret_cast<const float4*>(ap + i * 512);
+                    for (int i = 0; i < P / 4; ++i) a[i] = *reinterpret_cast<const ulonglong2*>(ap + i * 512);
                     float w[G];
                     load_unit_weights<G>(wq, u, w);
 #pragma unroll
-                    for (int i = 0; i < P / 4; ++i) {
-                        const float xv[4] = {a[i].x, a[i].y, a[i].z, a[i].w};
+                    for (int rr = 0; rr < G; ++rr) {
+                        const f32x2 ww = pack2(w[rr], w[rr]);
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-#pragma unroll
-                            for (int rr = 0; rr < G; ++rr)
-                                acc[q][i * 4 + e][rr] = fmaf(xv[e], w[rr], acc[q][i * 4 + e][rr]);
+                        for (int i = 0; i < P / 4; ++i) {
+                            fma2(acc[q][2 * i][rr], a[i].x, ww);
+                            fma2(acc[q][2 * i + 1][rr], a[i].y, ww);
+                        }
                     }
                 }
             }
@@ -194,8 +210,12 @@ conv1x1_gs_kernel(const float* __restrict__ X, float* __restrict__ Y, const floa
                 float* yp = Y + (size_t)m * Cout + g * G;
                 float v[G];
 #pragma unroll
-                for (int rr = 0; rr < G; ++rr)
-                    v[rr] = relu ? fmaxf(acc[q][i * 4 + e][rr], 0.0f) : acc[q][i * 4 + e][rr];
+                for (int rr = 0; rr < G; ++rr) {
+                    float lo, hi;
+                    unpack2(acc[q][(i * 4 + e) / 2][rr], lo, hi);
+                    const float t = (e & 1) ? hi : lo;
+                    v[rr] = relu ? fmaxf(t, 0.0f) : t;
+                }
                 if constexpr (G >= 4) {
 #pragma unroll
                     for (int vv = 0; vv < G / 4; ++vv)
@@ -379,7 +399,7 @@ sbnn_status prepare_default_1x1(const sbnn_packed* p) {
         sbnn_status r = get_stream(p, choose_cfg(p, M), &s);
         if (r != SBNN_OK) return r;
     }
-    return SBNN_OK;
+    return p->Cin >= 128 ? prepare_default_cm(p) : SBNN_OK;
 }
 
 void free_streams_1x1(sbnn_packed* p) {
@@ -404,6 +424,8 @@ extern "C" sbnn_status sbnn_conv1x1_gs(const sbnn_packed* w, const float* x_dev,
     if ((st = check_device()) != SBNN_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (flags & SBNN_BF16_TC) return conv1x1_bf16(w, x_dev, y_dev, (int)M, flags & SBNN_RELU, s);
+    bool done = false;
+    if ((st = conv1x1_via_cm(w, x_dev, y_dev, (int)M, flags & SBNN_RELU, s, &done)) != SBNN_OK || done) return st;
     return dispatch(w, choose_cfg(w, M), x_dev, y_dev, (int)M, flags & SBNN_RELU, s);
 }
 

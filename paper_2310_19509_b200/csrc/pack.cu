@@ -211,6 +211,7 @@ extern "C" sbnn_status sbnn_packed_free(sbnn_packed* p) {
         int cur = 0;
         bool sw = cudaGetDevice(&cur) == cudaSuccess && cur != p->device && cudaSetDevice(p->device) == cudaSuccess;
         free_streams_1x1(p);
+        free_streams_cm(p);
         free_stream_bf16(p);
         free_streams_3x3(p);
         cudaFree(p->d_group_ptr);
@@ -230,5 +231,9 @@ extern "C" sbnn_status sbnn_get_async_status(void* stream) {
     if (e != cudaSuccess) return fail(SBNN_ERR_CUDA, "stream failed: %s", cudaGetErrorString(e));
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(SBNN_ERR_CUDA, "pending error: %s", cudaGetErrorString(e));
+    int word = 0;
+    sbnn_status st = read_async_status(&word);
+    if (st != SBNN_OK) return st;
+    if (word) return fail((sbnn_status)word, "a bounded wait inside a kernel gave up (device status %d)", word);
     return SBNN_OK;
 }

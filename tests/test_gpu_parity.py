@@ -225,3 +225,70 @@ def test_3x3_dense_and_empty_masks():
         y = run_3x3(d)
         ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
         assert_within(y, ref, s, what=f"3x3 sp={sp}")
+
+
+CM_CFGS = {1: [(8, 4, 8, 32)], 2: [(8, 2, 8, 32)],
+           4: [(8, 1, 16, 32), (8, 2, 8, 32), (8, 2, 16, 32), (4, 1, 8, 32)],
+           8: [(8, 1, 8, 32), (4, 1, 16, 32)], 16: [(4, 1, 8, 32)]}
+
+
+def run_cm(d, flags, tile, out_cm):
+    x = d["x"]
+    n, h, w, cin = x.shape
+    m = n * h * w
+    cout = d["w"].shape[0]
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], d["g"])
+    ld = (m + 3) // 4 * 4
+    xt = torch.full((cin, ld), float("nan"), device="cuda")
+    sbnn.to_channel_major(dev(x), xt, m, cin, ld)
+    if out_cm:
+        yd = torch.full((cout, ld), float("nan"), device="cuda")
+        sbnn.conv1x1_gs_cm(p, xt, ld, yd, ld, m, flags | sbnn.SBNN_OUT_CM, tile)
+        sbnn.get_async_status()
+        y = yd.cpu().numpy()[:, :m].T.reshape(n, h, w, cout)
+    else:
+        yd = torch.full((m, cout), float("nan"), device="cuda")
+        sbnn.conv1x1_gs_cm(p, xt, ld, yd, cout, m, flags, tile)
+        sbnn.get_async_status()
+        y = yd.cpu().numpy().reshape(n, h, w, cout)
+    p.free()
+    return y
+
+
+def test_to_channel_major_is_a_transpose():
+    x = torch.rand((1000 + 3, 70), device="cuda")
+    ld = 1004
+    xt = torch.zeros((70, ld), device="cuda")
+    sbnn.to_channel_major(x, xt, 1003, 70, ld)
+    assert torch.equal(xt[:, :1003], x.t())
+
+
+@pytest.mark.parametrize("g", [1, 2, 4, 8, 16])
+def test_channel_major_kernel_instances(g):
+    """Every compiled instance of the bulk-copy pipeline kernel: several pixel tiles with a ragged tail that is
+    not a multiple of 4, more channel steps than pipeline stages with a ragged last step, a ragged group tile."""
+    for cfg in CM_CFGS[g]:
+        tm = 32 * cfg[0]
+        d = WL.single_conv_inputs(1, 1, 2 * tm + 37, 212, 16 * 11, 1, g, 50, seed=8, mask_mode="layer_global")
+        for relu, out_cm in ((True, False), (False, True)):
+            y = run_cm(d, sbnn.SBNN_RELU if relu else 0, cfg, out_cm)
+            ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
+            assert_within(y, ref, s, what=f"cm G={g} cfg={cfg} relu={relu} out_cm={out_cm}")
+
+
+def test_channel_major_kernel_edge_cases():
+    for sp in (0, 100):
+        d = WL.single_conv_inputs(1, 3, 5, 40, 24, 1, 4, sp, seed=10)
+        y = run_cm(d, sbnn.SBNN_RELU, (0, 0, 0, 0), False)
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+        assert_within(y, ref, s, what=f"cm sp={sp}")
+
+
+def test_wide_layer_through_the_nhwc_entry_point():
+    """Config 5's layer shape at a reduced batch: the NHWC entry point routes it through the channel-major kernel."""
+    for g, sp in ((4, 50), (8, 70)):
+        d = WL.config5(g, sp, n=24)            # M = 4704 >= 4096
+        y = run_1x1(d)
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+        worst = assert_within(y, ref, s, what=f"config 5 G={g} s={sp} (n=24)")
+        assert worst < 0.5
