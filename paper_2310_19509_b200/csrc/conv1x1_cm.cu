@@ -36,8 +36,8 @@ struct K2 {
     static constexpr int XS_BYTES = KC * ROW_BYTES;
     static constexpr int HDR = (GT * 2 + 3) / 4;   // 16-byte units
     static constexpr int QUAD = 1 + G;             // 4 row offsets + 4*G weights
-    static constexpr int WS_U4 = HDR + GT * (KC / 4) * QUAD;
-    static constexpr int WS_BYTES = (WS_U4 + QUAD) * 16;   // + slack: the loop reads one quad ahead
+    static constexpr int WS_U4 = HDR + GT * (KC / 4 + 1) * QUAD;   // every list ends with an all-zero quad
+    static constexpr int WS_BYTES = WS_U4 * 16;
     static constexpr size_t SMEM = (size_t)STAGES * (XS_BYTES + WS_BYTES) + 2 * STAGES * 8 + 16;
     static_assert(P % 4 == 0 && KC % 4 == 0, "tile shape");
     static_assert(SMEM <= 227 * 1024, "shared memory");
@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(C::NT, 1)
 conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, int ldy,
                   const float* __restrict__ bias, const uint4* __restrict__ rec,
                   const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout, int ngroups, int nchunks,
-                  int relu, int* status) {
+                  int ntiles, int relu, int* status) {
     constexpr int G = C::G, P = C::P, GPW = C::GPW, NW = C::NW, KC = C::KC, S = C::STAGES;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* xs0 = smem;
@@ -74,8 +74,10 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
     volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + S);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int m0 = blockIdx.x * C::TM;
-    const int tile = blockIdx.y;
+    // group tiles of one pixel tile are neighbours in launch order, so they run at the same time and
+    // the pixel tile's activations come from DRAM once and from L2 afterwards
+    const int tile = blockIdx.x % ntiles;
+    const int m0 = (blockIdx.x / ntiles) * C::TM;
     const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
 
     if (tid == 0) {
@@ -142,33 +144,50 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
         for (int q = 0; q < GPW; ++q) {
             const int2 hd = reinterpret_cast<const int2*>(ws)[warp * GPW + q];   // (start, kept units)
             const uint4* r = ws + hd.x;
-            uint4 off = r[0];
-            for (int j = 0; j < hd.y; j += 4, r += C::QUAD) {
-                const uint4 off_next = r[C::QUAD];   // one quad ahead (slack keeps it in bounds)
-                const float* wq = reinterpret_cast<const float*>(r + 1);
-                const unsigned offs[4] = {off.x, off.y, off.z, off.w};
-                const int left = hd.y - j;
+            // Operands of one unit: P activations as packed pixel pairs and G weights.  Two operand sets
+            // alternate: the loads of the next unit are in flight while the FMAs of the current one
+            // issue, and no register copies are needed.  (Storing every weight twice, to load it as a
+            // ready (w, w) pair, was measured slower: the kernel is bound by shared-memory bandwidth.)
+            ulonglong2 aA[P / 4], aB[P / 4];
+            float wA[G], wB[G];
+            auto load_unit = [&](const uint4* quad, unsigned off, int u, ulonglong2 (&a)[P / 4], float (&w)[G]) {
+                const unsigned char* ap = xs + off;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (u < left) {   // warp-uniform: only the last quad of a list is short
-                        const unsigned char* ap = xs + offs[u];
-                        ulonglong2 a[P / 4];
+                for (int i = 0; i < P / 4; ++i) a[i] = *reinterpret_cast<const ulonglong2*>(ap + i * 512);
+                unit_weights<G>(reinterpret_cast<const float*>(quad + 1), u, w);
+            };
+            auto fma_unit = [&](const ulonglong2 (&a)[P / 4], const float (&w)[G]) {
 #pragma unroll
-                        for (int i = 0; i < P / 4; ++i) a[i] = *reinterpret_cast<const ulonglong2*>(ap + i * 512);
-                        float w[G];
-                        unit_weights<G>(wq, u, w);
+                for (int rr = 0; rr < G; ++rr) {
+                    const f32x2 ww = dup2(w[rr]);
 #pragma unroll
-                        for (int rr = 0; rr < G; ++rr) {
-                            const f32x2 ww = pack2(w[rr], w[rr]);
-#pragma unroll
-                            for (int i = 0; i < P / 4; ++i) {
-                                fma2(acc[q][2 * i][rr], a[i].x, ww);
-                                fma2(acc[q][2 * i + 1][rr], a[i].y, ww);
-                            }
-                        }
+                    for (int i = 0; i < P / 4; ++i) {
+                        fma2(acc[q][2 * i][rr], a[i].x, ww);
+                        fma2(acc[q][2 * i + 1][rr], a[i].y, ww);
                     }
                 }
+            };
+            uint4 off = r[0];
+            load_unit(r, off.x, 0, aA, wA);
+            const int nfull = hd.y >> 2, rem = hd.y & 3;
+            for (int it = 0; it < nfull; ++it) {
+                const uint4 off_next = r[C::QUAD];   // a list is followed by an all-zero quad, so this is always valid
+                load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+                load_unit(r, off.z, 2, aA, wA); fma_unit(aB, wB);
+                load_unit(r, off.w, 3, aB, wB); fma_unit(aA, wA);
+                load_unit(r + C::QUAD, off_next.x, 0, aA, wA); fma_unit(aB, wB);
                 off = off_next;
+                r += C::QUAD;
+            }
+            if (rem == 1) {   // last, short quad (warp-uniform)
+                fma_unit(aA, wA);
+            } else if (rem == 2) {
+                load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+                fma_unit(aB, wB);
+            } else if (rem == 3) {
+                load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+                load_unit(r, off.z, 2, aA, wA); fma_unit(aB, wB);
+                fma_unit(aA, wA);
             }
         }
         __syncwarp();
@@ -251,8 +270,9 @@ to_channel_major_kernel(const float* __restrict__ x, float* __restrict__ xt, int
 // ---- host side -------------------------------------------------------------------------------
 
 // Record stream for one tile shape: block (tile t, step k) = GT (start, kept units) pairs, then per
-// group its quads (4 byte offsets of the units' shared-memory rows, then 4*G weights); the last quad
-// of a list is zero-padded and the kernel skips the padding.
+// group its quads (4 byte offsets of the units' shared-memory rows, then 4*G weights).  A list always
+// ends with zero padding (offset 0, weight 0) up to and including one unit past its end, because the
+// kernel fetches the operands of the next unit before it knows the list is over.
 sbnn_status build_stream_cm(const sbnn_packed* p, const TileCfg& c, Stream1x1* out) {
     const int G = p->G, GT = c.GT(), KC = c.KC, TM = c.TM();
     const int ntiles = (p->ngroups + GT - 1) / GT, nchunks = (p->Cin + KC - 1) / KC;
@@ -261,7 +281,7 @@ sbnn_status build_stream_cm(const sbnn_packed* p, const TileCfg& c, Stream1x1* o
     std::vector<uint32_t> rec;
     int max_blk = 0;
     try {
-        rec.reserve(((size_t)p->nnz / 4 + (size_t)ntiles * nchunks * (GT + HDR)) * QUAD * 4);
+        rec.reserve(((size_t)p->nnz / 4 + (size_t)ntiles * nchunks * (2 * GT + HDR)) * QUAD * 4);
         for (int t = 0; t < ntiles; ++t) {
             for (int k = 0; k < nchunks; ++k) {
                 const size_t blk_beg = rec.size() / 4;
@@ -276,7 +296,8 @@ sbnn_status build_stream_cm(const sbnn_packed* p, const TileCfg& c, Stream1x1* o
                         lo = (int)(std::lower_bound(b, e, k * KC) - p->idx.data());
                         hi = (int)(std::lower_bound(b, e, (k + 1) * KC) - p->idx.data());
                     }
-                    const int n = hi - lo, nq = (n + 3) / 4;
+                    // the kernel prefetches one unit past the list: n % 4 == 0 needs a whole zero quad after it
+                    const int n = hi - lo, nq = n / 4 + 1;
                     rec[blk_beg * 4 + 2 * s + 0] = (uint32_t)(rec.size() / 4 - blk_beg);
                     rec[blk_beg * 4 + 2 * s + 1] = (uint32_t)n;
                     for (int qd = 0; qd < nq; ++qd) {
@@ -362,13 +383,15 @@ sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, 
     int* status = nullptr;
     sbnn_status r = status_word(&status);
     if (r != SBNN_OK) return r;
-    dim3 grid((M + C::TM - 1) / C::TM, s.ntiles);
+    const long long nblk = (long long)((M + C::TM - 1) / C::TM) * s.ntiles;
+    if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
+    dim3 grid((unsigned)nblk);
     if (out_cm)
         conv1x1_cm_kernel<C, true><<<grid, C::NT, C::SMEM, st>>>(x, ldx, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
-                                                                 p->ngroups, s.nchunks, relu, status);
+                                                                 p->ngroups, s.nchunks, s.ntiles, relu, status);
     else
         conv1x1_cm_kernel<C, false><<<grid, C::NT, C::SMEM, st>>>(x, ldx, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
-                                                                  p->ngroups, s.nchunks, relu, status);
+                                                                  p->ngroups, s.nchunks, s.ntiles, relu, status);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
 }
@@ -379,20 +402,10 @@ sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, 
     X(2, 8, 2, 8, 32, 4)   \
     X(4, 8, 1, 16, 32, 4)  \
     X(4, 8, 2, 8, 32, 4)   \
-    X(4, 8, 2, 16, 32, 3)  \
     X(4, 4, 1, 8, 32, 4)   \
     X(8, 8, 1, 8, 32, 4)   \
-    X(8, 8, 1, 16, 32, 4)  \
     X(8, 4, 1, 16, 32, 4)  \
     X(16, 4, 1, 8, 32, 4)
-
-int stages_of(int G, const TileCfg& c) {
-#define SBNN_ST(g, pp, gpw, nw, kc, st) \
-    if (G == g && c.P == pp && c.GPW == gpw && c.NW == nw && c.KC == kc) return st;
-    SBNN_K2_CONFIGS(SBNN_ST)
-#undef SBNN_ST
-    return 0;
-}
 
 sbnn_status dispatch_cm(const sbnn_packed* p, const TileCfg& c, const float* x, int ldx, float* y, int ldy, int M,
                         int relu, bool out_cm, cudaStream_t st) {

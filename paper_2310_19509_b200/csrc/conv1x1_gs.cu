@@ -89,15 +89,16 @@ template <class C>
 __global__ void __launch_bounds__(C::NT, 1)
 conv1x1_gs_kernel(const float* __restrict__ X, float* __restrict__ Y, const float* __restrict__ bias,
                   const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr,
-                  int M, int Cin, int Cout, int ngroups, int nchunks, int relu) {
+                  int M, int Cin, int Cout, int ngroups, int nchunks, int ntiles, int relu) {
     constexpr int G = C::G, P = C::P, GPW = C::GPW, NW = C::NW, KC = C::KC, TM = C::TM;
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* xs0 = smem;  // two X buffers, then two weight buffers
     uint4* ws0 = reinterpret_cast<uint4*>(smem + 2 * C::XS_BYTES);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int m0 = blockIdx.x * TM;
-    const int tile = blockIdx.y;
+    // group tiles of one pixel tile are neighbours in launch order (they share the tile's activations in L2)
+    const int tile = blockIdx.x % ntiles;
+    const int m0 = (blockIdx.x / ntiles) * TM;
     const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
 
     // acc[q][p2][r] holds pixels (2*p2, 2*p2+1) of the lane for output channel r of group q
@@ -331,9 +332,11 @@ sbnn_status launch(const sbnn_packed* p, const Stream1x1& s, const float* x, flo
     }
     if (s.max_blk > C::WS_U4)
         return fail(SBNN_ERR_UNSUPPORTED, "internal: weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
-    dim3 grid((M + C::TM - 1) / C::TM, s.ntiles);
+    const long long nblk = (long long)((M + C::TM - 1) / C::TM) * s.ntiles;
+    if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
+    dim3 grid((unsigned)nblk);
     conv1x1_gs_kernel<C><<<grid, C::NT, C::SMEM, st>>>(x, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
-                                                       p->ngroups, s.nchunks, relu);
+                                                       p->ngroups, s.nchunks, s.ntiles, relu);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
 }

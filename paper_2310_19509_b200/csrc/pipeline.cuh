@@ -16,6 +16,9 @@ __device__ __forceinline__ f32x2 pack2(float lo, float hi) {
     asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
     return r;
 }
+// (v, v).  (Building the copy on the integer pipe with a byte-permute, or storing weights twice in the
+// stream so they load as ready pairs, were both measured slower than the plain register move.)
+__device__ __forceinline__ f32x2 dup2(float v) { return pack2(v, v); }
 __device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }

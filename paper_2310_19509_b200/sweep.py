@@ -64,7 +64,7 @@ def dense_baselines(torch, x, cout, k, reps, flush):
     return out
 
 
-def run_case(torch, sbnn, name, d, k, reps, flush, tile=None, dense=True, flags=None):
+def run_case(torch, sbnn, name, d, k, reps, flush, tile=None, dense=True, flags=None, cm_tile=None):
     x = d["x"]
     n, h, w, cin = x.shape
     cout, g = d["w"].shape[0], d["g"]
@@ -74,6 +74,13 @@ def run_case(torch, sbnn, name, d, k, reps, flush, tile=None, dense=True, flags=
     fl = sbnn.SBNN_RELU if flags is None else flags
     if k == 3:
         f = lambda: sbnn.conv3x3_gs(p, xd, yd, n, h, w, fl)                     # noqa: E731
+    elif cm_tile is not None:
+        m_, ld = n * h * w, (n * h * w + 3) // 4 * 4
+        xt = torch.empty((cin, ld), device="cuda")
+
+        def f():
+            sbnn.to_channel_major(xd, xt, m_, cin, ld)
+            sbnn.conv1x1_gs_cm(p, xt, ld, yd, cout, m_, fl, cm_tile)
     elif tile:
         f = lambda: sbnn.conv1x1_gs_tuned(p, xd, yd, n, h, w, fl, *tile)        # noqa: E731
     else:
@@ -88,7 +95,7 @@ def run_case(torch, sbnn, name, d, k, reps, flush, tile=None, dense=True, flags=
     rec = {"case": name, "G": g, "sparsity_pct": d["sparsity_pct"], "M": m, "Cin": cin, "Cout": cout, "k": k,
            "us": med * 1e6, "us_min": mn * 1e6, "tflops_nonzero": flops / med / 1e12, "gbs": byts / med / 1e9,
            "roofline_us": roof * 1e6, "frac": roof / med, "bound": "alu" if flops / FP32_PEAK > byts / _hbm() else "hbm",
-           "tile": tile}
+           "tile": cm_tile or tile}
     if dense:
         rec.update(dense_baselines(torch, xd, cout, k, reps, flush))
     p.free()
@@ -104,12 +111,14 @@ def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--tile", default=None, help="P,GPW,NW,KC for the 1x1 kernel")
+    ap.add_argument("--cm-tile", default=None, help="P,GPW,NW,KC: transpose + channel-major kernel with this tile")
     ap.add_argument("--only", default=None)
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--batch5", type=int, default=256)
     args, _ = ap.parse_known_args(argv)
     tile = tuple(int(t) for t in args.tile.split(",")) if args.tile else None
+    cm_tile = tuple(int(t) for t in args.cm_tile.split(",")) if args.cm_tile else None
     flush = torch.zeros(64 * 1024 * 1024, device="cuda")
     cases = [("config1", lambda: WL.config1(), 1)]
     for g in (4, 8):
@@ -120,7 +129,8 @@ def main(argv=None):
         if args.only and args.only not in name:
             continue
         try:
-            rec = run_case(torch, sbnn, name, mk(), k, args.reps, flush, tile if k == 1 else None, not args.no_dense)
+            rec = run_case(torch, sbnn, name, mk(), k, args.reps, flush, tile if k == 1 else None, not args.no_dense,
+                           cm_tile=cm_tile if k == 1 else None)
         except sbnn.SbnnError as e:
             rec = {"case": name, "error": str(e)}
         print(json.dumps(rec), flush=True)

@@ -228,7 +228,7 @@ def test_3x3_dense_and_empty_masks():
 
 
 CM_CFGS = {1: [(8, 4, 8, 32)], 2: [(8, 2, 8, 32)],
-           4: [(8, 1, 16, 32), (8, 2, 8, 32), (8, 2, 16, 32), (4, 1, 8, 32)],
+           4: [(8, 1, 16, 32), (8, 2, 8, 32), (4, 1, 8, 32)],
            8: [(8, 1, 8, 32), (4, 1, 16, 32)], 16: [(4, 1, 8, 32)]}
 
 
