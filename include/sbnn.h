@@ -121,6 +121,9 @@ enum {
  *   w      packed 1x1 layer (KH = KW = 1)
  *   x_dev  [N][H][W][Cin] fp32, y_dev [N][H][W][Cout] fp32
  * Cin must be a multiple of 4 (else SBNN_ERR_UNSUPPORTED).  N*H*W == 0 returns SBNN_OK without a launch.
+ * With SBNN_BF16_TC the activations and the kept weights are rounded to bf16 (to nearest even) and the
+ * products are summed in fp32 on the tensor cores; bias and ReLU stay fp32.  The first call of a layer in
+ * that mode builds a private re-layout of its weights (allocates and copies synchronously).
  */
 SBNN_API sbnn_status sbnn_conv1x1_gs(const sbnn_packed* w, const float* x_dev, float* y_dev,
                                      int N, int H, int W, int flags, void* cuda_stream);

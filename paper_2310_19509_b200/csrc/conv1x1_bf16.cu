@@ -1,8 +1,288 @@
-// bf16 tensor-core variant of the group-sparse 1x1 convolution (placeholder until the kernel lands).
+// bf16 tensor-core mode of the group-sparse 1x1 convolution (flag SBNN_BF16_TC).
+//
+// Activations and kept weights are rounded to bf16 (round to nearest even), products are exact in
+// fp32 and accumulate in fp32 inside the tensor core; bias and ReLU stay fp32.
+//
+// Per group the work is a dense contraction  Y_g[pixels x G] = Xg[pixels x K'] * Wg[K' x G]  whose A
+// operand is a *gather* of K' channel rows.  The 5th-generation tensor-core path (tcgen05) reads its
+// operands from shared memory in fixed canonical layouts, so a per-channel gather would first have
+// to be copied into such a layout, which costs the shared-memory traffic the FFMA kernel already
+// pays.  The warp-level path does not have that restriction: ldmatrix takes one address per 8x8
+// sub-matrix row, and in the [channel][pixel] tile a sub-matrix row is 8 consecutive pixels of one
+// (arbitrary) channel.  So one `ldmatrix.x4.trans` with gathered row addresses yields the 16x16 A
+// fragment of an m16n8k16 MMA at 4 shared-memory wavefronts per 2048 MACs, against 9 per 1024 in
+// the fp32 kernel.  The N = 8 columns of the MMA are the group's output channels (G = 8 fills them,
+// G = 4 uses half, G = 16 takes two MMAs per A fragment).
+//
+// CTA = 128 pixels x 8 warps; a warp owns GPW groups over all 128 pixels (8 row blocks of 16), i.e.
+// 32 fp32 accumulators per N-tile.  Each channel step the CTA converts its X tile to bf16 and stores
+// it transposed; the weight stream holds, per 16 kept channels, 16 row offsets and the B fragments in
+// register order.
+#include <cuda_bf16.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
 #include "common.h"
+
 namespace sbnn {
-sbnn_status conv1x1_bf16(const sbnn_packed*, const float*, float*, int, int, cudaStream_t) {
-    return fail(SBNN_ERR_UNSUPPORTED, "bf16 tensor-core mode not built yet");
+namespace {
+
+constexpr int TM = 128;                    // pixels per CTA
+constexpr int KC = 64;                     // channels per step
+constexpr int ROWB = TM * 2 + 16;          // bytes per channel row (+16: spreads rows over bank groups)
+constexpr int NWARP = 8;
+
+struct StreamBf16 {
+    uint4* rec = nullptr;
+    int32_t* blk_ptr = nullptr;
+    int ntiles = 0, nchunks = 0, max_blk = 0, GT = 0;
+};
+
+template <int NT8>   // N-tiles of 8 output channels per group (1 for G <= 8, 2 for G = 16)
+struct KB {
+    static constexpr int BLK = 4 + NT8 * 16;   // one 16-channel block: 16 offsets + B fragments, 16-byte units
+};
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&a)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
+                 : "r"(addr));
 }
-void free_stream_bf16(sbnn_packed*) {}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int G, int GPW>
+__global__ void __launch_bounds__(NWARP * 32)
+conv1x1_bf16_kernel(const float* __restrict__ X, float* __restrict__ Y, const float* __restrict__ bias,
+                    const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout,
+                    int ngroups, int nchunks, int ntiles, int ws_u4, int relu) {
+    constexpr int NT8 = (G + 7) / 8;
+    constexpr int GT = NWARP * GPW;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* xs = smem;                                          // [KC][ROWB]
+    uint4* ws = reinterpret_cast<uint4*>(smem + KC * ROWB);            // weight block of the step
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tile = blockIdx.x % ntiles;
+    const int m0 = (blockIdx.x / ntiles) * TM;
+    const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
+    const int gq = lane >> 2, tq = lane & 3;
+
+    float acc[GPW][NT8][8][4];
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * GT + warp * GPW + q;
+#pragma unroll
+        for (int n = 0; n < NT8; ++n) {
+            const int c0 = n * 8 + 2 * tq;
+            const float b0 = (g < ngroups && c0 < G) ? bias[g * G + c0] : 0.f;
+            const float b1 = (g < ngroups && c0 + 1 < G) ? bias[g * G + c0 + 1] : 0.f;
+#pragma unroll
+            for (int pb = 0; pb < 8; ++pb) {
+                acc[q][n][pb][0] = b0; acc[q][n][pb][1] = b1; acc[q][n][pb][2] = b0; acc[q][n][pb][3] = b1;
+            }
+        }
+    }
+    // ldmatrix: lane l addresses row (l & 7) of sub-matrix (l >> 3): channels 8*(l>>4) + (l&7), pixels 8*((l>>3)&1)..
+    const int off_idx = 8 * (lane >> 4) + (lane & 7);
+    const uint32_t xs_lane = static_cast<uint32_t>(__cvta_generic_to_shared(xs)) + ((lane >> 3) & 1) * 16;
+
+    for (int k = 0; k < nchunks; ++k) {
+        __syncthreads();
+        {   // stage: X tile -> bf16, transposed; weight block
+            const int beg = bp[k], n = bp[k + 1] - beg;
+            for (int i = tid; i < n; i += NWARP * 32) ws[i] = rec[beg + i];
+            for (int e = tid; e < TM * (KC / 4); e += NWARP * 32) {
+                const int cq = e % (KC / 4), p = e / (KC / 4);
+                const int m = m0 + p, c = k * KC + cq * 4;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (m < M && c < Cin) v = __ldg(reinterpret_cast<const float4*>(X + (size_t)m * Cin + c));
+                __nv_bfloat16* d = reinterpret_cast<__nv_bfloat16*>(xs + (size_t)(cq * 4) * ROWB) + p;
+                d[0] = __float2bfloat16_rn(v.x);
+                d[ROWB / 2] = __float2bfloat16_rn(v.y);
+                d[ROWB] = __float2bfloat16_rn(v.z);
+                d[3 * (ROWB / 2)] = __float2bfloat16_rn(v.w);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < GPW; ++q) {
+            const int2 hd = reinterpret_cast<const int2*>(ws)[warp * GPW + q];   // (start, 16-channel blocks)
+            const uint4* r = ws + hd.x;
+            for (int it = 0; it < hd.y; ++it, r += KB<NT8>::BLK) {
+                const uint32_t row = xs_lane + reinterpret_cast<const uint32_t*>(r)[off_idx];
+                uint32_t b[NT8][2];
+#pragma unroll
+                for (int n = 0; n < NT8; ++n) {
+                    const uint2 t = reinterpret_cast<const uint2*>(r + 4 + n * 16)[lane];
+                    b[n][0] = t.x; b[n][1] = t.y;
+                }
+#pragma unroll
+                for (int pb = 0; pb < 8; ++pb) {
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(a, row + pb * 32);
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n) mma_bf16(acc[q][n][pb], a, b[n][0], b[n][1]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * GT + warp * GPW + q;
+        if (g >= ngroups) continue;
+#pragma unroll
+        for (int n = 0; n < NT8; ++n) {
+            const int c0 = n * 8 + 2 * tq;
+            if (c0 >= G) continue;
+#pragma unroll
+            for (int pb = 0; pb < 8; ++pb)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int m = m0 + pb * 16 + gq + 8 * h;
+                    if (m >= M) continue;
+                    float v0 = acc[q][n][pb][2 * h], v1 = acc[q][n][pb][2 * h + 1];
+                    if (relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+                    float* yp = Y + (size_t)m * Cout + g * G + c0;
+                    if (G >= 2) *reinterpret_cast<float2*>(yp) = make_float2(v0, v1);
+                    else yp[0] = v0;
+                }
+        }
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------
+
+// fp32 -> bf16 bits, round to nearest even (bf16 is the upper half of an IEEE-754 binary32).
+uint16_t bf16_bits(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u) return (uint16_t)(u >> 16);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+// Stream: block (tile t, step k) = GT (start, blocks) pairs, then per group its 16-channel blocks:
+// 16 byte offsets of the channels' shared-memory rows, then per N-tile the B fragment of m16n8k16 in
+// register order (lane l: {B[2t][g], B[2t+1][g]}, {B[2t+8][g], B[2t+9][g]}, g = l/4, t = l%4).
+sbnn_status build_stream_bf16(const sbnn_packed* p, StreamBf16* out) {
+    const int G = p->G, NT8 = (G + 7) / 8, GT = NWARP, BLK = 4 + NT8 * 16;
+    const int ntiles = (p->ngroups + GT - 1) / GT, nchunks = (p->Cin + KC - 1) / KC;
+    const int HDR = (GT * 2 + 3) / 4;
+    std::vector<int32_t> blk((size_t)ntiles * (nchunks + 1));
+    std::vector<uint32_t> rec;
+    int max_blk = 0;
+    try {
+        for (int t = 0; t < ntiles; ++t) {
+            for (int k = 0; k < nchunks; ++k) {
+                const size_t blk_beg = rec.size() / 4;
+                blk[(size_t)t * (nchunks + 1) + k] = (int32_t)blk_beg;
+                rec.resize(rec.size() + (size_t)HDR * 4, 0u);
+                for (int s = 0; s < GT; ++s) {
+                    const int g = t * GT + s;
+                    int lo = 0, hi = 0;
+                    if (g < p->ngroups) {
+                        const int32_t* b = p->idx.data() + p->group_ptr[g];
+                        const int32_t* e = p->idx.data() + p->group_ptr[g + 1];
+                        lo = (int)(std::lower_bound(b, e, k * KC) - p->idx.data());
+                        hi = (int)(std::lower_bound(b, e, (k + 1) * KC) - p->idx.data());
+                    }
+                    const int nb = (hi - lo + 15) / 16;
+                    rec[blk_beg * 4 + 2 * s + 0] = (uint32_t)(rec.size() / 4 - blk_beg);
+                    rec[blk_beg * 4 + 2 * s + 1] = (uint32_t)nb;
+                    for (int b16 = 0; b16 < nb; ++b16) {
+                        const size_t base = rec.size();
+                        rec.resize(base + (size_t)BLK * 4, 0u);   // padding: row 0, zero weights
+                        auto wbits = [&](int kk, int col) -> uint32_t {
+                            const int j = lo + b16 * 16 + kk;
+                            if (j >= hi || col >= G) return 0u;
+                            return bf16_bits(p->val[(size_t)j * G + col]);
+                        };
+                        for (int kk = 0; kk < 16; ++kk) {
+                            const int j = lo + b16 * 16 + kk;
+                            if (j < hi) rec[base + kk] = (uint32_t)(p->idx[j] - k * KC) * (uint32_t)ROWB;
+                        }
+                        for (int n = 0; n < NT8; ++n)
+                            for (int l = 0; l < 32; ++l) {
+                                const int gq = l >> 2, tq = l & 3, col = n * 8 + gq;
+                                rec[base + 16 + n * 64 + l * 2 + 0] = wbits(2 * tq, col) | (wbits(2 * tq + 1, col) << 16);
+                                rec[base + 16 + n * 64 + l * 2 + 1] = wbits(2 * tq + 8, col) | (wbits(2 * tq + 9, col) << 16);
+                            }
+                    }
+                }
+                max_blk = std::max(max_blk, (int)(rec.size() / 4 - blk_beg));
+            }
+            blk[(size_t)t * (nchunks + 1) + nchunks] = (int32_t)(rec.size() / 4);
+        }
+    } catch (const std::bad_alloc&) {
+        return fail(SBNN_ERR_ALLOC, "out of host memory building the bf16 weight stream");
+    }
+    StreamBf16 s;
+    s.ntiles = ntiles; s.nchunks = nchunks; s.max_blk = max_blk; s.GT = GT;
+    SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&s.rec), std::max<size_t>(rec.size() * 4, 16)));
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s.blk_ptr), blk.size() * 4);
+    if (e == cudaSuccess && !rec.empty()) e = cudaMemcpy(s.rec, rec.data(), rec.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(s.blk_ptr, blk.data(), blk.size() * 4, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(s.rec);
+        cudaFree(s.blk_ptr);
+        cudaGetLastError();
+        return fail(SBNN_ERR_CUDA, "uploading the bf16 weight stream: %s", cudaGetErrorString(e));
+    }
+    *out = s;
+    return SBNN_OK;
+}
+
+template <int G>
+sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, const float* x, float* y, int M, int relu, cudaStream_t st) {
+    const size_t smem = (size_t)KC * ROWB + (size_t)s.max_blk * 16;
+    if (smem > 48 * 1024) return fail(SBNN_ERR_UNSUPPORTED, "internal: bf16 tile needs %zu bytes of shared memory", smem);
+    const long long nblk = (long long)((M + TM - 1) / TM) * s.ntiles;
+    if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
+    conv1x1_bf16_kernel<G, 1><<<(unsigned)nblk, NWARP * 32, smem, st>>>(x, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
+                                                                        p->ngroups, s.nchunks, s.ntiles, s.max_blk, relu);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    return SBNN_OK;
+}
+
+}  // namespace
+
+sbnn_status conv1x1_bf16(const sbnn_packed* p, const float* x, float* y, int M, int relu, cudaStream_t st) {
+    StreamBf16* s = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(p->mu);
+        if (!p->bf16_stream) {   // first use of the mode on this layer: build the stream (allocates, copies)
+            StreamBf16* n = new (std::nothrow) StreamBf16;
+            if (!n) return fail(SBNN_ERR_ALLOC, "out of host memory");
+            sbnn_status r = build_stream_bf16(p, n);
+            if (r != SBNN_OK) {
+                delete n;
+                return r;
+            }
+            p->bf16_stream = n;
+        }
+        s = static_cast<StreamBf16*>(p->bf16_stream);
+    }
+    switch (p->G) {
+        case 1: return launch_bf16<1>(p, *s, x, y, M, relu, st);
+        case 2: return launch_bf16<2>(p, *s, x, y, M, relu, st);
+        case 4: return launch_bf16<4>(p, *s, x, y, M, relu, st);
+        case 8: return launch_bf16<8>(p, *s, x, y, M, relu, st);
+        default: return launch_bf16<16>(p, *s, x, y, M, relu, st);
+    }
+}
+
+void free_stream_bf16(sbnn_packed* p) {
+    if (!p->bf16_stream) return;
+    StreamBf16* s = static_cast<StreamBf16*>(p->bf16_stream);
+    cudaFree(s->rec);
+    cudaFree(s->blk_ptr);
+    delete s;
+    p->bf16_stream = nullptr;
+}
+
 }  // namespace sbnn

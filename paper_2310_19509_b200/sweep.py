@@ -112,6 +112,7 @@ def main(argv=None):
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--tile", default=None, help="P,GPW,NW,KC for the 1x1 kernel")
     ap.add_argument("--cm-tile", default=None, help="P,GPW,NW,KC: transpose + channel-major kernel with this tile")
+    ap.add_argument("--bf16", action="store_true", help="time the bf16 tensor-core mode instead of the fp32 kernel")
     ap.add_argument("--only", default=None)
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--no-dense", action="store_true")
@@ -129,8 +130,10 @@ def main(argv=None):
         if args.only and args.only not in name:
             continue
         try:
+            fl = (sbnn.SBNN_RELU | sbnn.SBNN_BF16_TC) if (args.bf16 and k == 1) else None
             rec = run_case(torch, sbnn, name, mk(), k, args.reps, flush, tile if k == 1 else None, not args.no_dense,
-                           cm_tile=cm_tile if k == 1 else None)
+                           flags=fl, cm_tile=cm_tile if k == 1 else None)
+            rec["mode"] = "bf16_tc" if fl else "fp32"
         except sbnn.SbnnError as e:
             rec = {"case": name, "error": str(e)}
         print(json.dumps(rec), flush=True)

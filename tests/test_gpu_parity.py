@@ -292,3 +292,25 @@ def test_wide_layer_through_the_nhwc_entry_point():
         ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
         worst = assert_within(y, ref, s, what=f"config 5 G={g} s={sp} (n=24)")
         assert worst < 0.5
+
+
+@pytest.mark.parametrize("g", [1, 2, 4, 8, 16])
+def test_bf16_tensor_core_mode(g):
+    """SBNN_BF16_TC against the oracle run on bf16-rounded operands (tight: products are exact in fp32,
+    accumulation is fp32) and against the fp32 oracle with the stated bf16 tolerance 1e-2 * S
+    (each operand is within 2^-9 relative after rounding, so 2 * 2^-9 * S plus accumulation)."""
+    d = WL.single_conv_inputs(1, 3, 131, 212, 16 * 11, 1, g, 50, seed=12, mask_mode="layer_global")
+    for relu in (True, False):
+        flags = sbnn.SBNN_BF16_TC | (sbnn.SBNN_RELU if relu else 0)
+        y = run_1x1(d, flags)
+        ref16, s16 = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu, bf16=True)
+        assert_within(y, ref16, s16, tol=1e-5, what=f"bf16 G={g} relu={relu} vs bf16 oracle")
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
+        assert_within(y, ref, s, tol=1e-2, what=f"bf16 G={g} relu={relu} vs fp32 oracle")
+
+
+def test_bf16_mode_on_config5_shape_reduced_batch():
+    d = WL.config5(8, 50, n=6)
+    y = run_1x1(d, sbnn.SBNN_BF16_TC | sbnn.SBNN_RELU)
+    ref16, s16 = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True, bf16=True)
+    assert_within(y, ref16, s16, tol=1e-5, what="config 5 G=8 bf16")
