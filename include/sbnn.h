@@ -147,7 +147,7 @@ SBNN_API sbnn_status sbnn_conv1x1_gs_tuned(const sbnn_packed* w, const float* x_
  *   output: y_dev [M][ldy] (pixel-major rows of ldy >= Cout floats), or, with SBNN_OUT_CM, [Cout][ldy]
  *   with ldy >= M; ldy a multiple of 4 in both cases.
  *   P, GPW, NW, KC: tile shape as in sbnn_conv1x1_gs_tuned, or all 0 for the default of the layer.
- * sbnn_conv1x1_gs itself takes this path for wide layers (Cin >= 128, M >= 4096): it first copies X
+ * sbnn_conv1x1_gs itself takes this path for wide layers (Cin >= 128, M >= 2048): it first copies X
  * into a channel-major scratch buffer kept per device, which it allocates or grows (synchronously) the
  * first time a size is seen.
  * sbnn_to_channel_major converts x_dev [M][C] to xt_dev [C][ld].

@@ -17,6 +17,8 @@
 // channels, accumulators packed in pairs of pixels and updated with fma.rn.f32x2.
 #include <string.h>
 
+#include <limits.h>
+
 #include <algorithm>
 
 #include "common.h"
@@ -34,9 +36,15 @@ struct K2 {
     static constexpr int TM = 32 * P, GT = NW * GPW, NT = (NW + 1) * 32;
     static constexpr int ROW_BYTES = TM * 4;
     static constexpr int XS_BYTES = KC * ROW_BYTES;
-    static constexpr int HDR = (GT * 2 + 3) / 4;   // 16-byte units
-    static constexpr int QUAD = 1 + G;             // 4 row offsets + 4*G weights
-    static constexpr int WS_U4 = HDR + GT * (KC / 4 + 1) * QUAD;   // every list ends with an all-zero quad
+    // GPW == 2 selects the union scheme: a warp's two groups share the activation fetch of every
+    // channel both keep; its lists are (both, only first, only second).
+    static constexpr bool UNION = (GPW == 2);
+    static constexpr int NL = UNION ? 3 : GPW;             // lists per warp and step
+    static constexpr int HDR = (NW * NL * 2 + 3) / 4;      // 16-byte units
+    static constexpr int QUAD = 1 + G;                     // 4 row offsets + 4*G weights
+    static constexpr int QUAD2 = 1 + 2 * G;                // the same for a unit that feeds two groups
+    static constexpr int NQ = KC / 4 + 1;                  // quads of a full list incl. its all-zero end quad
+    static constexpr int WS_U4 = UNION ? HDR + NW * (NQ * QUAD2 + 2 * NQ * QUAD) : HDR + GT * NQ * QUAD;
     static constexpr int WS_BYTES = WS_U4 * 16;
     static constexpr size_t SMEM = (size_t)STAGES * (XS_BYTES + WS_BYTES) + 2 * STAGES * 8 + 16;
     static_assert(P % 4 == 0 && KC % 4 == 0, "tile shape");
@@ -59,12 +67,70 @@ __device__ __forceinline__ void unit_weights(const float* wq, int u, float (&w)[
     }
 }
 
+// Runs one list of kept units against the stage: per unit P activations (packed pixel pairs) and
+// NG*G weights feed NG groups' accumulators.  Two operand sets alternate, so the loads of the next
+// unit are in flight while the FMAs of the current one issue and no register copies are needed.
+// (Storing every weight twice, to load it as a ready (w, w) pair, was measured slower: the kernel is
+// bound by shared-memory bandwidth.)  A list is followed by zero padding up to and including one
+// unit past its end, so the look-ahead never reads garbage.
+template <int P, int G, int NG>
+__device__ __forceinline__ void run_list(const uint4* r, int n, const unsigned char* xs, f32x2 (&acc0)[P / 2][G],
+                                         f32x2 (&acc1)[P / 2][G]) {
+    constexpr int QUAD = 1 + NG * G;
+    ulonglong2 aA[P / 4], aB[P / 4];
+    float wA[NG * G], wB[NG * G];
+    auto load_unit = [&](const uint4* quad, unsigned off, int u, ulonglong2 (&a)[P / 4], float (&w)[NG * G]) {
+        const unsigned char* ap = xs + off;
+#pragma unroll
+        for (int i = 0; i < P / 4; ++i) a[i] = *reinterpret_cast<const ulonglong2*>(ap + i * 512);
+        unit_weights<NG * G>(reinterpret_cast<const float*>(quad + 1), u, w);
+    };
+    auto fma_unit = [&](const ulonglong2 (&a)[P / 4], const float (&w)[NG * G]) {
+#pragma unroll
+        for (int rr = 0; rr < NG * G; ++rr) {
+            const f32x2 ww = dup2(w[rr]);
+#pragma unroll
+            for (int i = 0; i < P / 4; ++i) {
+                if (rr < G) {
+                    fma2(acc0[2 * i][rr], a[i].x, ww);
+                    fma2(acc0[2 * i + 1][rr], a[i].y, ww);
+                } else {
+                    fma2(acc1[2 * i][rr - G], a[i].x, ww);
+                    fma2(acc1[2 * i + 1][rr - G], a[i].y, ww);
+                }
+            }
+        }
+    };
+    uint4 off = r[0];
+    load_unit(r, off.x, 0, aA, wA);
+    const int nfull = n >> 2, rem = n & 3;
+    for (int it = 0; it < nfull; ++it) {
+        const uint4 off_next = r[QUAD];
+        load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+        load_unit(r, off.z, 2, aA, wA); fma_unit(aB, wB);
+        load_unit(r, off.w, 3, aB, wB); fma_unit(aA, wA);
+        load_unit(r + QUAD, off_next.x, 0, aA, wA); fma_unit(aB, wB);
+        off = off_next;
+        r += QUAD;
+    }
+    if (rem == 1) {   // last, short quad (warp-uniform)
+        fma_unit(aA, wA);
+    } else if (rem == 2) {
+        load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+        fma_unit(aB, wB);
+    } else if (rem == 3) {
+        load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+        load_unit(r, off.z, 2, aA, wA); fma_unit(aB, wB);
+        fma_unit(aA, wA);
+    }
+}
+
 template <class C, bool OUT_CM>
 __global__ void __launch_bounds__(C::NT, 1)
 conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, int ldy,
                   const float* __restrict__ bias, const uint4* __restrict__ rec,
                   const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout, int ngroups, int nchunks,
-                  int ntiles, int relu, int* status) {
+                  int ntiles, int total_tiles, int relu, int* status) {
     constexpr int G = C::G, P = C::P, GPW = C::GPW, NW = C::NW, KC = C::KC, S = C::STAGES;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* xs0 = smem;
@@ -74,11 +140,11 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
     volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + S);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // group tiles of one pixel tile are neighbours in launch order, so they run at the same time and
-    // the pixel tile's activations come from DRAM once and from L2 afterwards
-    const int tile = blockIdx.x % ntiles;
-    const int m0 = (blockIdx.x / ntiles) * C::TM;
-    const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
+    // Persistent CTAs: CTA b works on tiles b, b + gridDim.x, ...  A tile index t = ptile * ntiles + gtile
+    // keeps the group tiles of one pixel tile adjacent, so they run at about the same time and the pixel
+    // tile's activations come from DRAM once and from L2 afterwards.  Stage and phase counters run on
+    // across tiles: the producer is already filling stages for the next tile while the compute warps
+    // finish the current one and write its outputs.
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -92,22 +158,25 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
 
     if (warp == NW) {
         // ---------------- producer warp ----------------
-        const uint32_t row_bytes = (uint32_t)min(C::TM, ldx - m0) * 4u;
         int issued = 0;
         bool ok = true;
-        for (int k = 0; k < nchunks && ok; ++k) {
-            const int s = k % S;
-            if (k >= S) ok = mbar_wait(empty + s, ((k / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
-            if (!ok) break;
-            const int rows = min(KC, Cin - k * KC);
-            const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
-            if (lane == 0) mbar_arrive_expect_tx(full + s, (uint32_t)rows * row_bytes + (uint32_t)wn * 16u);
-            __syncwarp();
-            unsigned char* xs = xs0 + (size_t)s * C::XS_BYTES;
-            for (int r = lane; r < rows; r += 32)
-                bulk_g2s(xs + (size_t)r * C::ROW_BYTES, X + (size_t)(k * KC + r) * ldx + m0, row_bytes, full + s);
-            if (lane == 0) bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, full + s);
-            ++issued;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const int tile = t % ntiles, m0 = (t / ntiles) * C::TM;
+            const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
+            const uint32_t row_bytes = (uint32_t)min(C::TM, ldx - m0) * 4u;
+            for (int k = 0; k < nchunks; ++k, ++issued) {
+                const int s = issued % S;
+                if (issued >= S) ok = mbar_wait(empty + s, ((issued / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+                if (!ok) break;
+                const int rows = min(KC, Cin - k * KC);
+                const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
+                if (lane == 0) mbar_arrive_expect_tx(full + s, (uint32_t)rows * row_bytes + (uint32_t)wn * 16u);
+                __syncwarp();
+                unsigned char* xs = xs0 + (size_t)s * C::XS_BYTES;
+                for (int r = lane; r < rows; r += 32)
+                    bulk_g2s(xs + (size_t)r * C::ROW_BYTES, X + (size_t)(k * KC + r) * ldx + m0, row_bytes, full + s);
+                if (lane == 0) bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, full + s);
+            }
         }
         if (!ok) {
             // gave up: let the copies already issued land before the CTA's shared memory is released
@@ -120,6 +189,10 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
     }
 
     // ---------------- compute warps ----------------
+    const unsigned lane_off = lane * 16;
+    int consumed = 0;
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+    const int tile = t % ntiles, m0 = (t / ntiles) * C::TM;
     f32x2 acc[GPW][P / 2][G];   // acc[q][p2][r]: pixels (2*p2, 2*p2+1) of the lane, channel r of group q
 #pragma unroll
     for (int q = 0; q < GPW; ++q) {
@@ -132,62 +205,24 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
         }
     }
 
-    const unsigned lane_off = lane * 16;
     bool ok = true;
-    for (int k = 0; k < nchunks; ++k) {
-        const int s = k % S;
-        ok = mbar_wait(full + s, (k / S) & 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+    for (int k = 0; k < nchunks; ++k, ++consumed) {
+        const int s = consumed % S;
+        ok = mbar_wait(full + s, (consumed / S) & 1, abort_flag, status, SBNN_ERR_TIMEOUT);
         if (!ok) break;
         const unsigned char* xs = xs0 + (size_t)s * C::XS_BYTES + lane_off;
         const uint4* ws = reinterpret_cast<const uint4*>(ws0 + (size_t)s * C::WS_BYTES);
+        const int2* hdr = reinterpret_cast<const int2*>(ws) + warp * C::NL;   // (start, kept units) per list
+        if constexpr (C::UNION) {
+            const int2 hb = hdr[0], h0 = hdr[1], h1 = hdr[2];
+            run_list<P, G, 2>(ws + hb.x, hb.y, xs, acc[0], acc[1]);   // channels both groups keep
+            run_list<P, G, 1>(ws + h0.x, h0.y, xs, acc[0], acc[0]);   // only the first group
+            run_list<P, G, 1>(ws + h1.x, h1.y, xs, acc[1], acc[1]);   // only the second group
+        } else {
 #pragma unroll
-        for (int q = 0; q < GPW; ++q) {
-            const int2 hd = reinterpret_cast<const int2*>(ws)[warp * GPW + q];   // (start, kept units)
-            const uint4* r = ws + hd.x;
-            // Operands of one unit: P activations as packed pixel pairs and G weights.  Two operand sets
-            // alternate: the loads of the next unit are in flight while the FMAs of the current one
-            // issue, and no register copies are needed.  (Storing every weight twice, to load it as a
-            // ready (w, w) pair, was measured slower: the kernel is bound by shared-memory bandwidth.)
-            ulonglong2 aA[P / 4], aB[P / 4];
-            float wA[G], wB[G];
-            auto load_unit = [&](const uint4* quad, unsigned off, int u, ulonglong2 (&a)[P / 4], float (&w)[G]) {
-                const unsigned char* ap = xs + off;
-#pragma unroll
-                for (int i = 0; i < P / 4; ++i) a[i] = *reinterpret_cast<const ulonglong2*>(ap + i * 512);
-                unit_weights<G>(reinterpret_cast<const float*>(quad + 1), u, w);
-            };
-            auto fma_unit = [&](const ulonglong2 (&a)[P / 4], const float (&w)[G]) {
-#pragma unroll
-                for (int rr = 0; rr < G; ++rr) {
-                    const f32x2 ww = dup2(w[rr]);
-#pragma unroll
-                    for (int i = 0; i < P / 4; ++i) {
-                        fma2(acc[q][2 * i][rr], a[i].x, ww);
-                        fma2(acc[q][2 * i + 1][rr], a[i].y, ww);
-                    }
-                }
-            };
-            uint4 off = r[0];
-            load_unit(r, off.x, 0, aA, wA);
-            const int nfull = hd.y >> 2, rem = hd.y & 3;
-            for (int it = 0; it < nfull; ++it) {
-                const uint4 off_next = r[C::QUAD];   // a list is followed by an all-zero quad, so this is always valid
-                load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
-                load_unit(r, off.z, 2, aA, wA); fma_unit(aB, wB);
-                load_unit(r, off.w, 3, aB, wB); fma_unit(aA, wA);
-                load_unit(r + C::QUAD, off_next.x, 0, aA, wA); fma_unit(aB, wB);
-                off = off_next;
-                r += C::QUAD;
-            }
-            if (rem == 1) {   // last, short quad (warp-uniform)
-                fma_unit(aA, wA);
-            } else if (rem == 2) {
-                load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
-                fma_unit(aB, wB);
-            } else if (rem == 3) {
-                load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
-                load_unit(r, off.z, 2, aA, wA); fma_unit(aB, wB);
-                fma_unit(aA, wA);
+            for (int q = 0; q < GPW; ++q) {
+                const int2 hd = hdr[q];
+                run_list<P, G, 1>(ws + hd.x, hd.y, xs, acc[q], acc[q]);
             }
         }
         __syncwarp();
@@ -246,6 +281,7 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
             }
         }
     }
+    }   // tiles
 }
 
 // X [M][C] (row-major, C contiguous) -> Xt [C][ld]: 32 x 32 tiles through padded shared memory.
@@ -269,46 +305,80 @@ to_channel_major_kernel(const float* __restrict__ x, float* __restrict__ xt, int
 
 // ---- host side -------------------------------------------------------------------------------
 
-// Record stream for one tile shape: block (tile t, step k) = GT (start, kept units) pairs, then per
-// group its quads (4 byte offsets of the units' shared-memory rows, then 4*G weights).  A list always
-// ends with zero padding (offset 0, weight 0) up to and including one unit past its end, because the
-// kernel fetches the operands of the next unit before it knows the list is over.
+// Record stream for one tile shape.  Block (tile t, step k) = header of (start, kept units) per list,
+// then the lists.  A list is a run of quads (4 byte offsets of the units' shared-memory rows, then the
+// weights of the 4 units); it always ends with zero padding (offset 0, weight 0) up to and including
+// one unit past its end, because the kernel fetches the operands of the next unit before it knows the
+// list is over.  Plain layout: one list per group.  Union layout (GPW == 2): per warp the channels kept
+// by both of its groups (2*G weights per unit), then those kept only by the first, only by the second.
 sbnn_status build_stream_cm(const sbnn_packed* p, const TileCfg& c, Stream1x1* out) {
     const int G = p->G, GT = c.GT(), KC = c.KC, TM = c.TM();
+    const bool un = (c.GPW == 2);
+    const int NL = un ? 3 : c.GPW;
     const int ntiles = (p->ngroups + GT - 1) / GT, nchunks = (p->Cin + KC - 1) / KC;
-    const int HDR = (GT * 2 + 3) / 4, QUAD = 1 + G;
+    const int HDR = (c.NW * NL * 2 + 3) / 4;
     std::vector<int32_t> blk((size_t)ntiles * (nchunks + 1));
     std::vector<uint32_t> rec;
     int max_blk = 0;
+    // one kept unit of a list: position in the canonical arrays for each group it feeds (-1: none)
+    struct Unit { int c; int64_t j0, j1; };
+    std::vector<Unit> lists[3];
     try {
-        rec.reserve(((size_t)p->nnz / 4 + (size_t)ntiles * nchunks * (2 * GT + HDR)) * QUAD * 4);
+        rec.reserve(((size_t)p->nnz / 4 + (size_t)ntiles * nchunks * (2 * GT + HDR)) * (1 + G) * 4);
+        auto emit = [&](size_t blk_beg, int slot, const std::vector<Unit>& L, int ng, int k) {
+            const int QUAD = 1 + ng * G;
+            const int n = (int)L.size(), nq = n / 4 + 1;
+            rec[blk_beg * 4 + 2 * slot + 0] = (uint32_t)(rec.size() / 4 - blk_beg);
+            rec[blk_beg * 4 + 2 * slot + 1] = (uint32_t)n;
+            for (int qd = 0; qd < nq; ++qd) {
+                const size_t base = rec.size();
+                rec.resize(base + (size_t)QUAD * 4, 0u);
+                for (int u = 0; u < 4; ++u) {
+                    const int i = qd * 4 + u;
+                    if (i >= n) break;
+                    rec[base + u] = (uint32_t)(L[i].c - k * KC) * (uint32_t)(TM * 4);
+                    memcpy(&rec[base + 4 + u * ng * G], &p->val[(size_t)L[i].j0 * G], sizeof(float) * G);
+                    if (ng == 2) memcpy(&rec[base + 4 + u * ng * G + G], &p->val[(size_t)L[i].j1 * G], sizeof(float) * G);
+                }
+            }
+        };
+        auto range = [&](int g, int k, int64_t* lo, int64_t* hi) {
+            *lo = *hi = 0;
+            if (g >= p->ngroups) return;
+            const int32_t* b = p->idx.data() + p->group_ptr[g];
+            const int32_t* e = p->idx.data() + p->group_ptr[g + 1];
+            *lo = std::lower_bound(b, e, k * KC) - p->idx.data();
+            *hi = std::lower_bound(b, e, (k + 1) * KC) - p->idx.data();
+        };
         for (int t = 0; t < ntiles; ++t) {
             for (int k = 0; k < nchunks; ++k) {
                 const size_t blk_beg = rec.size() / 4;
                 blk[(size_t)t * (nchunks + 1) + k] = (int32_t)blk_beg;
                 rec.resize(rec.size() + (size_t)HDR * 4, 0u);
-                for (int s = 0; s < GT; ++s) {
-                    const int g = t * GT + s;
-                    int lo = 0, hi = 0;
-                    if (g < p->ngroups) {
-                        const int32_t* b = p->idx.data() + p->group_ptr[g];
-                        const int32_t* e = p->idx.data() + p->group_ptr[g + 1];
-                        lo = (int)(std::lower_bound(b, e, k * KC) - p->idx.data());
-                        hi = (int)(std::lower_bound(b, e, (k + 1) * KC) - p->idx.data());
+                if (!un) {
+                    for (int s = 0; s < GT; ++s) {
+                        int64_t lo, hi;
+                        range(t * GT + s, k, &lo, &hi);
+                        lists[0].clear();
+                        for (int64_t j = lo; j < hi; ++j) lists[0].push_back({p->idx[j], j, -1});
+                        emit(blk_beg, s, lists[0], 1, k);
                     }
-                    // the kernel prefetches one unit past the list: n % 4 == 0 needs a whole zero quad after it
-                    const int n = hi - lo, nq = n / 4 + 1;
-                    rec[blk_beg * 4 + 2 * s + 0] = (uint32_t)(rec.size() / 4 - blk_beg);
-                    rec[blk_beg * 4 + 2 * s + 1] = (uint32_t)n;
-                    for (int qd = 0; qd < nq; ++qd) {
-                        const size_t base = rec.size();
-                        rec.resize(base + (size_t)QUAD * 4, 0u);
-                        for (int u = 0; u < 4; ++u) {
-                            const int j = lo + qd * 4 + u;
-                            if (j >= hi) break;
-                            rec[base + u] = (uint32_t)(p->idx[j] - k * KC) * (uint32_t)(TM * 4);
-                            memcpy(&rec[base + 4 + u * G], &p->val[(size_t)j * G], sizeof(float) * G);
+                } else {
+                    for (int w = 0; w < c.NW; ++w) {
+                        int64_t lo0, hi0, lo1, hi1;
+                        range(t * GT + 2 * w, k, &lo0, &hi0);
+                        range(t * GT + 2 * w + 1, k, &lo1, &hi1);
+                        for (auto& L : lists) L.clear();
+                        int64_t i0 = lo0, i1 = lo1;   // merge the two ascending index lists
+                        while (i0 < hi0 || i1 < hi1) {
+                            const int c0 = i0 < hi0 ? p->idx[i0] : INT_MAX, c1 = i1 < hi1 ? p->idx[i1] : INT_MAX;
+                            if (c0 == c1) { lists[0].push_back({c0, i0, i1}); ++i0; ++i1; }
+                            else if (c0 < c1) { lists[1].push_back({c0, i0, -1}); ++i0; }
+                            else { lists[2].push_back({c1, i1, -1}); ++i1; }
                         }
+                        emit(blk_beg, 3 * w + 0, lists[0], 2, k);
+                        emit(blk_beg, 3 * w + 1, lists[1], 1, k);
+                        emit(blk_beg, 3 * w + 2, lists[2], 1, k);
                     }
                 }
                 max_blk = std::max(max_blk, (int)(rec.size() / 4 - blk_beg));
@@ -364,6 +434,22 @@ sbnn_status status_word(int** out) {
     return SBNN_OK;
 }
 
+// Number of SMs of the current device (one persistent CTA each).
+int sm_count() {
+    static std::mutex mu;
+    static std::map<int, int> n;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = n.find(dev);
+    if (it == n.end()) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        it = n.emplace(dev, v).first;
+    }
+    return it->second;
+}
+
 template <class C>
 sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, int ldx, float* y, int ldy, int M,
                       int relu, bool out_cm, cudaStream_t st) {
@@ -385,13 +471,14 @@ sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, 
     if (r != SBNN_OK) return r;
     const long long nblk = (long long)((M + C::TM - 1) / C::TM) * s.ntiles;
     if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
-    dim3 grid((unsigned)nblk);
+    const int total_tiles = (int)nblk;
+    dim3 grid((unsigned)std::min<long long>(nblk, sm_count()));
     if (out_cm)
         conv1x1_cm_kernel<C, true><<<grid, C::NT, C::SMEM, st>>>(x, ldx, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
-                                                                 p->ngroups, s.nchunks, s.ntiles, relu, status);
+                                                                 p->ngroups, s.nchunks, s.ntiles, total_tiles, relu, status);
     else
         conv1x1_cm_kernel<C, false><<<grid, C::NT, C::SMEM, st>>>(x, ldx, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
-                                                                  p->ngroups, s.nchunks, s.ntiles, relu, status);
+                                                                  p->ngroups, s.nchunks, s.ntiles, total_tiles, relu, status);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
 }
@@ -426,7 +513,7 @@ TileCfg default_cfg_cm(const sbnn_packed* p) {
     switch (p->G) {
         case 1: return {8, 4, 8, 32};
         case 2: return {8, 2, 8, 32};
-        case 4: return {8, 1, 16, 32};
+        case 4: return {8, 2, 8, 32};
         case 8: return {8, 1, 8, 32};
         default: return {4, 1, 8, 32};
     }
@@ -483,7 +570,7 @@ sbnn_status read_async_status(int* value) {
 sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st, bool* done) {
     *done = false;
     // worth the extra transposition pass only where the layer is bound by arithmetic
-    if (w->Cin < 128 || w->Cout < 64 || M < 4096) return SBNN_OK;
+    if (w->Cin < 128 || w->Cout < 64 || M < 2048) return SBNN_OK;
     const int ld = (M + 3) / 4 * 4;
     float* xt = nullptr;
     sbnn_status r = workspace((size_t)w->Cin * ld * sizeof(float), &xt);
