@@ -1,7 +1,9 @@
 // MobileNet-v1 (width 1.0, 224x224x3) forward chain: the engine's forward pass of Section 3.5
 // with the 13 pointwise layers group-sparse (the layers Tables 3 and 4 prune) and everything
 // else dense.  Launches only: conv0 -> 13 x (depthwise, pointwise) -> pool -> classifier on one
-// stream over two ping-pong workspaces.
+// stream over two ping-pong workspaces.  Between the image and the pooled features every
+// activation is kept channel-major ([C][ld], the pixels of a channel contiguous), the layout in
+// which the group-sparse 1x1 kernel's tiles are plain row copies; no layer transposes anything.
 #include <new>
 
 #include "common.h"
@@ -89,6 +91,11 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
     if (fc->KH != 1 || fc->Cin != 1024 || fc->Cout != 1000) return fail(SBNN_ERR_SHAPE, "classifier must be 1024->1000 1x1");
     sbnn_status st = check_device();
     if (st != SBNN_OK) return st;
+    // The kernel-private weight layouts of the channel-major 1x1 kernel are built here, not in forward.
+    for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
+        if (pw[i]->device < 0) return fail(SBNN_ERR_CUDA, "pointwise layer %d was packed without a CUDA device", i + 1);
+        if ((st = prepare_default_cm(pw[i])) != SBNN_OK) return st;
+    }
     sbnn_mbv1* n = new (std::nothrow) sbnn_mbv1;
     if (!n) return fail(SBNN_ERR_ALLOC, "out of host memory");
     for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
@@ -99,8 +106,8 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
     n->fc = fc; n->c0_w = conv0_w_dev; n->c0_b = conv0_b_dev; n->max_batch = max_batch;
     n->ws[0] = n->ws[1] = nullptr;
     cudaGetDevice(&n->device);
-    // Largest activation: pw1's output, 112*112*64 floats per image.
-    const size_t bytes = (size_t)max_batch * 112 * 112 * 64 * sizeof(float);
+    // Largest activation: pw1's output, 112*112*64 floats per image (+ row padding of the layout).
+    const size_t bytes = ((size_t)max_batch * 112 * 112 * 64 + 4 * 1024) * sizeof(float);
     for (int i = 0; i < 2; ++i) {
         cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&n->ws[i]), bytes);
         if (e != cudaSuccess) {
@@ -113,21 +120,51 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
     return SBNN_OK;
 }
 
+namespace {
+
+inline int round4(long long v) { return (int)((v + 3) / 4 * 4); }
+
+// One layer on channel-major buffers.  in: channel-major [Cin][ld_in] (layer 0: the NHWC image);
+// out: channel-major [Cout][ld_out] (pool: [N][C]; classifier: [N][1000], reading the pooled [N][C]).
+sbnn_status run_cm(sbnn_mbv1* net, int layer, const float* in, float* out, int N, void* stream) {
+    const LayerShape& L = layer_table()[layer];
+    const int blk = (layer - 1) / 2;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int ld_in = round4((long long)N * L.hin * L.hin), ld_out = round4((long long)N * L.hout * L.hout);
+    switch (L.kind) {
+        case 0: return launch_conv3x3_thin_cm(net->c0_w, net->c0_b, in, out, ld_out, N, L.hin, L.hin, L.cin, L.cout, L.stride, 1, st);
+        case 1: return launch_dwconv3x3_cm(net->dw_w[blk], net->dw_b[blk], in, ld_in, out, ld_out, N, L.hin, L.hin, L.cin, L.stride, 1, st);
+        case 2: return sbnn_conv1x1_gs_cm(net->pw[blk], in, ld_in, out, ld_out, N * L.hin * L.hin, SBNN_RELU | SBNN_OUT_CM, 0, 0, 0, 0, stream);
+        case 3: return launch_avgpool_cm(in, ld_in, out, N, L.hin * L.hin, L.cin, st);
+        default: return sbnn_conv1x1_gs(net->fc, in, out, N, 1, 1, 0, stream);
+    }
+}
+
+}  // namespace
+
 extern "C" sbnn_status sbnn_mobilenet_v1_run_layer(sbnn_mbv1* net, int layer, const float* in, float* outp, int N,
                                                    void* stream) {
     clear_error();
     if (!net || !in || !outp) return fail(SBNN_ERR_NULL, "net, in_dev and out_dev must not be NULL");
     if (layer < 0 || layer >= SBNN_MBV1_NUM_LAYERS) return fail(SBNN_ERR_SHAPE, "layer %d out of range", layer);
-    if (N < 0) return fail(SBNN_ERR_SHAPE, "N=%d", N);
+    if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
+    if (N == 0) return SBNN_OK;
+    // The chain's kernels work on channel-major buffers; this entry point takes and returns NHWC, so
+    // it converts on the way in and out through the network's own workspaces.
     const LayerShape& L = layer_table()[layer];
-    const int blk = (layer - 1) / 2;
-    switch (L.kind) {
-        case 0: return sbnn_conv3x3_dense(net->c0_w, net->c0_b, in, outp, N, L.hin, L.hin, L.cin, L.cout, L.stride, SBNN_RELU, stream);
-        case 1: return sbnn_dwconv3x3(net->dw_w[blk], net->dw_b[blk], in, outp, N, L.hin, L.hin, L.cin, L.stride, SBNN_RELU, stream);
-        case 2: return sbnn_conv1x1_gs(net->pw[blk], in, outp, N, L.hin, L.hin, SBNN_RELU, stream);
-        case 3: return sbnn_avgpool(in, outp, N, L.hin * L.hin, L.cin, stream);
-        default: return sbnn_conv1x1_gs(net->fc, in, outp, N, 1, 1, 0, stream);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int M_in = N * L.hin * L.hin, M_out = N * L.hout * L.hout;
+    const int ld_in = round4(M_in), ld_out = round4(M_out);
+    sbnn_status r;
+    if (L.kind == 4) return run_cm(net, layer, in, outp, N, stream);                     // classifier: [N][C] in, [N][1000] out
+    const float* src = in;
+    if (L.kind != 0) {                                                                   // NHWC [M][C] -> [C][ld]
+        if ((r = launch_transpose(in, L.cin, net->ws[0], ld_in, M_in, L.cin, st)) != SBNN_OK) return r;
+        src = net->ws[0];
     }
+    if (L.kind == 3) return run_cm(net, layer, src, outp, N, stream);                    // pool writes [N][C] directly
+    if ((r = run_cm(net, layer, src, net->ws[1], N, stream)) != SBNN_OK) return r;
+    return launch_transpose(net->ws[1], ld_out, outp, L.cout, L.cout, M_out, st);        // [C][ld] -> NHWC
 }
 
 extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_dev, float* logits_dev, int N,
@@ -140,7 +177,7 @@ extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_
     const float* cur = x_dev;
     for (int l = 0; l < SBNN_MBV1_NUM_LAYERS; ++l) {
         float* dst = (l == SBNN_MBV1_NUM_LAYERS - 1) ? logits_dev : net->ws[l & 1];
-        sbnn_status st = sbnn_mobilenet_v1_run_layer(net, l, cur, dst, N, stream);
+        sbnn_status st = run_cm(net, l, cur, dst, N, stream);
         if (st != SBNN_OK) return st;
         cur = dst;
     }
