@@ -29,66 +29,97 @@ transpose_kernel(const float* __restrict__ in, int ld_in, float* __restrict__ ou
 
 // ---- depthwise 3x3 on channel-major planes ------------------------------------------------------
 // Rows of the whole batch are numbered f = n*Ho + oy on the output side and g = n*H + iy on the input
-// side; with H = S*Ho the input rows of output row f are S*f - 1 .. S*f + 1, so a CTA's block of TR
-// output rows needs one contiguous span of input rows, which it stages in shared memory with
-// coalesced loads.  A thread then computes up to 4 consecutive outputs of one row from a 3 x (3S+3)
-// register window.  Rows that belong to a neighbouring image are masked by the row index inside the
-// image (top padding; bottom padding for stride 1).
+// side; with H = S*Ho the input rows of output row f are S*f - 1 .. S*f + 1.  Rows that belong to a
+// neighbouring image are masked by the row index inside the image.
+//
+// Vector kernel (W and Wo multiples of 4): a thread owns 4 consecutive outputs of one row and one
+// channel.  Per input row it reads the aligned float4 under its strip and the float4s left and right
+// of it (the neighbours' strips, so those reads hit L1); consecutive lanes own consecutive strips,
+// which makes every access a contiguous 512-byte warp transaction.
 template <int S>
 __global__ void __launch_bounds__(256)
-dwconv3x3_cm_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
-                    float* __restrict__ y, int ldy, int N, int H, int W, int Ho, int Wo, int TR, int SPR, int relu) {
-    extern __shared__ float xs[];   // (S*TR + 2) rows x W
-    const int c = blockIdx.y;
-    const int f0 = blockIdx.x * TR;
-    const long long NHo = (long long)N * Ho, NH = (long long)N * H;
-    const int in_rows = S * TR + 2;
-    const long long g0 = (long long)S * f0 - 1;          // first staged input row (may be -1)
-    const float* xc = x + (size_t)c * ldx;
-    for (int i = threadIdx.x; i < in_rows * W; i += blockDim.x) {
-        const long long g = g0 + i / W;
-        xs[i] = (g >= 0 && g < NH) ? __ldg(xc + g * W + (i % W)) : 0.0f;
-    }
+dwconv3x3_cm_vec_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
+                        float* __restrict__ y, int ldy, long long NHo, int H, int W, int Ho, int Wo, int relu) {
+    const int c = blockIdx.y, C = gridDim.y;
+    const int spr = Wo >> 2;                                       // strips per output row
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= NHo * spr) return;
+    const int strip = (int)(t % spr);
+    const long long f = t / spr;
+    const int oy = (int)(f % Ho);
     float wk[9];
 #pragma unroll
-    for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * gridDim.y + c);   // weights are [3][3][C]
+    for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);      // weights are [3][3][C]
     const float bias = b ? __ldg(b + c) : 0.0f;
-    __syncthreads();
-
-    const int lr = threadIdx.x / SPR, strip = threadIdx.x % SPR;
-    const long long f = (long long)f0 + lr;
-    if (lr >= TR || f >= NHo) return;
-    const int oy = (int)(f % Ho);
-    const int ox0 = strip * 4;
-    constexpr int IW = 3 * S + 3;
     float acc[4] = {bias, bias, bias, bias};
+    const float* xc = x + (size_t)c * ldx;
+    const int ix0 = strip * 4 * S;                                 // first input column under the strip
 #pragma unroll
     for (int kh = 0; kh < 3; ++kh) {
         const int iy = oy * S + kh - 1;
-        if (iy < 0 || iy >= H) continue;                 // row of another image or outside: zero padding
-        const float* row = xs + (S * lr + kh) * W;       // staged row g0 + S*lr + kh = S*f + kh - 1
-        float in[IW];
+        if (iy < 0 || iy >= H) continue;
+        const float* row = xc + (f * S + kh - 1) * W;              // input row g = S*f + kh - 1
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 L = ix0 >= 4 ? __ldg(reinterpret_cast<const float4*>(row + ix0 - 4)) : z;
+        const float4 A = __ldg(reinterpret_cast<const float4*>(row + ix0));
+        const float k0 = wk[kh * 3], k1 = wk[kh * 3 + 1], k2 = wk[kh * 3 + 2];
+        if constexpr (S == 1) {
+            const float4 R = ix0 + 4 < W ? __ldg(reinterpret_cast<const float4*>(row + ix0 + 4)) : z;
+            const float in[6] = {L.w, A.x, A.y, A.z, A.w, R.x};
 #pragma unroll
-        for (int j = 0; j < IW; ++j) {
-            const int ix = ox0 * S - 1 + j;
-            in[j] = (ix >= 0 && ix < W) ? row[ix] : 0.0f;
+            for (int i = 0; i < 4; ++i) acc[i] = fmaf(in[i + 2], k2, fmaf(in[i + 1], k1, fmaf(in[i], k0, acc[i])));
+        } else {
+            const float4 B = __ldg(reinterpret_cast<const float4*>(row + ix0 + 4));   // ix0 + 7 < W always
+            const float in[9] = {L.w, A.x, A.y, A.z, A.w, B.x, B.y, B.z, B.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                acc[i] = fmaf(in[2 * i + 2], k2, fmaf(in[2 * i + 1], k1, fmaf(in[2 * i], k0, acc[i])));
         }
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int kw = 0; kw < 3; ++kw) acc[i] = fmaf(in[i * S + kw], wk[kh * 3 + kw], acc[i]);
     }
-    float* yp = y + (size_t)c * ldy + f * Wo + ox0;
     if (relu) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[i] = fmaxf(acc[i], 0.0f);
     }
-    if (ox0 + 3 < Wo && ((f * Wo + ox0) & 3) == 0) {
-        *reinterpret_cast<float4*>(yp) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    } else {
+    *reinterpret_cast<float4*>(y + (size_t)c * ldy + f * Wo + strip * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+}
+
+// Kernel for the other widths (the 14- and 7-wide maps of the network).  A thread owns one output
+// position (oy, ox) of one channel in up to NI consecutive images: the index arithmetic and the
+// padding masks are computed once and reused for every image.  Consecutive lanes own consecutive
+// positions of the plane, so each of the 9 taps is one shifted, contiguous window.
+template <int S, int NI>
+__global__ void __launch_bounds__(256)
+dwconv3x3_cm_px_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
+                       float* __restrict__ y, int ldy, int N, int H, int W, int Ho, int Wo, int QB, int relu) {
+    const int c = blockIdx.y, C = gridDim.y;
+    const int q = (blockIdx.x % QB) * blockDim.x + threadIdx.x;     // position inside an output plane
+    const int n0 = (blockIdx.x / QB) * NI;                           // first image of this thread
+    const int HoWo = Ho * Wo;
+    if (q >= HoWo) return;
+    const int oy = q / Wo, ox = q - oy * Wo;
+    float wk[9];
+    int off[9];
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (ox0 + i < Wo) yp[i] = acc[i];
+    for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+        for (int kw = 0; kw < 3; ++kw) {
+            const int iy = oy * S + kh - 1, ix = ox * S + kw - 1;
+            const bool ok = iy >= 0 && iy < H && ix >= 0 && ix < W;
+            off[kh * 3 + kw] = ok ? iy * W + ix : 0;                 // a masked tap reads position 0 with weight 0
+            wk[kh * 3 + kw] = ok ? __ldg(w + (kh * 3 + kw) * C + c) : 0.0f;
+        }
+    const float bias = b ? __ldg(b + c) : 0.0f;
+    const float* xc = x + (size_t)c * ldx;
+    float* yc = y + (size_t)c * ldy + q;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const int n = n0 + i;
+        if (n >= N) break;
+        const float* xi = xc + (size_t)n * H * W;
+        float acc = bias;
+#pragma unroll
+        for (int t = 0; t < 9; ++t) acc = fmaf(__ldg(xi + off[t]), wk[t], acc);
+        yc[(size_t)n * HoWo] = relu ? fmaxf(acc, 0.0f) : acc;
     }
 }
 
@@ -196,21 +227,26 @@ sbnn_status launch_transpose(const float* in, int ld_in, float* out, int ld_out,
 sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, int ldx, float* y, int ldy, int N, int H,
                                 int W, int C, int stride, int relu, cudaStream_t st) {
     const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
-    if (H != stride * Ho) return fail(SBNN_ERR_UNSUPPORTED, "channel-major depthwise needs H divisible by the stride");
-    const int SPR = (Wo + 3) / 4;
-    if (SPR > 256) return fail(SBNN_ERR_UNSUPPORTED, "channel-major depthwise: row of %d pixels too wide", Wo);
-    int TR = 256 / SPR;
-    // keep the staged input span within the default shared-memory budget
-    while (TR > 1 && (size_t)(stride * TR + 2) * W * sizeof(float) > 40 * 1024) TR /= 2;
-    const size_t smem = (size_t)(stride * TR + 2) * W * sizeof(float);
-    if (smem > 48 * 1024) return fail(SBNN_ERR_UNSUPPORTED, "channel-major depthwise: row of %d pixels too wide", W);
-    const long long NHo = (long long)N * Ho;
-    dim3 grid((unsigned)((NHo + TR - 1) / TR), C);
+    if (H != stride * Ho || W != stride * Wo)
+        return fail(SBNN_ERR_UNSUPPORTED, "channel-major depthwise needs H and W divisible by the stride");
     if (C > 65535) return fail(SBNN_ERR_SHAPE, "too many channels");
-    if (stride == 1)
-        dwconv3x3_cm_kernel<1><<<grid, 256, smem, st>>>(w, b, x, ldx, y, ldy, N, H, W, Ho, Wo, TR, SPR, relu);
-    else
-        dwconv3x3_cm_kernel<2><<<grid, 256, smem, st>>>(w, b, x, ldx, y, ldy, N, H, W, Ho, Wo, TR, SPR, relu);
+    const long long NHo = (long long)N * Ho;
+    if (W % 4 == 0 && Wo % 4 == 0 && ldx % 4 == 0 && ldy % 4 == 0) {
+        const long long threads = NHo * (Wo / 4);
+        dim3 grid((unsigned)((threads + 255) / 256), C);
+        if (stride == 1)
+            dwconv3x3_cm_vec_kernel<1><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu);
+        else
+            dwconv3x3_cm_vec_kernel<2><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu);
+    } else {
+        constexpr int NI = 4;
+        const int QB = (Ho * Wo + 255) / 256;
+        dim3 grid((unsigned)(QB * ((N + NI - 1) / NI)), C);
+        if (stride == 1)
+            dwconv3x3_cm_px_kernel<1, NI><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, Ho, Wo, QB, relu);
+        else
+            dwconv3x3_cm_px_kernel<2, NI><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, Ho, Wo, QB, relu);
+    }
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
 }
