@@ -84,42 +84,50 @@ dwconv3x3_cm_vec_kernel(const float* __restrict__ w, const float* __restrict__ b
 }
 
 // Kernel for the other widths (the 14- and 7-wide maps of the network).  A thread owns one output
-// position (oy, ox) of one channel in up to NI consecutive images: the index arithmetic and the
-// padding masks are computed once and reused for every image.  Consecutive lanes own consecutive
-// positions of the plane, so each of the 9 taps is one shifted, contiguous window.
-template <int S, int NI>
+// position (oy, ox) of one channel in up to NI consecutive images: the padding masks are computed
+// once and reused for every image.  Consecutive lanes own consecutive positions of the plane, so each
+// of the 9 taps is one shifted, contiguous window.  WT > 0 fixes the input width at compile time, which
+// turns the 9 tap offsets into immediates of the load instructions (the kernel is bound by
+// instruction issue, not by memory).
+template <int S, int NI, int WT>
 __global__ void __launch_bounds__(256)
 dwconv3x3_cm_px_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
-                       float* __restrict__ y, int ldy, int N, int H, int W, int Ho, int Wo, int QB, int relu) {
+                       float* __restrict__ y, int ldy, int N, int H, int Wrt, int QB, int relu) {
+    const int W = WT ? WT : Wrt;
+    const int Ho = H / S, Wo = W / S;
     const int c = blockIdx.y, C = gridDim.y;
     const int q = (blockIdx.x % QB) * blockDim.x + threadIdx.x;     // position inside an output plane
     const int n0 = (blockIdx.x / QB) * NI;                           // first image of this thread
-    const int HoWo = Ho * Wo;
+    const int HoWo = Ho * Wo, HW = H * W;
     if (q >= HoWo) return;
     const int oy = q / Wo, ox = q - oy * Wo;
     float wk[9];
-    int off[9];
+    bool ok[9];
 #pragma unroll
     for (int kh = 0; kh < 3; ++kh)
 #pragma unroll
         for (int kw = 0; kw < 3; ++kw) {
             const int iy = oy * S + kh - 1, ix = ox * S + kw - 1;
-            const bool ok = iy >= 0 && iy < H && ix >= 0 && ix < W;
-            off[kh * 3 + kw] = ok ? iy * W + ix : 0;                 // a masked tap reads position 0 with weight 0
-            wk[kh * 3 + kw] = ok ? __ldg(w + (kh * 3 + kw) * C + c) : 0.0f;
+            ok[kh * 3 + kw] = iy >= 0 && iy < H && ix >= 0 && ix < W;
+            wk[kh * 3 + kw] = __ldg(w + (kh * 3 + kw) * C + c);
         }
     const float bias = b ? __ldg(b + c) : 0.0f;
-    const float* xc = x + (size_t)c * ldx;
-    float* yc = y + (size_t)c * ldy + q;
+    const float* pc = x + (size_t)c * ldx + (size_t)n0 * HW + oy * S * W + ox * S;   // centre tap, first image
+    float* yc = y + (size_t)c * ldy + (size_t)n0 * HoWo + q;
 #pragma unroll
     for (int i = 0; i < NI; ++i) {
-        const int n = n0 + i;
-        if (n >= N) break;
-        const float* xi = xc + (size_t)n * H * W;
+        if (n0 + i >= N) break;
         float acc = bias;
 #pragma unroll
-        for (int t = 0; t < 9; ++t) acc = fmaf(__ldg(xi + off[t]), wk[t], acc);
-        yc[(size_t)n * HoWo] = relu ? fmaxf(acc, 0.0f) : acc;
+        for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+            for (int kw = 0; kw < 3; ++kw) {
+                const float v = ok[kh * 3 + kw] ? __ldg(pc + (kh - 1) * W + (kw - 1)) : 0.0f;
+                acc = fmaf(v, wk[kh * 3 + kw], acc);
+            }
+        *yc = relu ? fmaxf(acc, 0.0f) : acc;
+        pc += HW;
+        yc += HoWo;
     }
 }
 
@@ -242,10 +250,17 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
         constexpr int NI = 4;
         const int QB = (Ho * Wo + 255) / 256;
         dim3 grid((unsigned)(QB * ((N + NI - 1) / NI)), C);
-        if (stride == 1)
-            dwconv3x3_cm_px_kernel<1, NI><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, Ho, Wo, QB, relu);
-        else
-            dwconv3x3_cm_px_kernel<2, NI><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, Ho, Wo, QB, relu);
+#define SBNN_DW_PX(S_, WT_) dwconv3x3_cm_px_kernel<S_, NI, WT_><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, QB, relu)
+        if (stride == 1) {
+            if (W == 14) SBNN_DW_PX(1, 14);
+            else if (W == 7) SBNN_DW_PX(1, 7);
+            else SBNN_DW_PX(1, 0);
+        } else {
+            if (W == 28) SBNN_DW_PX(2, 28);
+            else if (W == 14) SBNN_DW_PX(2, 14);
+            else SBNN_DW_PX(2, 0);
+        }
+#undef SBNN_DW_PX
     }
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
