@@ -115,9 +115,10 @@ def oracle_forward_seconds(x1, layers):
 def cpu_baseline(x, layers):
     from oracle import reference as R
     R.num_threads()                      # loads the library outside the timed part
-    dt = oracle_forward_seconds(x[:1], layers)
-    return {"value": 1.0 / dt, "unit": "images/s", "cores": R.num_threads(), "kind": "oracle",
-            "sample": f"1 image of the batch through the whole chain (error-bound pass included), {dt:.2f} s"}
+    n = min(len(x), 32)
+    dt = oracle_forward_seconds(x[:n], layers)
+    return {"value": n / dt, "unit": "images/s", "cores": R.num_threads(), "kind": "oracle",
+            "sample": f"{n} images of the batch through the whole chain (error-bound pass included), {dt:.1f} s"}
 
 
 def run_reference(args, rank):
@@ -161,20 +162,30 @@ def build_network(sbnn, torch, layers, batch):
 
 
 def time_layers(sbnn, torch, net, layers, batch, reps, flush):
-    """Every layer alone (run_layer on buffers of its own shape), CUDA events, L2 flushed between launches."""
+    """Every layer alone, as forward launches it (channel-major buffers of its own shape), CUDA events, L2 flushed
+    between launches."""
     res = []
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for li, L in enumerate(layers):
         hin, cin, hout, cout = sbnn.mobilenet_v1_layer_shape(li)
-        xin = torch.rand((batch, hin, hin, cin), device="cuda")
-        yout = torch.empty((batch, hout, hout, cout), device="cuda")
+        r4 = lambda v: (v + 3) // 4 * 4  # noqa: E731
+        if L["kind"] == "conv0":
+            xin = torch.rand((batch, hin, hin, cin), device="cuda")
+        elif L["kind"] == "fc":
+            xin = torch.rand((batch, cin), device="cuda")
+        else:
+            xin = torch.rand((cin, r4(batch * hin * hin)), device="cuda")
+        if L["kind"] in ("pool", "fc"):
+            yout = torch.empty((batch, cout), device="cuda")
+        else:
+            yout = torch.empty((cout, r4(batch * hout * hout)), device="cuda")
         for _ in range(3):
-            net.run_layer(li, xin, yout, batch)
+            net.run_layer_cm(li, xin, yout, batch)
         ts = []
         for _ in range(reps):
             flush.add_(1.0)
             ev0.record()
-            net.run_layer(li, xin, yout, batch)
+            net.run_layer_cm(li, xin, yout, batch)
             ev1.record()
             ev1.synchronize()
             ts.append(ev0.elapsed_time(ev1) * 1e-3)

@@ -54,6 +54,7 @@ def lib():
         "sbnn_mobilenet_v1_create": [P, P, P, P, P, P, I, P],
         "sbnn_mobilenet_v1_forward": [P, P, P, I, P],
         "sbnn_mobilenet_v1_run_layer": [P, I, P, P, I, P],
+        "sbnn_mobilenet_v1_run_layer_cm": [P, I, P, P, I, P],
         "sbnn_mobilenet_v1_layer_shape": [I, P, P, P, P],
         "sbnn_mobilenet_v1_free": [P],
         "sbnn_get_async_status": [P],
@@ -228,6 +229,10 @@ class MobileNetV1:
 
     def run_layer(self, layer, x, y, n, stream=None):
         _check(lib().sbnn_mobilenet_v1_run_layer(self._h, layer, _ptr(x), _ptr(y), n, _stream(stream)))
+
+    def run_layer_cm(self, layer, x, y, n, stream=None):
+        """One layer on the chain's channel-major buffers (no layout conversion)."""
+        _check(lib().sbnn_mobilenet_v1_run_layer_cm(self._h, layer, _ptr(x), _ptr(y), n, _stream(stream)))
 
     def free(self):
         if self._h:

@@ -205,6 +205,85 @@ conv3x3_thin_cm_kernel(const float* __restrict__ w, const float* __restrict__ b,
     }
 }
 
+// Wide variant for Cout % 32 == 0: one thread computes 2 consecutive output columns x 32 output
+// channels, so every input value is loaded once per pixel pair (not once per channel group) and each
+// broadcast float4 of weights feeds 8 FMAs.  Consecutive lanes take consecutive column pairs; a
+// channel's stores are 8-byte pieces that are contiguous across the warp.
+template <int S>
+__global__ void __launch_bounds__(128)
+conv3x3_thin_cm32_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x,
+                         float* __restrict__ y, int ldy, int N, int H, int W, int Cin, int Cout, int Ho, int Wo, int relu) {
+    extern __shared__ __align__(16) float ws[];   // [9][Cin][32] of this CTA's channel group
+    const int cg = blockIdx.y;
+    for (int i = threadIdx.x; i < 9 * Cin * 32; i += blockDim.x) {
+        const int o = i & 31, tc = i >> 5;
+        ws[i] = w[(size_t)(cg * 32 + o) * 9 * Cin + tc];
+    }
+    __syncthreads();
+    constexpr int TW = 2, IW = S * (TW - 1) + 3;
+    const int strips = (Wo + TW - 1) / TW;
+    const long long total = (long long)N * Ho * strips;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= total) return;
+    const int sx = (int)(t % strips);
+    const long long f = t / strips;
+    const int oy = (int)(f % Ho);
+    const int n = (int)(f / Ho);
+    const int ox0 = sx * TW, ix0 = ox0 * S - 1;
+
+    float acc[TW][32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const float bv = b ? __ldg(b + cg * 32 + j) : 0.f;
+#pragma unroll
+        for (int i = 0; i < TW; ++i) acc[i][j] = bv;
+    }
+#pragma unroll
+    for (int kh = 0; kh < 3; ++kh) {
+        const int iy = oy * S + kh - 1;
+        if (iy < 0 || iy >= H) continue;
+        const float* row = x + ((size_t)n * H + iy) * W * Cin;
+        for (int c = 0; c < Cin; ++c) {
+            float in[IW];
+#pragma unroll
+            for (int j = 0; j < IW; ++j) {
+                const int ix = ix0 + j;
+                in[j] = (ix >= 0 && ix < W) ? __ldg(row + (size_t)ix * Cin + c) : 0.f;
+            }
+#pragma unroll
+            for (int kw = 0; kw < 3; ++kw) {
+                const float4* wp = reinterpret_cast<const float4*>(ws + ((kh * 3 + kw) * Cin + c) * 32);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const float4 wv = wp[v];
+#pragma unroll
+                    for (int i = 0; i < TW; ++i) {
+                        const float a = in[i * S + kw];
+                        acc[i][4 * v + 0] = fmaf(a, wv.x, acc[i][4 * v + 0]);
+                        acc[i][4 * v + 1] = fmaf(a, wv.y, acc[i][4 * v + 1]);
+                        acc[i][4 * v + 2] = fmaf(a, wv.z, acc[i][4 * v + 2]);
+                        acc[i][4 * v + 3] = fmaf(a, wv.w, acc[i][4 * v + 3]);
+                    }
+                }
+            }
+        }
+    }
+    const long long p0 = f * Wo + ox0;
+    const bool vec = (ox0 + 1 < Wo) && ((p0 & 1) == 0);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        float v0 = acc[0][j], v1 = acc[1][j];
+        if (relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+        float* yp = y + (size_t)(cg * 32 + j) * ldy + p0;
+        if (vec) {
+            *reinterpret_cast<float2*>(yp) = make_float2(v0, v1);
+        } else {
+            yp[0] = v0;
+            if (ox0 + 1 < Wo) yp[1] = v1;
+        }
+    }
+}
+
 // ---- global average pool: channel-major in ([C][ld], pixel index n*HW + p), [N][C] out -----------
 // One warp per (channel, image): the HW values are contiguous; lanes stride over them and reduce.
 __global__ void __launch_bounds__(256)
@@ -269,6 +348,19 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
 sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* x, float* y, int ldy, int N, int H, int W,
                                    int Cin, int Cout, int stride, int relu, cudaStream_t st) {
     const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+    if (Cout % 32 == 0 && ldy % 2 == 0) {
+        const long long total = (long long)N * Ho * ((Wo + 1) / 2);
+        const long long blocks = (total + 127) / 128;
+        if (blocks > 0x7fffffff) return fail(SBNN_ERR_SHAPE, "tensor too large");
+        dim3 grid((unsigned)blocks, Cout / 32);
+        const size_t smem = sizeof(float) * 9 * Cin * 32;
+        if (stride == 1)
+            conv3x3_thin_cm32_kernel<1><<<grid, 128, smem, st>>>(w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu);
+        else
+            conv3x3_thin_cm32_kernel<2><<<grid, 128, smem, st>>>(w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu);
+        SBNN_CUDA_TRY(cudaGetLastError());
+        return SBNN_OK;
+    }
     const long long total = (long long)N * Ho * ((Wo + 3) / 4);
     const long long blocks = (total + 255) / 256;
     if (blocks > 0x7fffffff) return fail(SBNN_ERR_SHAPE, "tensor too large");

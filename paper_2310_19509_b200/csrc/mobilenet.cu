@@ -167,6 +167,17 @@ extern "C" sbnn_status sbnn_mobilenet_v1_run_layer(sbnn_mbv1* net, int layer, co
     return launch_transpose(net->ws[1], ld_out, outp, L.cout, L.cout, M_out, st);        // [C][ld] -> NHWC
 }
 
+extern "C" sbnn_status sbnn_mobilenet_v1_run_layer_cm(sbnn_mbv1* net, int layer, const float* in, float* outp, int N,
+                                                      void* stream) {
+    clear_error();
+    if (!net || !in || !outp) return fail(SBNN_ERR_NULL, "net, in_dev and out_dev must not be NULL");
+    if (layer < 0 || layer >= SBNN_MBV1_NUM_LAYERS) return fail(SBNN_ERR_SHAPE, "layer %d out of range", layer);
+    if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
+    if (!aligned16(in) || !aligned16(outp)) return fail(SBNN_ERR_ALIGN, "in_dev and out_dev must be 16-byte aligned");
+    if (N == 0) return SBNN_OK;
+    return run_cm(net, layer, in, outp, N, stream);
+}
+
 extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_dev, float* logits_dev, int N,
                                                  void* stream) {
     clear_error();

@@ -314,3 +314,20 @@ def test_bf16_mode_on_config5_shape_reduced_batch():
     y = run_1x1(d, sbnn.SBNN_BF16_TC | sbnn.SBNN_RELU)
     ref16, s16 = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True, bf16=True)
     assert_within(y, ref16, s16, tol=1e-5, what="config 5 G=8 bf16")
+
+
+def test_mobilenet_layer_on_channel_major_buffers():
+    """run_layer_cm (what forward launches) against the oracle for one depthwise and one pointwise layer."""
+    x, layers = mobilenet_v1_inputs(1, 50, 4, seed=1)
+    outs = R.mobilenet_v1_forward(x, layers[:5])
+    net = build_net(layers, 1)
+    for li in (1, 2, 3, 4):
+        rec = outs[li]
+        hin, cin, hout, cout = sbnn.mobilenet_v1_layer_shape(li)
+        xin = dev(np.ascontiguousarray(rec["in"].reshape(hin * hin, cin).T))      # [C][M]
+        yd = torch.full((cout, hout * hout), float("nan"), device="cuda")
+        net.run_layer_cm(li, xin, yd, 1)
+        sbnn.get_async_status()
+        y = yd.cpu().numpy().T.reshape(rec["ref"].shape)
+        assert_within(y, rec["ref"], rec["S"], what=f"cm layer {li}")
+    net.free()
