@@ -171,11 +171,9 @@ def time_layers(sbnn, torch, net, layers, batch, reps, flush):
         r4 = lambda v: (v + 3) // 4 * 4  # noqa: E731
         if L["kind"] == "conv0":
             xin = torch.rand((batch, hin, hin, cin), device="cuda")
-        elif L["kind"] == "fc":
-            xin = torch.rand((batch, cin), device="cuda")
         else:
             xin = torch.rand((cin, r4(batch * hin * hin)), device="cuda")
-        if L["kind"] in ("pool", "fc"):
+        if L["kind"] == "fc":
             yout = torch.empty((batch, cout), device="cuda")
         else:
             yout = torch.empty((cout, r4(batch * hout * hout)), device="cuda")

@@ -235,8 +235,8 @@ SBNN_API sbnn_status sbnn_mobilenet_v1_run_layer(sbnn_mbv1* net, int layer, cons
 /*
  * The same layer in the chain's own activation layout, without conversions (what forward launches):
  * in_dev and out_dev are channel-major, [C][ld] with ld = N*side*side rounded up to a multiple of 4 and
- * the pixel index n*side*side + y*side + x.  Exceptions: layer 0 reads the NHWC image, the pool
- * (layer 27) writes [N][1024], the classifier (layer 28) reads [N][1024] and writes [N][1000].
+ * the pixel index n*side*side + y*side + x (the pool's output has side 1: [1024][N rounded up to 4]).
+ * Exceptions: layer 0 reads the NHWC image, the classifier (layer 28) writes [N][1000].
  */
 SBNN_API sbnn_status sbnn_mobilenet_v1_run_layer_cm(sbnn_mbv1* net, int layer, const float* in_dev, float* out_dev,
                                                     int N, void* cuda_stream);

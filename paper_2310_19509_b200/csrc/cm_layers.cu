@@ -284,10 +284,10 @@ conv3x3_thin_cm32_kernel(const float* __restrict__ w, const float* __restrict__ 
     }
 }
 
-// ---- global average pool: channel-major in ([C][ld], pixel index n*HW + p), [N][C] out -----------
+// ---- global average pool: channel-major in ([C][ld], pixel index n*HW + p), channel-major [C][ldy] out --
 // One warp per (channel, image): the HW values are contiguous; lanes stride over them and reduce.
 __global__ void __launch_bounds__(256)
-avgpool_cm_kernel(const float* __restrict__ x, int ldx, float* __restrict__ y, int N, int HW, int C) {
+avgpool_cm_kernel(const float* __restrict__ x, int ldx, float* __restrict__ y, int ldy, int N, int HW, int C) {
     const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (wid >= N * C) return;
     const int n = wid % N, c = wid / N;
@@ -296,7 +296,7 @@ avgpool_cm_kernel(const float* __restrict__ x, int ldx, float* __restrict__ y, i
     for (int i = lane; i < HW; i += 32) s += __ldg(p + i);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (lane == 0) y[(size_t)n * C + c] = s * (1.0f / (float)HW);
+    if (lane == 0) y[(size_t)c * ldy + n] = s * (1.0f / (float)HW);
 }
 
 }  // namespace
@@ -374,9 +374,9 @@ sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* 
     return SBNN_OK;
 }
 
-sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int N, int HW, int C, cudaStream_t st) {
+sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int ldy, int N, int HW, int C, cudaStream_t st) {
     const long long threads = (long long)N * C * 32;
-    avgpool_cm_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(x, ldx, y, N, HW, C);
+    avgpool_cm_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(x, ldx, y, ldy, N, HW, C);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
 }

@@ -89,6 +89,7 @@ sbnn_status prepare_default_1x1(const sbnn_packed* p);
 void free_streams_1x1(sbnn_packed* p);
 // conv1x1_cm.cu
 sbnn_status prepare_default_cm(const sbnn_packed* p);
+sbnn_status prepare_cm(const sbnn_packed* p, int P, int GPW, int NW, int KC);   // builds the stream of one tile shape
 void free_streams_cm(sbnn_packed* p);
 // Runs the NHWC call through the channel-major kernel if the shape profits; *done tells whether it did.
 sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st, bool* done);
@@ -99,7 +100,7 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
                                 int W, int C, int stride, int relu, cudaStream_t st);
 sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* x, float* y, int ldy, int N, int H, int W,
                                    int Cin, int Cout, int stride, int relu, cudaStream_t st);
-sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int N, int HW, int C, cudaStream_t st);
+sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int ldy, int N, int HW, int C, cudaStream_t st);
 // conv1x1_bf16.cu
 sbnn_status conv1x1_bf16(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st);
 void free_stream_bf16(sbnn_packed* p);

@@ -550,6 +550,11 @@ sbnn_status prepare_default_cm(const sbnn_packed* p) {
     return get_stream_cm(p, default_cfg_cm(p), &s);
 }
 
+sbnn_status prepare_cm(const sbnn_packed* p, int P, int GPW, int NW, int KC) {
+    Stream1x1 s;
+    return get_stream_cm(p, TileCfg{P, GPW, NW, KC}, &s);
+}
+
 void free_streams_cm(sbnn_packed* p) {
     for (auto& kv : p->streams_cm) {
         cudaFree(kv.second.rec);

@@ -41,6 +41,15 @@ const LayerShape* layer_table() {
     return tab.t;
 }
 
+inline int round4(long long v) { return (int)((v + 3) / 4 * 4); }
+
+// Tile of the channel-major 1x1 kernel used for the classifier (0s = the layer's default).
+inline void fc_tile(int G, int* P, int* GPW, int* NW, int* KC) {
+    *P = *GPW = *NW = *KC = 0;
+    if (G == 4 || G == 16) { *P = 4; *GPW = 1; *NW = 8; *KC = 32; }
+    if (G == 8) { *P = 4; *GPW = 1; *NW = 16; *KC = 32; }
+}
+
 }  // namespace
 }  // namespace sbnn
 
@@ -96,6 +105,12 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
         if (pw[i]->device < 0) return fail(SBNN_ERR_CUDA, "pointwise layer %d was packed without a CUDA device", i + 1);
         if ((st = prepare_default_cm(pw[i])) != SBNN_OK) return st;
     }
+    if (fc->device < 0) return fail(SBNN_ERR_CUDA, "the classifier was packed without a CUDA device");
+    {
+        int P, GPW, NW, KC;
+        fc_tile(fc->G, &P, &GPW, &NW, &KC);
+        if ((st = P ? prepare_cm(fc, P, GPW, NW, KC) : prepare_default_cm(fc)) != SBNN_OK) return st;
+    }
     sbnn_mbv1* n = new (std::nothrow) sbnn_mbv1;
     if (!n) return fail(SBNN_ERR_ALLOC, "out of host memory");
     for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
@@ -122,7 +137,6 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
 
 namespace {
 
-inline int round4(long long v) { return (int)((v + 3) / 4 * 4); }
 
 // One layer on channel-major buffers.  in: channel-major [Cin][ld_in] (layer 0: the NHWC image);
 // out: channel-major [Cout][ld_out] (pool: [N][C]; classifier: [N][1000], reading the pooled [N][C]).
@@ -135,8 +149,12 @@ sbnn_status run_cm(sbnn_mbv1* net, int layer, const float* in, float* out, int N
         case 0: return launch_conv3x3_thin_cm(net->c0_w, net->c0_b, in, out, ld_out, N, L.hin, L.hin, L.cin, L.cout, L.stride, 1, st);
         case 1: return launch_dwconv3x3_cm(net->dw_w[blk], net->dw_b[blk], in, ld_in, out, ld_out, N, L.hin, L.hin, L.cin, L.stride, 1, st);
         case 2: return sbnn_conv1x1_gs_cm(net->pw[blk], in, ld_in, out, ld_out, N * L.hin * L.hin, SBNN_RELU | SBNN_OUT_CM, 0, 0, 0, 0, stream);
-        case 3: return launch_avgpool_cm(in, ld_in, out, N, L.hin * L.hin, L.cin, st);
-        default: return sbnn_conv1x1_gs(net->fc, in, out, N, 1, 1, 0, stream);
+        case 3: return launch_avgpool_cm(in, ld_in, out, round4(N), N, L.hin * L.hin, L.cin, st);
+        default: {   // classifier: pooled features [1024][ld] in, logits [N][1000] out; few pixels, so a narrow tile
+            int P, GPW, NW, KC;
+            fc_tile(net->fc->G, &P, &GPW, &NW, &KC);
+            return sbnn_conv1x1_gs_cm(net->fc, in, round4(N), out, L.cout, N, 0, P, GPW, NW, KC, stream);
+        }
     }
 }
 
@@ -156,13 +174,12 @@ extern "C" sbnn_status sbnn_mobilenet_v1_run_layer(sbnn_mbv1* net, int layer, co
     const int M_in = N * L.hin * L.hin, M_out = N * L.hout * L.hout;
     const int ld_in = round4(M_in), ld_out = round4(M_out);
     sbnn_status r;
-    if (L.kind == 4) return run_cm(net, layer, in, outp, N, stream);                     // classifier: [N][C] in, [N][1000] out
     const float* src = in;
     if (L.kind != 0) {                                                                   // NHWC [M][C] -> [C][ld]
         if ((r = launch_transpose(in, L.cin, net->ws[0], ld_in, M_in, L.cin, st)) != SBNN_OK) return r;
         src = net->ws[0];
     }
-    if (L.kind == 3) return run_cm(net, layer, src, outp, N, stream);                    // pool writes [N][C] directly
+    if (L.kind == 4) return run_cm(net, layer, src, outp, N, stream);                    // classifier writes [N][1000] directly
     if ((r = run_cm(net, layer, src, net->ws[1], N, stream)) != SBNN_OK) return r;
     return launch_transpose(net->ws[1], ld_out, outp, L.cout, L.cout, M_out, st);        // [C][ld] -> NHWC
 }
