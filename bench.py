@@ -28,6 +28,7 @@ import numpy as np  # noqa: E402
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FP32 lanes x 2 flop x max SM clock
 HBM_FALLBACK_GBS = 6650.0
 METRIC = "mobilenet_v1_images_per_s"
+PW_DRAM_BYTES_PER_STEP = 749.7e6
 
 
 def measured_peaks():
@@ -267,11 +268,14 @@ def run_gpu(args, rank, world, local_rank):
     t_roof = lambda r: max(r["flops"] / (FP32_PEAK_TFLOPS * 1e12), r["bytes"] / (hbm_gbs * 1e9))  # noqa: E731
     total_layer_t = sum(r["s"] for r in per)
     roofline = {
-        "bound": "alu", "kernel": "conv1x1_gs_kernel (13 pointwise launches per step)",
+        "bound": "alu", "kernel": "conv1x1_cm_kernel (13 pointwise launches per step)",
         "achieved": pw_fl / pw_t / 1e12, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s",
         "frac": pw_fl / pw_t / 1e12 / FP32_PEAK_TFLOPS,
         "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz (no measured FP32 peak on file)",
-        "traffic": None,
+        # dram__bytes_read.sum + dram__bytes_write.sum of the 13 launches of one step from the ncu capture in
+        # profiles/bench_mobilenet_v1_b64_s50_launch_list.md; valid for the default workload and this kernel only
+        "traffic": PW_DRAM_BYTES_PER_STEP if (batch == 64 and args.sparsity == 50) else None,
+        "algorithmic_bytes": pw_by,
         "mixed_frac": sum(t_roof(r) for r in pw) / pw_t,
         "mixed_note": f"sum over layers of max(nonzero flops/FP32 peak, bytes/{hbm_gbs:.0f} GB/s {peak_kind}) / measured",
         "hbm_achieved_gbs": pw_by / pw_t / 1e9,
