@@ -238,3 +238,41 @@ def mobilenet_v1_forward(x, layers, tol=1e-5):
         outs.append(rec)
         cur = ref.astype(np.float32)
     return outs
+
+
+def sample_outputs(x, w, mask, bias, positions, relu=True, bf16=False):
+    """The definition evaluated one output at a time, for checks at sizes where the full loops take too long.
+
+    positions: iterable of (n, y, x, o) output coordinates of a stride-1 convolution with zero padding
+    (K-1)/2.  Returns (ref, S) as float64 arrays of len(positions), computed as
+    b[o] + sum over taps and ALL input channels of w*m*x in fp64 (no zero skipping, as in conv2d).
+    """
+    x = np.asarray(x, dtype=np.float32)
+    w = np.asarray(w, dtype=np.float32)
+    mask = np.asarray(mask, dtype=np.uint8)
+    n_, h, wd, cin = x.shape
+    cout, kh, kw, _ = w.shape
+    ph, pw = (kh - 1) // 2, (kw - 1) // 2
+    ref = np.empty(len(positions), dtype=np.float64)
+    s = np.empty(len(positions), dtype=np.float64)
+    for i, (n, y, xx, o) in enumerate(positions):
+        b = float(bias[o]) if bias is not None else 0.0
+        acc, sa = b, abs(b)
+        for dy in range(kh):
+            iy = y + dy - ph
+            if iy < 0 or iy >= h:
+                continue
+            for dx in range(kw):
+                ix = xx + dx - pw
+                if ix < 0 or ix >= wd:
+                    continue
+                wm = np.where(mask[o, dy, dx] != 0, w[o, dy, dx], np.float32(0))
+                xv = x[n, iy, ix]
+                if bf16:
+                    wm, xv = bf16_round(wm), bf16_round(xv)
+                p = wm.astype(np.float64) * xv.astype(np.float64)
+                acc += float(p.sum())
+                sa += float(np.abs(p).sum())
+        ref[i] = max(acc, 0.0) if relu else acc
+        s[i] = sa
+    return ref, s

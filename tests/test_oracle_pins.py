@@ -233,3 +233,12 @@ def test_chain_error_bound_grows_and_layers_chain():
     np.testing.assert_array_equal(outs[1]["in"], outs[0]["ref"].astype(np.float32))
     assert np.all(outs[-1]["E"] >= 1e-5 * outs[-1]["S"])
     assert outs[-1]["ref"].shape == (1, 8, 8, 128)
+
+
+def test_sample_outputs_agrees_with_the_full_loops():
+    x, wt, b, m, _ = _rand_layer(2, 6, 5, 12, 8, 3, 4)
+    ref, s = R.conv2d(x, wt, m, b, relu=True)
+    pos = [(0, 0, 0, 0), (1, 5, 4, 7), (0, 3, 2, 5), (1, 0, 4, 2)]
+    r2, s2 = R.sample_outputs(x, wt, m, b, pos, relu=True)
+    for i, (n, y, xx, o) in enumerate(pos):
+        assert abs(r2[i] - ref[n, y, xx, o]) < 1e-12 and abs(s2[i] - s[n, y, xx, o]) < 1e-12
