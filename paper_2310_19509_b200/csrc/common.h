@@ -94,6 +94,8 @@ void free_streams_cm(sbnn_packed* p);
 // Runs the NHWC call through the channel-major kernel if the shape profits; *done tells whether it did.
 sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st, bool* done);
 sbnn_status read_async_status(int* value);
+// Per-device scratch buffer for channel-major copies made on behalf of NHWC callers (grows on demand, synchronously).
+sbnn_status scratch_workspace(size_t bytes, float** out);
 // cm_layers.cu: dense layers on channel-major activations ([C][ld]); arguments validated by the callers
 sbnn_status launch_transpose(const float* in, int ld_in, float* out, int ld_out, int R, int Ccols, cudaStream_t st);
 sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, int ldx, float* y, int ldy, int N, int H,

@@ -545,6 +545,8 @@ sbnn_status workspace(size_t bytes, float** out) {
 
 }  // namespace
 
+sbnn_status scratch_workspace(size_t bytes, float** out) { return workspace(bytes, out); }
+
 sbnn_status prepare_default_cm(const sbnn_packed* p) {
     Stream1x1 s;
     return get_stream_cm(p, default_cfg_cm(p), &s);

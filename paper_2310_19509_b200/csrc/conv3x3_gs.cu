@@ -22,6 +22,7 @@
 #include <algorithm>
 
 #include "common.h"
+#include "pipeline.cuh"
 
 namespace sbnn {
 namespace {
@@ -182,6 +183,177 @@ conv3x3_gs_kernel(const float* __restrict__ X, float* __restrict__ Y, const floa
     }
 }
 
+
+// ---- channel-major variant --------------------------------------------------------------------
+// Same decomposition, but X is given as planes ([Cin][ldx], pixel index f*W + x) with W a multiple of 4.
+// A plane row is then W/4 aligned 16-byte pieces, which cp.async copies straight into the shared
+// memory plane (column = x + 4, so pieces stay 16-byte aligned; column 3 is the zero column for x = -1):
+// no registers, no transposing stores, and the copies of step k+1 run while step k is computed
+// (two buffers).  Accumulators are packed pairs of output channels updated with fma.rn.f32x2.
+__device__ __forceinline__ void cp_async16_3(void* smem, const void* gmem) {
+    unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem) : "memory");
+}
+
+template <class C>
+__global__ void __launch_bounds__(C::NT, 1)
+conv3x3_gs_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, const float* __restrict__ bias,
+                     const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, Geo3 geo, int relu) {
+    constexpr int G = C::G, CW = C::CW, GPW = C::GPW, KC = C::KC;
+    constexpr int GP = (G + 1) / 2;                 // packed channel pairs per group
+    constexpr int NIT = 2;                          // staged (row, piece) positions per thread (checked on the host)
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int xs_floats = KC * geo.plane;
+    float* xs0 = reinterpret_cast<float*>(smem);                                          // two plane sets
+    uint4* ws0 = reinterpret_cast<uint4*>(smem + (size_t)2 * xs_floats * 4);              // two weight blocks
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pw = warp % C::NPW, gw = warp / C::NPW;
+    const int f0 = blockIdx.x * geo.R;
+    const int tile = blockIdx.y;
+    const int NH = geo.N * geo.H, W = geo.W;
+    const int32_t* bp = blk_ptr + (size_t)tile * (geo.nchunks + 1);
+
+    for (int i = tid; i < 2 * xs_floats; i += C::NT) xs0[i] = 0.0f;   // zero rows / columns stay zero for good
+
+    // staging: a thread owns up to NIT (staged row, 16-byte piece) positions and copies them for every
+    // channel of the step (source and destination advance by one plane per channel)
+    const int QW = W >> 2, rows = geo.R + 2, pieces = rows * QW;
+    int src_off[NIT], dst_off[NIT];
+#pragma unroll
+    for (int j = 0; j < NIT; ++j) {
+        const int i = tid + j * C::NT;
+        src_off[j] = -1;
+        dst_off[j] = 0;
+        if (i < pieces) {
+            const int q = i % QW, row = i / QW;
+            const long long f = (long long)f0 - 1 + row;
+            if (f >= 0 && f < NH) {
+                src_off[j] = (int)f * W + 4 * q;
+                dst_off[j] = (row + 1) * geo.pitch + 4 + 4 * q;
+            }
+        }
+    }
+    auto issue = [&](int k, int buf) {
+        const float* xk = X + (size_t)k * KC * ldx;
+        float* xd = xs0 + buf * xs_floats;
+        const int nc = min(KC, geo.Cin - k * KC);                                // channels of this step
+#pragma unroll
+        for (int j = 0; j < NIT; ++j)
+            if (src_off[j] >= 0)
+                for (int c = 0; c < nc; ++c) cp_async16_3(xd + c * geo.plane + dst_off[j], xk + (size_t)c * ldx + src_off[j]);
+        uint4* wd = ws0 + buf * C::WS_U4;
+        const int beg = bp[k], n = bp[k + 1] - beg;
+        for (int i = tid; i < n; i += C::NT) cp_async16_3(wd + i, rec + beg + i);
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+    };
+
+    const int lrow = pw * geo.RPW + lane / geo.LPR;
+    const int lx = (lane % geo.LPR) * CW;
+    const int f = f0 + lrow;
+    const int y = f % geo.H;
+    int rowoff[3];
+    rowoff[0] = (y > 0) ? (lrow + 1) * geo.pitch : 0;
+    rowoff[1] = (lrow + 2) * geo.pitch;
+    rowoff[2] = (y < geo.H - 1) ? (lrow + 3) * geo.pitch : 0;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) rowoff[k] += lx + 3;   // column of x = lx - 1
+
+    f32x2 acc[GPW][CW][GP];
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * C::GT + gw * GPW + q;
+#pragma unroll
+        for (int r = 0; r < GP; ++r) {
+            const float b0 = (g < geo.ngroups) ? bias[g * G + 2 * r] : 0.0f;
+            const float b1 = (g < geo.ngroups && 2 * r + 1 < G) ? bias[g * G + 2 * r + 1] : 0.0f;
+#pragma unroll
+            for (int p = 0; p < CW; ++p) acc[q][p][r] = pack2(b0, b1);
+        }
+    }
+
+    __syncthreads();            // zero fill done before the first copies land
+    issue(0, 0);
+    for (int k = 0; k < geo.nchunks; ++k) {
+        const int cur = k & 1;
+        if (k + 1 < geo.nchunks) {
+            issue(k + 1, cur ^ 1);
+            asm volatile("cp.async.wait_group 1;\n" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+        }
+        __syncthreads();
+        const float* xs = xs0 + cur * xs_floats;
+        const uint4* ws = ws0 + cur * C::WS_U4;
+#pragma unroll
+        for (int q = 0; q < GPW; ++q) {
+            const int2 hd = reinterpret_cast<const int2*>(ws)[gw * GPW + q];
+            const uint4* r = ws + hd.x;
+            for (int it = 0; it < hd.y; ++it, r += C::UNIT) {
+                const float* plane = xs + r[0].x;
+                const float* wq = reinterpret_cast<const float*>(r + 1);   // [9][G]
+#pragma unroll
+                for (int kh = 0; kh < 3; ++kh) {
+                    const float* arow = plane + rowoff[kh];
+                    f32x2 a[CW + 2];
+#pragma unroll
+                    for (int i = 0; i < CW + 2; ++i) a[i] = dup2(arow[i]);
+#pragma unroll
+                    for (int kw = 0; kw < 3; ++kw) {
+                        f32x2 w[GP];
+                        if constexpr (G % 4 == 0) {
+#pragma unroll
+                            for (int v = 0; v < G / 4; ++v) {
+                                const ulonglong2 t = reinterpret_cast<const ulonglong2*>(wq + (kh * 3 + kw) * G)[v];
+                                w[2 * v] = t.x;
+                                w[2 * v + 1] = t.y;
+                            }
+                        } else if constexpr (G == 2) {
+                            w[0] = *reinterpret_cast<const unsigned long long*>(wq + (kh * 3 + kw) * 2);
+                        } else {
+                            w[0] = pack2(wq[kh * 3 + kw], 0.0f);
+                        }
+#pragma unroll
+                        for (int p = 0; p < CW; ++p)
+#pragma unroll
+                            for (int rr = 0; rr < GP; ++rr) fma2(acc[q][p][rr], a[p + kw], w[rr]);
+                    }
+                }
+            }
+        }
+        __syncthreads();        // everyone is done with this buffer before the copies of step k+2 are issued
+    }
+
+    if (f >= NH) return;
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * C::GT + gw * GPW + q;
+        if (g >= geo.ngroups) continue;
+#pragma unroll
+        for (int p = 0; p < CW; ++p) {
+            const int x = lx + p;
+            if (x >= W) continue;
+            float* yp = Y + ((size_t)f * W + x) * geo.Cout + g * G;
+            float v[2 * GP];
+#pragma unroll
+            for (int rr = 0; rr < GP; ++rr) unpack2(acc[q][p][rr], v[2 * rr], v[2 * rr + 1]);
+            if (relu) {
+#pragma unroll
+                for (int rr = 0; rr < 2 * GP; ++rr) v[rr] = fmaxf(v[rr], 0.0f);
+            }
+            if constexpr (G >= 4) {
+#pragma unroll
+                for (int vv = 0; vv < G / 4; ++vv)
+                    reinterpret_cast<float4*>(yp)[vv] = make_float4(v[4 * vv], v[4 * vv + 1], v[4 * vv + 2], v[4 * vv + 3]);
+            } else if constexpr (G == 2) {
+                *reinterpret_cast<float2*>(yp) = make_float2(v[0], v[1]);
+            } else {
+                yp[0] = v[0];
+            }
+        }
+    }
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 int pow2_ceil(int v) {
@@ -309,6 +481,76 @@ sbnn_status launch3(const sbnn_packed* p, const float* x, float* y, int N, int H
     return SBNN_OK;
 }
 
+// Pitch for the channel-major variant: a multiple of 4 (16-byte aligned row pieces), >= LPR*CW + 5, and such
+// that the first reads of the 32 lanes fall into 32 distinct banks if possible.
+int pick_pitch4(int LPR, int CW) {
+    const int lo = (LPR * CW + 5 + 3) / 4 * 4;
+    for (int p = lo; p < lo + 128; p += 4) {
+        unsigned used = 0;
+        bool ok = true;
+        for (int l = 0; l < 32 && ok; ++l) {
+            const int b = ((l / LPR) * p + (l % LPR) * CW) & 31;
+            ok = !((used >> b) & 1u);
+            used |= 1u << b;
+        }
+        if (ok) return p;
+    }
+    return lo;
+}
+
+// Launches the channel-major variant; *done = false (and SBNN_OK) if the shape does not fit it.
+template <class C>
+sbnn_status launch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
+                       cudaStream_t st, bool* done) {
+    *done = false;
+    Geo3 g;
+    g.N = N; g.H = H; g.W = W; g.Cin = p->Cin; g.Cout = p->Cout; g.ngroups = p->ngroups;
+    g.LPR = lanes_per_row(W, C::CW);
+    g.RPW = 32 / g.LPR;
+    g.R = C::NPW * g.RPW;
+    g.pitch = pick_pitch4(g.LPR, C::CW);
+    const int plane = ((g.R + 3) * g.pitch + 7) / 8 * 8 + 4;   // multiple of 4 floats
+    g.plane = plane;
+    g.nchunks = (p->Cin + C::KC - 1) / C::KC;
+    g.dpp_row = g.dpp_x = 0;
+    const size_t smem = (size_t)2 * C::KC * plane * 4 + (size_t)2 * C::WS_U4 * 16;
+    const long long pieces = (long long)(g.R + 2) * (W / 4);
+    if (smem > 227 * 1024 || pieces > 2LL * C::NT || (long long)N * H * W * 1 > 0x7fffffffLL / 2) return SBNN_OK;
+    Stream3x3 s;
+    {
+        std::lock_guard<std::mutex> lk(p->mu);
+        const int key = (plane << 8) | (C::GT << 4) | (C::KC / 4);
+        auto it = p->streams3x3.find(key);
+        if (it == p->streams3x3.end()) {
+            sbnn_status r = build_stream3(p, C::GT, C::KC, plane, &s);
+            if (r != SBNN_OK) return r;
+            p->streams3x3[key] = s;
+        } else {
+            s = it->second;
+        }
+    }
+    if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
+    SBNN_CUDA_TRY(cudaFuncSetAttribute(conv3x3_gs_cm_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const long long NH = (long long)N * H;
+    dim3 grid((unsigned)((NH + g.R - 1) / g.R), s.ntiles);
+    conv3x3_gs_cm_kernel<C><<<grid, C::NT, smem, st>>>(xt, ldx, y, p->d_bias, s.rec, s.blk_ptr, g, relu);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    *done = true;
+    return SBNN_OK;
+}
+
+template <int CW>
+sbnn_status dispatch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
+                         cudaStream_t st, bool* done) {
+    switch (p->G) {
+        case 1: return launch3_cm<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        case 2: return launch3_cm<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        case 4: return launch3_cm<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        case 8: return launch3_cm<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        default: return launch3_cm<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+    }
+}
+
 // Column width per lane: the one that tiles the row with least waste (ties go to 8).
 int choose_cw(int W) {
     const int l7 = lanes_per_row(W, 7), l8 = lanes_per_row(W, 8);
@@ -361,6 +603,17 @@ extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev,
     sbnn_status st = check_device();
     if (st != SBNN_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (W % 4 == 0) {
+        // fast path: planes of the input ([Cin][ld]) in the per-device scratch buffer, then the cp.async kernel
+        const int M = N * H * W, ld = (M + 3) / 4 * 4;
+        float* xt = nullptr;
+        if ((st = scratch_workspace((size_t)w->Cin * ld * sizeof(float), &xt)) != SBNN_OK) return st;
+        if ((st = launch_transpose(x_dev, w->Cin, xt, ld, M, w->Cin, s)) != SBNN_OK) return st;
+        bool done = false;
+        st = cw == 7 ? dispatch3_cm<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
+                     : dispatch3_cm<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);
+        if (st != SBNN_OK || done) return st;
+    }
     return cw == 7 ? dispatch3<7>(w, x_dev, y_dev, N, H, W, flags & SBNN_RELU, s)
                    : dispatch3<8>(w, x_dev, y_dev, N, H, W, flags & SBNN_RELU, s);
 }
