@@ -194,6 +194,22 @@ def time_layers(sbnn, torch, net, layers, batch, reps, flush):
     return res
 
 
+def max_over_ranks(values, world, device="cpu"):
+    """Element-wise maximum of per-rank timings over the process group (the job is as slow as its slowest replica)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(per_rank_units, steps, world, seconds):
+    """Whole-job rate of batch-sharded replicas: every rank processes per_rank_units per step, no exchange."""
+    return per_rank_units * world * steps / seconds
+
+
 def run_gpu(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -250,10 +266,7 @@ def run_gpu(args, rank, world, local_rank):
     e2e_elapsed = ev0.elapsed_time(ev1) * 1e-3
     clocks = sampler.stop() if rank == 0 else None
 
-    if world > 1:
-        t = torch.tensor([elapsed, e2e_elapsed], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed, e2e_elapsed = float(t[0]), float(t[1])
+    elapsed, e2e_elapsed = max_over_ranks([elapsed, e2e_elapsed], world, "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -287,6 +300,7 @@ def run_gpu(args, rank, world, local_rank):
 
     cpu = cpu_baseline(x, layers) if world == 1 and not args.no_cpu else None
     imgs = batch * world * args.steps
+    assert abs(job_throughput(batch, args.steps, world, elapsed) - imgs / elapsed) < 1e-6 * imgs / elapsed
     line = {
         "metric": METRIC, "value": imgs / elapsed, "unit": "images/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": elapsed / args.steps * 1e3, "higher_is_better": True,
