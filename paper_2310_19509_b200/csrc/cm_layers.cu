@@ -131,6 +131,59 @@ dwconv3x3_cm_px_kernel(const float* __restrict__ w, const float* __restrict__ b,
     }
 }
 
+// Row-strip kernel for the 14- and 7-wide outputs (Wo a multiple of 7): a thread owns 7 consecutive
+// outputs of one row of one channel in up to NI consecutive images and slides a 3 x (6S+3) register
+// window over them, so an input value is loaded once per thread instead of once per tap.
+template <int S, int NI, int WT>
+__global__ void __launch_bounds__(128)
+dwconv3x3_cm_strip7_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
+                           float* __restrict__ y, int ldy, int N, int H, int relu) {
+    constexpr int W = WT, Wo = WT / S, SPR = Wo / 7, IW = 6 * S + 3;
+    const int Ho = H / S;
+    const int c = blockIdx.y, C = gridDim.y;
+    const int items = Ho * SPR;                                      // (row, strip) items of a plane
+    const int QB = (items + blockDim.x - 1) / blockDim.x;
+    const int q = (blockIdx.x % QB) * blockDim.x + threadIdx.x;
+    const int n0 = (blockIdx.x / QB) * NI;
+    if (q >= items) return;
+    const int oy = q / SPR, ox0 = (q - oy * SPR) * 7;
+    float wk[9];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);
+    const float bias = b ? __ldg(b + c) : 0.0f;
+    bool rok[3];
+#pragma unroll
+    for (int kh = 0; kh < 3; ++kh) rok[kh] = (oy * S + kh - 1 >= 0) && (oy * S + kh - 1 < H);
+    const bool lok = ox0 > 0, rokx = (ox0 * S + IW - 2) < W;        // first / last window column inside the row
+    const float* pc = x + (size_t)c * ldx + (size_t)n0 * H * W + (oy * S - 1) * W + ox0 * S - 1;   // window origin
+    float* yc = y + (size_t)c * ldy + (size_t)n0 * Ho * Wo + oy * Wo + ox0;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        if (n0 + i >= N) break;
+        float acc[7];
+#pragma unroll
+        for (int o = 0; o < 7; ++o) acc[o] = bias;
+#pragma unroll
+        for (int kh = 0; kh < 3; ++kh) {
+            if (!rok[kh]) continue;
+            float in[IW];
+#pragma unroll
+            for (int j = 0; j < IW; ++j) {
+                const bool ok = (j > 0 || lok) && (j < IW - 1 || rokx);
+                in[j] = ok ? __ldg(pc + kh * W + j) : 0.0f;
+            }
+#pragma unroll
+            for (int o = 0; o < 7; ++o)
+#pragma unroll
+                for (int kw = 0; kw < 3; ++kw) acc[o] = fmaf(in[o * S + kw], wk[kh * 3 + kw], acc[o]);
+        }
+#pragma unroll
+        for (int o = 0; o < 7; ++o) yc[o] = relu ? fmaxf(acc[o], 0.0f) : acc[o];
+        pc += H * W;
+        yc += Ho * Wo;
+    }
+}
+
 // ---- first layer: NHWC image with Cin <= 4 in, channel-major out --------------------------------
 // One thread: 4 consecutive output columns of one row x 8 output channels; consecutive lanes take
 // consecutive column strips, so each channel's stores are contiguous across the warp.
@@ -330,15 +383,22 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
         const int QB = (Ho * Wo + 255) / 256;
         dim3 grid((unsigned)(QB * ((N + NI - 1) / NI)), C);
 #define SBNN_DW_PX(S_, WT_) dwconv3x3_cm_px_kernel<S_, NI, WT_><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, QB, relu)
+#define SBNN_DW_S7(S_, WT_)                                                                                   \
+    {                                                                                                         \
+        const int items = Ho * (Wo / 7), qb = (items + 127) / 128;                                            \
+        dim3 g7((unsigned)(qb * ((N + NI - 1) / NI)), C);                                                     \
+        dwconv3x3_cm_strip7_kernel<S_, NI, WT_><<<g7, 128, 0, st>>>(w, b, x, ldx, y, ldy, N, H, relu);         \
+    }
         if (stride == 1) {
-            if (W == 14) SBNN_DW_PX(1, 14);
-            else if (W == 7) SBNN_DW_PX(1, 7);
+            if (W == 14) SBNN_DW_S7(1, 14)
+            else if (W == 7) SBNN_DW_S7(1, 7)
             else SBNN_DW_PX(1, 0);
         } else {
-            if (W == 28) SBNN_DW_PX(2, 28);
+            if (W == 28) SBNN_DW_PX(2, 28);      // stride 2: the per-position kernel measured faster
             else if (W == 14) SBNN_DW_PX(2, 14);
             else SBNN_DW_PX(2, 0);
         }
+#undef SBNN_DW_S7
 #undef SBNN_DW_PX
     }
     SBNN_CUDA_TRY(cudaGetLastError());
