@@ -151,6 +151,8 @@ SBNN_API sbnn_status sbnn_conv1x1_gs_tuned(const sbnn_packed* w, const float* x_
  * into a channel-major scratch buffer kept per device, which it allocates or grows (synchronously) the
  * first time a size is seen.
  * sbnn_to_channel_major converts x_dev [M][C] to xt_dev [C][ld].
+ * The scratch buffer is one per device and is also used by the bf16 mode and by sbnn_conv3x3_gs: calls that
+ * use it must be ordered on the GPU (same stream, or events); overlapping ones race on it.
  */
 SBNN_API sbnn_status sbnn_conv1x1_gs_cm(const sbnn_packed* w, const float* xt_dev, int ldx, float* y_dev, int ldy,
                                         int M, int flags, int P, int GPW, int NW, int KC, void* cuda_stream);

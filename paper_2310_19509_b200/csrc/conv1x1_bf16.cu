@@ -15,9 +15,10 @@
 // G = 4 uses half, G = 16 takes two MMAs per A fragment).
 //
 // CTA = 128 pixels x 8 warps; a warp owns GPW groups over all 128 pixels (8 row blocks of 16), i.e.
-// 32 fp32 accumulators per N-tile.  Each channel step the CTA converts its X tile to bf16 and stores
-// it transposed; the weight stream holds, per 16 kept channels, 16 row offsets and the B fragments in
-// register order.
+// 32 fp32 accumulators per N-tile.  A pre-pass converts X once to bf16 in channel-major order
+// ([Cin][ld], pixels contiguous); the kernel then fills its [channel][pixel] tile with 16-byte
+// cp.async pieces into two buffers, so the copies of step k+1 run under the MMAs of step k.  The
+// weight stream holds, per 16 kept channels, 16 row offsets and the B fragments in register order.
 #include <cuda_bf16.h>
 #include <string.h>
 
@@ -58,14 +59,14 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
 
 template <int G, int GPW>
 __global__ void __launch_bounds__(NWARP * 32)
-conv1x1_bf16_kernel(const float* __restrict__ X, float* __restrict__ Y, const float* __restrict__ bias,
+conv1x1_bf16_kernel(const __nv_bfloat16* __restrict__ Xb, int ldb, float* __restrict__ Y, const float* __restrict__ bias,
                     const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout,
                     int ngroups, int nchunks, int ntiles, int ws_u4, int relu) {
     constexpr int NT8 = (G + 7) / 8;
     constexpr int GT = NWARP * GPW;
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* xs = smem;                                          // [KC][ROWB]
-    uint4* ws = reinterpret_cast<uint4*>(smem + KC * ROWB);            // weight block of the step
+    unsigned char* xs0 = smem;                                         // two buffers of [KC][ROWB]
+    uint4* ws0 = reinterpret_cast<uint4*>(smem + 2 * KC * ROWB);       // two weight blocks of ws_u4 units
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile = blockIdx.x % ntiles;
     const int m0 = (blockIdx.x / ntiles) * TM;
@@ -89,26 +90,36 @@ conv1x1_bf16_kernel(const float* __restrict__ X, float* __restrict__ Y, const fl
     }
     // ldmatrix: lane l addresses row (l & 7) of sub-matrix (l >> 3): channels 8*(l>>4) + (l&7), pixels 8*((l>>3)&1)..
     const int off_idx = 8 * (lane >> 4) + (lane & 7);
-    const uint32_t xs_lane = static_cast<uint32_t>(__cvta_generic_to_shared(xs)) + ((lane >> 3) & 1) * 16;
+    const uint32_t xs_base = static_cast<uint32_t>(__cvta_generic_to_shared(xs0)) + ((lane >> 3) & 1) * 16;
 
+    auto cp16 = [](void* dst, const void* src) {
+        const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(dst));
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(src) : "memory");
+    };
+    auto issue = [&](int k, int buf) {   // rows of 128 pixels = 16 pieces of 16 bytes; then the weight block
+        unsigned char* xd = xs0 + buf * (KC * ROWB);
+        for (int i = tid; i < KC * 16; i += NWARP * 32) {
+            const int c = i >> 4, pc = i & 15;
+            if (k * KC + c < Cin) cp16(xd + c * ROWB + pc * 16, Xb + (size_t)(k * KC + c) * ldb + m0 + pc * 8);
+        }
+        uint4* wd = ws0 + buf * ws_u4;
+        const int beg = bp[k], n = bp[k + 1] - beg;
+        for (int i = tid; i < n; i += NWARP * 32) cp16(wd + i, rec + beg + i);
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+    };
+
+    issue(0, 0);
     for (int k = 0; k < nchunks; ++k) {
-        __syncthreads();
-        {   // stage: X tile -> bf16, transposed; weight block
-            const int beg = bp[k], n = bp[k + 1] - beg;
-            for (int i = tid; i < n; i += NWARP * 32) ws[i] = rec[beg + i];
-            for (int e = tid; e < TM * (KC / 4); e += NWARP * 32) {
-                const int cq = e % (KC / 4), p = e / (KC / 4);
-                const int m = m0 + p, c = k * KC + cq * 4;
-                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (m < M && c < Cin) v = __ldg(reinterpret_cast<const float4*>(X + (size_t)m * Cin + c));
-                __nv_bfloat16* d = reinterpret_cast<__nv_bfloat16*>(xs + (size_t)(cq * 4) * ROWB) + p;
-                d[0] = __float2bfloat16_rn(v.x);
-                d[ROWB / 2] = __float2bfloat16_rn(v.y);
-                d[ROWB] = __float2bfloat16_rn(v.z);
-                d[3 * (ROWB / 2)] = __float2bfloat16_rn(v.w);
-            }
+        const int cur = k & 1;
+        if (k + 1 < nchunks) {
+            issue(k + 1, cur ^ 1);
+            asm volatile("cp.async.wait_group 1;\n" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;\n" ::: "memory");
         }
         __syncthreads();
+        const uint4* ws = ws0 + cur * ws_u4;
+        const uint32_t xs_lane = xs_base + cur * (KC * ROWB);
 #pragma unroll
         for (int q = 0; q < GPW; ++q) {
             const int2 hd = reinterpret_cast<const int2*>(ws)[warp * GPW + q];   // (start, 16-channel blocks)
@@ -130,6 +141,7 @@ conv1x1_bf16_kernel(const float* __restrict__ X, float* __restrict__ Y, const fl
                 }
             }
         }
+        __syncthreads();   // done with this buffer before the copies of step k+2 are issued
     }
 #pragma unroll
     for (int q = 0; q < GPW; ++q) {
@@ -155,6 +167,25 @@ conv1x1_bf16_kernel(const float* __restrict__ X, float* __restrict__ Y, const fl
     }
 }
 
+// X [M][C] fp32 (row-major) -> Xb [C][ldb] bf16, round to nearest even; 32 x 32 tiles through shared memory.
+__global__ void __launch_bounds__(256)
+to_channel_major_bf16_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ xb, int M, int C, int ldb) {
+    __shared__ float t[32][33];
+    const int m0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty + 8 * i, c = c0 + tx;
+        t[ty + 8 * i][tx] = (m < M && c < C) ? x[(size_t)m * C + c] : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = c0 + ty + 8 * i, m = m0 + tx;
+        if (m < ldb && c < C) xb[(size_t)c * ldb + m] = __float2bfloat16_rn(t[tx][ty + 8 * i]);
+    }
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 // fp32 -> bf16 bits, round to nearest even (bf16 is the upper half of an IEEE-754 binary32).
@@ -170,7 +201,7 @@ uint16_t bf16_bits(float f) {
 // 16 byte offsets of the channels' shared-memory rows, then per N-tile the B fragment of m16n8k16 in
 // register order (lane l: {B[2t][g], B[2t+1][g]}, {B[2t+8][g], B[2t+9][g]}, g = l/4, t = l%4).
 sbnn_status build_stream_bf16(const sbnn_packed* p, StreamBf16* out) {
-    const int G = p->G, NT8 = (G + 7) / 8, GT = NWARP, BLK = 4 + NT8 * 16;
+    const int G = p->G, NT8 = (G + 7) / 8, GT = NWARP * (G <= 8 ? 2 : 1), BLK = 4 + NT8 * 16;
     const int ntiles = (p->ngroups + GT - 1) / GT, nchunks = (p->Cin + KC - 1) / KC;
     const int HDR = (GT * 2 + 3) / 4;
     std::vector<int32_t> blk((size_t)ntiles * (nchunks + 1));
@@ -192,19 +223,44 @@ sbnn_status build_stream_bf16(const sbnn_packed* p, StreamBf16* out) {
                         hi = (int)(std::lower_bound(b, e, (k + 1) * KC) - p->idx.data());
                     }
                     const int nb = (hi - lo + 15) / 16;
+                    // Order of the kept channels inside the step: each ldmatrix sub-matrix reads 8 rows at
+                    // once, and rows whose channel indices are equal mod 8 fall into the same banks (a row
+                    // is 17 x 16 bytes).  So deal the channels out in rounds of 8 with distinct residues,
+                    // taking from the fullest residue classes first.  (The sum does not depend on the order
+                    // beyond rounding.)
+                    std::vector<int> order;
+                    {
+                        std::vector<int> bucket[8];
+                        for (int j = hi - 1; j >= lo; --j) bucket[p->idx[j] & 7].push_back(j);
+                        int left = hi - lo;
+                        while (left > 0) {
+                            int cls[8] = {0, 1, 2, 3, 4, 5, 6, 7};
+                            std::sort(cls, cls + 8, [&](int a, int b) { return bucket[a].size() > bucket[b].size(); });
+                            for (int i = 0; i < 8 && left > 0; ++i) {
+                                if (bucket[cls[i]].empty()) continue;
+                                order.push_back(bucket[cls[i]].back());
+                                bucket[cls[i]].pop_back();
+                                --left;
+                            }
+                        }
+                    }
                     rec[blk_beg * 4 + 2 * s + 0] = (uint32_t)(rec.size() / 4 - blk_beg);
                     rec[blk_beg * 4 + 2 * s + 1] = (uint32_t)nb;
                     for (int b16 = 0; b16 < nb; ++b16) {
                         const size_t base = rec.size();
                         rec.resize(base + (size_t)BLK * 4, 0u);   // padding: row 0, zero weights
+                        auto unit = [&](int kk) -> int {
+                            const size_t i = (size_t)b16 * 16 + kk;
+                            return i < order.size() ? order[i] : -1;
+                        };
                         auto wbits = [&](int kk, int col) -> uint32_t {
-                            const int j = lo + b16 * 16 + kk;
-                            if (j >= hi || col >= G) return 0u;
+                            const int j = unit(kk);
+                            if (j < 0 || col >= G) return 0u;
                             return bf16_bits(p->val[(size_t)j * G + col]);
                         };
                         for (int kk = 0; kk < 16; ++kk) {
-                            const int j = lo + b16 * 16 + kk;
-                            if (j < hi) rec[base + kk] = (uint32_t)(p->idx[j] - k * KC) * (uint32_t)ROWB;
+                            const int j = unit(kk);
+                            if (j >= 0) rec[base + kk] = (uint32_t)(p->idx[j] - k * KC) * (uint32_t)ROWB;
                         }
                         for (int n = 0; n < NT8; ++n)
                             for (int l = 0; l < 32; ++l) {
@@ -239,12 +295,24 @@ sbnn_status build_stream_bf16(const sbnn_packed* p, StreamBf16* out) {
 
 template <int G>
 sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, const float* x, float* y, int M, int relu, cudaStream_t st) {
-    const size_t smem = (size_t)KC * ROWB + (size_t)s.max_blk * 16;
-    if (smem > 48 * 1024) return fail(SBNN_ERR_UNSUPPORTED, "internal: bf16 tile needs %zu bytes of shared memory", smem);
-    const long long nblk = (long long)((M + TM - 1) / TM) * s.ntiles;
+    constexpr int GPW = (G <= 8) ? 2 : 1;
+    // bf16 channel-major copy of X in the per-device scratch buffer; rows padded to whole pixel tiles
+    const int ldb = (M + TM - 1) / TM * TM;
+    float* scratch = nullptr;
+    sbnn_status r = scratch_workspace((size_t)p->Cin * ldb * sizeof(__nv_bfloat16), &scratch);
+    if (r != SBNN_OK) return r;
+    __nv_bfloat16* xb = reinterpret_cast<__nv_bfloat16*>(scratch);
+    dim3 tg((ldb + 31) / 32, (p->Cin + 31) / 32);
+    to_channel_major_bf16_kernel<<<tg, 256, 0, st>>>(x, xb, M, p->Cin, ldb);
+    SBNN_CUDA_TRY(cudaGetLastError());
+
+    const size_t smem = (size_t)2 * KC * ROWB + (size_t)2 * s.max_blk * 16;
+    if (smem > 200 * 1024) return fail(SBNN_ERR_UNSUPPORTED, "internal: bf16 tile needs %zu bytes of shared memory", smem);
+    SBNN_CUDA_TRY(cudaFuncSetAttribute(conv1x1_bf16_kernel<G, GPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const long long nblk = (long long)(ldb / TM) * s.ntiles;
     if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
-    conv1x1_bf16_kernel<G, 1><<<(unsigned)nblk, NWARP * 32, smem, st>>>(x, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
-                                                                        p->ngroups, s.nchunks, s.ntiles, s.max_blk, relu);
+    conv1x1_bf16_kernel<G, GPW><<<(unsigned)nblk, NWARP * 32, smem, st>>>(xb, ldb, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin,
+                                                                          p->Cout, p->ngroups, s.nchunks, s.ntiles, s.max_blk, relu);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
 }
