@@ -283,6 +283,14 @@ SBNN_API sbnn_status sbnn_head_noalloc(const sbnn_packed* fc, const float* x_dev
  */
 SBNN_API sbnn_status sbnn_get_async_status(void* cuda_stream);
 
+/*
+ * Diagnostic for the bounded waits of the pipelined kernels: enqueues a one-warp kernel that waits, with a
+ * cap of 2000 polls, on a barrier nothing completes.  The kernel gives up, records SBNN_ERR_TIMEOUT in the
+ * device status word and returns normally; the next sbnn_get_async_status on the stream reports
+ * SBNN_ERR_TIMEOUT once (the word is cleared by that call) and the context stays usable.
+ */
+SBNN_API sbnn_status sbnn_selftest_wait_timeout(void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,6 +25,7 @@ from .binding import (  # noqa: F401
     lib_path,
     mobilenet_v1_layer_shape,
     pack_weights,
+    selftest_wait_timeout,
     status_str,
     to_channel_major,
 )

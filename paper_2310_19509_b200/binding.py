@@ -59,6 +59,7 @@ def lib():
         "sbnn_mobilenet_v1_free": [P],
         "sbnn_get_async_status": [P],
         "sbnn_head_noalloc": [P, P, P, I, I, P],
+        "sbnn_selftest_wait_timeout": [P],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -193,6 +194,11 @@ def avgpool(x, y, n, hw, c, stream=None):
 def head_noalloc(fc: Packed, x, logits, n, hw, stream=None):
     """Average pool + classifier through the library's fixed scratch array; allocates nothing."""
     _check(lib().sbnn_head_noalloc(fc.handle, _ptr(x), _ptr(logits), n, hw, _stream(stream)))
+
+
+def selftest_wait_timeout(stream=None):
+    """Enqueue the diagnostic kernel whose bounded wait expires (see sbnn_selftest_wait_timeout)."""
+    _check(lib().sbnn_selftest_wait_timeout(_stream(stream)))
 
 
 def get_async_status(stream=None):

@@ -284,6 +284,20 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
     }   // tiles
 }
 
+// Diagnostic: one warp waits, with a short cap, on an mbarrier that nothing ever completes.  Exercises the
+// path a stalled pipeline takes (status word set, kernel returns normally) without any fault.
+__global__ void wait_timeout_selftest_kernel(int* status, uint32_t limit) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    mbar_wait(&bar, 0, &abort_flag, status, SBNN_ERR_TIMEOUT, limit);
+}
+
 // X [M][C] (row-major, C contiguous) -> Xt [C][ld]: 32 x 32 tiles through padded shared memory.
 __global__ void __launch_bounds__(256)
 to_channel_major_kernel(const float* __restrict__ x, float* __restrict__ xt, int M, int C, int ld) {
@@ -593,6 +607,17 @@ sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M
 }  // namespace sbnn
 
 using namespace sbnn;
+
+extern "C" sbnn_status sbnn_selftest_wait_timeout(void* cuda_stream) {
+    clear_error();
+    sbnn_status st = check_device();
+    if (st != SBNN_OK) return st;
+    int* status = nullptr;
+    if ((st = status_word(&status)) != SBNN_OK) return st;
+    wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(status, 2000u);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    return SBNN_OK;
+}
 
 extern "C" sbnn_status sbnn_to_channel_major(const float* x_dev, float* xt_dev, int M, int C, int ld, void* cuda_stream) {
     clear_error();

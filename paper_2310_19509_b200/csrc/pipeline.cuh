@@ -60,8 +60,9 @@ constexpr uint32_t kWaitLimit = 1u << 22;
 
 // Waits for the phase with the given parity.  Returns false, after recording `code` in *status,
 // when the cap is reached or another thread of the CTA has already given up (*abort != 0).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int* status, int code) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int* status, int code,
+                                          uint32_t limit = kWaitLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 64) {
             if (*abort) return false;

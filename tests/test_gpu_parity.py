@@ -331,3 +331,17 @@ def test_mobilenet_layer_on_channel_major_buffers():
         y = yd.cpu().numpy().T.reshape(rec["ref"].shape)
         assert_within(y, rec["ref"], rec["S"], what=f"cm layer {li}")
     net.free()
+
+
+def test_expired_wait_is_reported_and_the_context_stays_usable():
+    """A bounded device-side wait that runs out sets the status word; nothing faults, later calls work."""
+    sbnn.get_async_status()                                   # clean slate
+    sbnn.selftest_wait_timeout()
+    with pytest.raises(sbnn.SbnnError) as e:
+        sbnn.get_async_status()
+    assert e.value.name == "SBNN_ERR_TIMEOUT"
+    sbnn.get_async_status()                                   # reported once, then clear
+    d = WL.single_conv_inputs(1, 4, 4, 16, 16, 1, 4, 50, seed=3)
+    y = run_1x1(d)
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    assert_within(y, ref, s, what="after an expired wait")
