@@ -92,14 +92,17 @@ dwconv3x3_cm_vec_kernel(const float* __restrict__ w, const float* __restrict__ b
 template <int S, int NI, int WT>
 __global__ void __launch_bounds__(256)
 dwconv3x3_cm_px_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
-                       float* __restrict__ y, int ldy, int N, int H, int Wrt, int QB, int relu) {
+                       float* __restrict__ y, int ldy, int N, int H, int Wrt, int C, int QB, int relu) {
     const int W = WT ? WT : Wrt;
     const int Ho = H / S, Wo = W / S;
-    const int c = blockIdx.y, C = gridDim.y;
-    const int q = (blockIdx.x % QB) * blockDim.x + threadIdx.x;     // position inside an output plane
-    const int n0 = (blockIdx.x / QB) * NI;                           // first image of this thread
     const int HoWo = Ho * Wo, HW = H * W;
-    if (q >= HoWo) return;
+    // small planes: a CTA takes CPB channels (CPB * HoWo <= blockDim.x), so its lanes are not left idle
+    const int CPB = HoWo < (int)blockDim.x ? (int)blockDim.x / HoWo : 1;
+    const int cl = CPB > 1 ? (int)threadIdx.x / HoWo : 0;
+    const int c = blockIdx.y * CPB + cl;
+    const int q = CPB > 1 ? (int)threadIdx.x - cl * HoWo : (blockIdx.x % QB) * (int)blockDim.x + (int)threadIdx.x;
+    const int n0 = (blockIdx.x / QB) * NI;                           // first image of this thread
+    if (q >= HoWo || cl >= CPB || c >= C) return;
     const int oy = q / Wo, ox = q - oy * Wo;
     float wk[9];
     bool ok[9];
@@ -131,32 +134,32 @@ dwconv3x3_cm_px_kernel(const float* __restrict__ w, const float* __restrict__ b,
     }
 }
 
-// Row-strip kernel for the 14- and 7-wide outputs (Wo a multiple of 7): a thread owns 7 consecutive
-// outputs of one row of one channel in up to NI consecutive images and slides a 3 x (6S+3) register
-// window over them, so an input value is loaded once per thread instead of once per tap.
-template <int S, int NI, int WT>
+// Column-strip kernel for the stride-1 14- and 7-wide maps (H a multiple of 7): a thread owns 7 consecutive
+// output rows of one column of one channel in up to NI consecutive images and slides a 9 x 3 register
+// window down the column, so an input value is loaded once per thread instead of once per tap.  Consecutive
+// lanes own consecutive columns, so every load and store of a warp covers contiguous runs of a row.
+template <int NI, int WT>
 __global__ void __launch_bounds__(128)
-dwconv3x3_cm_strip7_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
-                           float* __restrict__ y, int ldy, int N, int H, int relu) {
-    constexpr int W = WT, Wo = WT / S, SPR = Wo / 7, IW = 6 * S + 3;
-    const int Ho = H / S;
-    const int c = blockIdx.y, C = gridDim.y;
-    const int items = Ho * SPR;                                      // (row, strip) items of a plane
+dwconv3x3_cm_col7_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
+                         float* __restrict__ y, int ldy, int N, int H, int C, int relu) {
+    constexpr int W = WT;
+    const int items = (H / 7) * W;                                   // (vertical strip, column) items of a plane
     const int QB = (items + blockDim.x - 1) / blockDim.x;
-    const int q = (blockIdx.x % QB) * blockDim.x + threadIdx.x;
+    // small planes: a CTA takes CPB channels (CPB * items <= blockDim.x), so its lanes are not left idle
+    const int CPB = items < (int)blockDim.x ? (int)blockDim.x / items : 1;
+    const int cl = CPB > 1 ? (int)threadIdx.x / items : 0;
+    const int c = blockIdx.y * CPB + cl;
+    const int q = CPB > 1 ? (int)threadIdx.x - cl * items : (blockIdx.x % QB) * (int)blockDim.x + (int)threadIdx.x;
     const int n0 = (blockIdx.x / QB) * NI;
-    if (q >= items) return;
-    const int oy = q / SPR, ox0 = (q - oy * SPR) * 7;
+    if (q >= items || cl >= CPB || c >= C) return;
+    const int vs = q / W, ox = q - vs * W, oy0 = vs * 7;
     float wk[9];
 #pragma unroll
     for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);
     const float bias = b ? __ldg(b + c) : 0.0f;
-    bool rok[3];
-#pragma unroll
-    for (int kh = 0; kh < 3; ++kh) rok[kh] = (oy * S + kh - 1 >= 0) && (oy * S + kh - 1 < H);
-    const bool lok = ox0 > 0, rokx = (ox0 * S + IW - 2) < W;        // first / last window column inside the row
-    const float* pc = x + (size_t)c * ldx + (size_t)n0 * H * W + (oy * S - 1) * W + ox0 * S - 1;   // window origin
-    float* yc = y + (size_t)c * ldy + (size_t)n0 * Ho * Wo + oy * Wo + ox0;
+    const bool lok = ox > 0, rok = ox + 1 < W, top = oy0 > 0, bot = oy0 + 7 < H;
+    const float* pc = x + (size_t)c * ldx + (size_t)n0 * H * W + (oy0 - 1) * W + ox;   // window origin (centre column)
+    float* yc = y + (size_t)c * ldy + (size_t)n0 * H * W + oy0 * W + ox;
 #pragma unroll
     for (int i = 0; i < NI; ++i) {
         if (n0 + i >= N) break;
@@ -164,23 +167,22 @@ dwconv3x3_cm_strip7_kernel(const float* __restrict__ w, const float* __restrict_
 #pragma unroll
         for (int o = 0; o < 7; ++o) acc[o] = bias;
 #pragma unroll
-        for (int kh = 0; kh < 3; ++kh) {
-            if (!rok[kh]) continue;
-            float in[IW];
+        for (int r = 0; r < 9; ++r) {                                // input rows oy0-1 .. oy0+7
+            const bool rowok = (r > 0 || top) && (r < 8 || bot);
+            const float l = (rowok && lok) ? __ldg(pc + r * W - 1) : 0.0f;
+            const float m = rowok ? __ldg(pc + r * W) : 0.0f;
+            const float rr = (rowok && rok) ? __ldg(pc + r * W + 1) : 0.0f;
 #pragma unroll
-            for (int j = 0; j < IW; ++j) {
-                const bool ok = (j > 0 || lok) && (j < IW - 1 || rokx);
-                in[j] = ok ? __ldg(pc + kh * W + j) : 0.0f;
+            for (int kh = 0; kh < 3; ++kh) {
+                const int o = r - kh;                                // output row fed by this input row through tap row kh
+                if (o >= 0 && o < 7)
+                    acc[o] = fmaf(rr, wk[kh * 3 + 2], fmaf(m, wk[kh * 3 + 1], fmaf(l, wk[kh * 3], acc[o])));
             }
-#pragma unroll
-            for (int o = 0; o < 7; ++o)
-#pragma unroll
-                for (int kw = 0; kw < 3; ++kw) acc[o] = fmaf(in[o * S + kw], wk[kh * 3 + kw], acc[o]);
         }
 #pragma unroll
-        for (int o = 0; o < 7; ++o) yc[o] = relu ? fmaxf(acc[o], 0.0f) : acc[o];
+        for (int o = 0; o < 7; ++o) yc[o * W] = relu ? fmaxf(acc[o], 0.0f) : acc[o];
         pc += H * W;
-        yc += Ho * Wo;
+        yc += H * W;
     }
 }
 
@@ -381,24 +383,26 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
     } else {
         constexpr int NI = 4;
         const int QB = (Ho * Wo + 255) / 256;
-        dim3 grid((unsigned)(QB * ((N + NI - 1) / NI)), C);
-#define SBNN_DW_PX(S_, WT_) dwconv3x3_cm_px_kernel<S_, NI, WT_><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, QB, relu)
-#define SBNN_DW_S7(S_, WT_)                                                                                   \
+        const int cpb = Ho * Wo < 256 ? 256 / (Ho * Wo) : 1;          // channels per CTA for small planes
+        dim3 grid((unsigned)(QB * ((N + NI - 1) / NI)), (C + cpb - 1) / cpb);
+#define SBNN_DW_PX(S_, WT_) dwconv3x3_cm_px_kernel<S_, NI, WT_><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, C, QB, relu)
+#define SBNN_DW_C7(WT_)                                                                                       \
     {                                                                                                         \
-        const int items = Ho * (Wo / 7), qb = (items + 127) / 128;                                            \
-        dim3 g7((unsigned)(qb * ((N + NI - 1) / NI)), C);                                                     \
-        dwconv3x3_cm_strip7_kernel<S_, NI, WT_><<<g7, 128, 0, st>>>(w, b, x, ldx, y, ldy, N, H, relu);         \
+        const int items = (H / 7) * W, qb = (items + 127) / 128;                                              \
+        const int cpb7 = items < 128 ? 128 / items : 1;                                                       \
+        dim3 g7((unsigned)(qb * ((N + NI - 1) / NI)), (C + cpb7 - 1) / cpb7);                                 \
+        dwconv3x3_cm_col7_kernel<NI, WT_><<<g7, 128, 0, st>>>(w, b, x, ldx, y, ldy, N, H, C, relu);            \
     }
         if (stride == 1) {
-            if (W == 14) SBNN_DW_S7(1, 14)
-            else if (W == 7) SBNN_DW_S7(1, 7)
+            if (W == 14 && H % 7 == 0) SBNN_DW_C7(14)
+            else if (W == 7 && H % 7 == 0) SBNN_DW_C7(7)
             else SBNN_DW_PX(1, 0);
         } else {
             if (W == 28) SBNN_DW_PX(2, 28);      // stride 2: the per-position kernel measured faster
             else if (W == 14) SBNN_DW_PX(2, 14);
             else SBNN_DW_PX(2, 0);
         }
-#undef SBNN_DW_S7
+#undef SBNN_DW_C7
 #undef SBNN_DW_PX
     }
     SBNN_CUDA_TRY(cudaGetLastError());
