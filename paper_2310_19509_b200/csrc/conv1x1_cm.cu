@@ -21,6 +21,8 @@
 
 #include <algorithm>
 
+#include <cuda.h>   // CUtensorMap and the encode call's types only; the call itself is looked up at run time
+
 #include "common.h"
 #include "pipeline.cuh"
 
@@ -127,7 +129,7 @@ __device__ __forceinline__ void run_list(const uint4* r, int n, const unsigned c
 
 template <class C, bool OUT_CM>
 __global__ void __launch_bounds__(C::NT, 1)
-conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, int ldy,
+conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ Y, int ldy,
                   const float* __restrict__ bias, const uint4* __restrict__ rec,
                   const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout, int ngroups, int nchunks,
                   int ntiles, int total_tiles, int relu, int* status) {
@@ -163,19 +165,18 @@ conv1x1_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y, i
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const int tile = t % ntiles, m0 = (t / ntiles) * C::TM;
             const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
-            const uint32_t row_bytes = (uint32_t)min(C::TM, ldx - m0) * 4u;
             for (int k = 0; k < nchunks; ++k, ++issued) {
                 const int s = issued % S;
                 if (issued >= S) ok = mbar_wait(empty + s, ((issued / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
                 if (!ok) break;
-                const int rows = min(KC, Cin - k * KC);
-                const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
-                if (lane == 0) mbar_arrive_expect_tx(full + s, (uint32_t)rows * row_bytes + (uint32_t)wn * 16u);
-                __syncwarp();
-                unsigned char* xs = xs0 + (size_t)s * C::XS_BYTES;
-                for (int r = lane; r < rows; r += 32)
-                    bulk_g2s(xs + (size_t)r * C::ROW_BYTES, X + (size_t)(k * KC + r) * ldx + m0, row_bytes, full + s);
-                if (lane == 0) bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, full + s);
+                if (lane == 0) {
+                    // one tiled copy brings the step's KC x TM box of X (pixels past M and channels past Cin
+                    // arrive as zeros and count towards the bytes), a linear one the step's weight block
+                    const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
+                    mbar_arrive_expect_tx(full + s, (uint32_t)C::XS_BYTES + (uint32_t)wn * 16u);
+                    tensor_g2s_2d(xs0 + (size_t)s * C::XS_BYTES, &xmap, m0, k * KC, full + s);
+                    bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, full + s);
+                }
             }
         }
         if (!ok) {
@@ -464,6 +465,35 @@ int sm_count() {
     return it->second;
 }
 
+// Tensor map of the channel-major activations X [Cin][ldx] (M valid pixels per row), copied in boxes of
+// `box_rows` channels x `box_px` pixels.  The driver's encode routine is looked up once per process.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+sbnn_status encode_x_map(const float* x, int ldx, int M, int Cin, int box_px, int box_rows, CUtensorMap* out) {
+    static std::mutex mu;
+    static EncodeTiledFn encode = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        if (!encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            SBNN_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+            if (!fn || q != cudaDriverEntryPointSuccess) return fail(SBNN_ERR_CUDA, "driver has no cuTensorMapEncodeTiled");
+            encode = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+    }
+    if (!aligned16(x) || ldx % 4) return fail(SBNN_ERR_ALIGN, "channel-major activations need a 16-byte aligned base and ld %% 4 == 0");
+    const cuuint64_t dims[2] = {(cuuint64_t)M, (cuuint64_t)Cin};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)box_px, (cuuint32_t)box_rows}, elem_strides[2] = {1, 1};
+    const CUresult cr = encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(x), dims, strides, box, elem_strides,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return fail(SBNN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for M=%d Cin=%d ld=%d", (int)cr, M, Cin, ldx);
+    return SBNN_OK;
+}
+
 template <class C>
 sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, int ldx, float* y, int ldy, int M,
                       int relu, bool out_cm, cudaStream_t st) {
@@ -487,11 +517,14 @@ sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, 
     if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
     const int total_tiles = (int)nblk;
     dim3 grid((unsigned)std::min<long long>(nblk, sm_count()));
+    CUtensorMap xmap;
+    r = encode_x_map(x, ldx, M, p->Cin, C::TM, C::KC, &xmap);
+    if (r != SBNN_OK) return r;
     if (out_cm)
-        conv1x1_cm_kernel<C, true><<<grid, C::NT, C::SMEM, st>>>(x, ldx, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
+        conv1x1_cm_kernel<C, true><<<grid, C::NT, C::SMEM, st>>>(xmap, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
                                                                  p->ngroups, s.nchunks, s.ntiles, total_tiles, relu, status);
     else
-        conv1x1_cm_kernel<C, false><<<grid, C::NT, C::SMEM, st>>>(x, ldx, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
+        conv1x1_cm_kernel<C, false><<<grid, C::NT, C::SMEM, st>>>(xmap, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
                                                                   p->ngroups, s.nchunks, s.ntiles, total_tiles, relu, status);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;

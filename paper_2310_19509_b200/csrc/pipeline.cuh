@@ -81,4 +81,14 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, u
                  : "memory");
 }
 
+// ---- tiled copy global -> shared through a 2-D tensor map (opaque 128-byte descriptor made on the host) ----
+// Brings the box whose first element is (x, y) -- x along the contiguous dimension -- as [box rows][box width];
+// x * element size must be a multiple of 16 bytes, the destination 128-byte aligned.  Elements outside the
+// tensor arrive as zeros and count towards the completed bytes.
+__device__ __forceinline__ void tensor_g2s_2d(void* dst_smem, const void* tensor_map, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst_smem)), "l"(tensor_map), "r"(x), "r"(y), "r"(smem_u32(bar))
+                 : "memory");
+}
+
 }  // namespace sbnn
