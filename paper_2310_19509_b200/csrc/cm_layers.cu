@@ -83,6 +83,66 @@ dwconv3x3_cm_vec_kernel(const float* __restrict__ w, const float* __restrict__ b
     *reinterpret_cast<float4*>(y + (size_t)c * ldy + f * Wo + strip * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
 }
 
+// Row-block kernel (stride 1, W a multiple of 4, H a multiple of RR): a thread owns a strip of 4 columns in RR
+// consecutive output rows of one channel and walks the RR + 2 input rows once, so an input value is loaded
+// once per thread and the index arithmetic is shared by 4*RR outputs (the single-row kernel above is bound
+// by instruction issue).  The values left and right of the strip come from the neighbouring lanes by
+// shuffle; only the first and last lane of a warp fetch theirs from memory.  No thread leaves before the
+// shuffles: threads past the end work on a clamped position and store nothing.
+template <int RR>
+__global__ void __launch_bounds__(256)
+dwconv3x3_cm_rows_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
+                         float* __restrict__ y, int ldy, int items, int H, int W, int relu) {
+    const int c = blockIdx.y, C = gridDim.y;
+    const int spr = W >> 2;                                        // strips per row
+    const int t0 = blockIdx.x * blockDim.x + threadIdx.x, lane = threadIdx.x & 31;
+    const bool live = t0 < items;
+    const int t = live ? t0 : items - 1;
+    const int strip = t % spr, f0 = (t / spr) * RR;                // first output row (batch-wide row number)
+    const int oy0 = f0 % H;
+    float wk[9];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);
+    const float bias = b ? __ldg(b + c) : 0.0f;
+    float acc[RR][4];
+#pragma unroll
+    for (int o = 0; o < RR; ++o)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[o][i] = bias;
+    const float* xc = x + (size_t)c * ldx + (size_t)f0 * W + strip * 4;
+    const bool first = strip == 0, last = strip == spr - 1;
+#pragma unroll
+    for (int j = 0; j < RR + 2; ++j) {                             // input row f0 - 1 + j
+        const int iy = oy0 - 1 + j;
+        const bool rowok = iy >= 0 && iy < H;                      // else a row of the padding (or of the next image)
+        const float* row = xc + (j - 1) * W;
+        const float4 A = rowok ? __ldg(reinterpret_cast<const float4*>(row)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float Lw = __shfl_up_sync(0xffffffffu, A.w, 1), Rx = __shfl_down_sync(0xffffffffu, A.x, 1);
+        if (lane == 0 && !first && rowok) Lw = __ldg(row - 1);
+        if (lane == 31 && !last && rowok) Rx = __ldg(row + 4);
+        if (first) Lw = 0.0f;
+        if (last) Rx = 0.0f;
+        const float in[6] = {Lw, A.x, A.y, A.z, A.w, Rx};
+#pragma unroll
+        for (int kh = 0; kh < 3; ++kh) {
+            const int o = j - kh;                                  // output row fed through tap row kh
+            if (o >= 0 && o < RR) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    acc[o][i] = fmaf(in[i + 2], wk[kh * 3 + 2], fmaf(in[i + 1], wk[kh * 3 + 1], fmaf(in[i], wk[kh * 3], acc[o][i])));
+            }
+        }
+    }
+    if (!live) return;
+    float* yc = y + (size_t)c * ldy + (size_t)f0 * W + strip * 4;
+#pragma unroll
+    for (int o = 0; o < RR; ++o) {
+        float4 v = make_float4(acc[o][0], acc[o][1], acc[o][2], acc[o][3]);
+        if (relu) v = make_float4(fmaxf(v.x, 0.f), fmaxf(v.y, 0.f), fmaxf(v.z, 0.f), fmaxf(v.w, 0.f));
+        *reinterpret_cast<float4*>(yc + o * W) = v;
+    }
+}
+
 // Kernel for the other widths (the 14- and 7-wide maps of the network).  A thread owns one output
 // position (oy, ox) of one channel in up to NI consecutive images: the padding masks are computed
 // once and reused for every image.  Consecutive lanes own consecutive positions of the plane, so each
@@ -376,7 +436,12 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
     if (W % 4 == 0 && Wo % 4 == 0 && ldx % 4 == 0 && ldy % 4 == 0) {
         const long long threads = NHo * (Wo / 4);
         dim3 grid((unsigned)((threads + 255) / 256), C);
-        if (stride == 1)
+        constexpr int RR = 4;
+        const long long items = NHo / RR * (W / 4);
+        if (stride == 1 && H % RR == 0 && items > 0 && items < 0x7fffffffLL / 2) {
+            dim3 gr((unsigned)((items + 255) / 256), C);
+            dwconv3x3_cm_rows_kernel<RR><<<gr, 256, 0, st>>>(w, b, x, ldx, y, ldy, (int)items, H, W, relu);
+        } else if (stride == 1)
             dwconv3x3_cm_vec_kernel<1><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu);
         else
             dwconv3x3_cm_vec_kernel<2><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu);
