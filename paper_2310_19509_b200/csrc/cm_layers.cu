@@ -143,6 +143,63 @@ dwconv3x3_cm_rows_kernel(const float* __restrict__ w, const float* __restrict__ 
     }
 }
 
+// The same for stride 2 (W a multiple of 8, Ho a multiple of RR): 4 output columns x RR output rows per thread,
+// 2*RR + 1 input rows of 8 columns each plus the column left of them, which is the left neighbour's last.
+template <int RR>
+__global__ void __launch_bounds__(256)
+dwconv3x3_cm_rows_s2_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
+                            float* __restrict__ y, int ldy, int items, int Ho, int W, int relu) {
+    const int c = blockIdx.y, C = gridDim.y;
+    const int Wo = W >> 1, spr = Wo >> 2;
+    const int t0 = blockIdx.x * blockDim.x + threadIdx.x, lane = threadIdx.x & 31;
+    const bool live = t0 < items;
+    const int t = live ? t0 : items - 1;
+    const int strip = t % spr, f0 = (t / spr) * RR;                // first output row (batch-wide row number)
+    const int oy0 = f0 % Ho;
+    float wk[9];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);
+    const float bias = b ? __ldg(b + c) : 0.0f;
+    float acc[RR][4];
+#pragma unroll
+    for (int o = 0; o < RR; ++o)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[o][i] = bias;
+    const float* xc = x + (size_t)c * ldx + (size_t)(2 * f0) * W + strip * 8;   // input row 2*f0, first column of the strip
+    const bool first = strip == 0;
+#pragma unroll
+    for (int j = 0; j < 2 * RR + 1; ++j) {                         // input row 2*f0 - 1 + j
+        const bool rowok = j > 0 || oy0 > 0;                       // only the row above an image is padding
+        const float* row = xc + (j - 1) * W;
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 A = rowok ? __ldg(reinterpret_cast<const float4*>(row)) : z;
+        const float4 B = rowok ? __ldg(reinterpret_cast<const float4*>(row + 4)) : z;
+        float Lw = __shfl_up_sync(0xffffffffu, B.w, 1);
+        if (lane == 0 && !first && rowok) Lw = __ldg(row - 1);
+        if (first) Lw = 0.0f;
+        const float in[9] = {Lw, A.x, A.y, A.z, A.w, B.x, B.y, B.z, B.w};
+#pragma unroll
+        for (int kh = 0; kh < 3; ++kh) {
+            if ((j - kh) % 2 != 0) continue;
+            const int o = (j - kh) / 2;                            // output row fed through tap row kh
+            if (j - kh >= 0 && o < RR) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    acc[o][i] = fmaf(in[2 * i + 2], wk[kh * 3 + 2],
+                                     fmaf(in[2 * i + 1], wk[kh * 3 + 1], fmaf(in[2 * i], wk[kh * 3], acc[o][i])));
+            }
+        }
+    }
+    if (!live) return;
+    float* yc = y + (size_t)c * ldy + (size_t)f0 * Wo + strip * 4;
+#pragma unroll
+    for (int o = 0; o < RR; ++o) {
+        float4 v = make_float4(acc[o][0], acc[o][1], acc[o][2], acc[o][3]);
+        if (relu) v = make_float4(fmaxf(v.x, 0.f), fmaxf(v.y, 0.f), fmaxf(v.z, 0.f), fmaxf(v.w, 0.f));
+        *reinterpret_cast<float4*>(yc + o * Wo) = v;
+    }
+}
+
 // Kernel for the other widths (the 14- and 7-wide maps of the network).  A thread owns one output
 // position (oy, ox) of one channel in up to NI consecutive images: the padding masks are computed
 // once and reused for every image.  Consecutive lanes own consecutive positions of the plane, so each
@@ -441,6 +498,10 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
         if (stride == 1 && H % RR == 0 && items > 0 && items < 0x7fffffffLL / 2) {
             dim3 gr((unsigned)((items + 255) / 256), C);
             dwconv3x3_cm_rows_kernel<RR><<<gr, 256, 0, st>>>(w, b, x, ldx, y, ldy, (int)items, H, W, relu);
+        } else if (stride == 2 && Ho % RR == 0 && NHo / RR * (Wo / 4) > 0 && NHo / RR * (Wo / 4) < 0x7fffffffLL / 2) {
+            const long long items2 = NHo / RR * (Wo / 4);
+            dim3 gr((unsigned)((items2 + 255) / 256), C);
+            dwconv3x3_cm_rows_s2_kernel<RR><<<gr, 256, 0, st>>>(w, b, x, ldx, y, ldy, (int)items2, Ho, W, relu);
         } else if (stride == 1)
             dwconv3x3_cm_vec_kernel<1><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu);
         else
