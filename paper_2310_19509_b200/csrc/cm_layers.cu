@@ -90,7 +90,7 @@ dwconv3x3_cm_vec_kernel(const float* __restrict__ w, const float* __restrict__ b
 // shuffle; only the first and last lane of a warp fetch theirs from memory.  No thread leaves before the
 // shuffles: threads past the end work on a clamped position and store nothing.
 template <int RR>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 dwconv3x3_cm_rows_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
                          float* __restrict__ y, int ldy, int items, int H, int W, int relu) {
     const int c = blockIdx.y, C = gridDim.y;
@@ -111,18 +111,26 @@ dwconv3x3_cm_rows_kernel(const float* __restrict__ w, const float* __restrict__ 
         for (int i = 0; i < 4; ++i) acc[o][i] = bias;
     const float* xc = x + (size_t)c * ldx + (size_t)f0 * W + strip * 4;
     const bool first = strip == 0, last = strip == spr - 1;
+    // all loads first (they are independent), so that a thread has RR + 2 rows in flight
+    float4 A[RR + 2];
+    float Le[RR + 2], Re[RR + 2];
 #pragma unroll
     for (int j = 0; j < RR + 2; ++j) {                             // input row f0 - 1 + j
         const int iy = oy0 - 1 + j;
         const bool rowok = iy >= 0 && iy < H;                      // else a row of the padding (or of the next image)
         const float* row = xc + (j - 1) * W;
-        const float4 A = rowok ? __ldg(reinterpret_cast<const float4*>(row)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        float Lw = __shfl_up_sync(0xffffffffu, A.w, 1), Rx = __shfl_down_sync(0xffffffffu, A.x, 1);
-        if (lane == 0 && !first && rowok) Lw = __ldg(row - 1);
-        if (lane == 31 && !last && rowok) Rx = __ldg(row + 4);
+        A[j] = rowok ? __ldg(reinterpret_cast<const float4*>(row)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        Le[j] = (lane == 0 && !first && rowok) ? __ldg(row - 1) : 0.0f;
+        Re[j] = (lane == 31 && !last && rowok) ? __ldg(row + 4) : 0.0f;
+    }
+#pragma unroll
+    for (int j = 0; j < RR + 2; ++j) {
+        float Lw = __shfl_up_sync(0xffffffffu, A[j].w, 1), Rx = __shfl_down_sync(0xffffffffu, A[j].x, 1);
+        if (lane == 0) Lw = Le[j];
+        if (lane == 31) Rx = Re[j];
         if (first) Lw = 0.0f;
         if (last) Rx = 0.0f;
-        const float in[6] = {Lw, A.x, A.y, A.z, A.w, Rx};
+        const float in[6] = {Lw, A[j].x, A[j].y, A[j].z, A[j].w, Rx};
 #pragma unroll
         for (int kh = 0; kh < 3; ++kh) {
             const int o = j - kh;                                  // output row fed through tap row kh
@@ -146,7 +154,7 @@ dwconv3x3_cm_rows_kernel(const float* __restrict__ w, const float* __restrict__ 
 // The same for stride 2 (W a multiple of 8, Ho a multiple of RR): 4 output columns x RR output rows per thread,
 // 2*RR + 1 input rows of 8 columns each plus the column left of them, which is the left neighbour's last.
 template <int RR>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 dwconv3x3_cm_rows_s2_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
                             float* __restrict__ y, int ldy, int items, int Ho, int W, int relu) {
     const int c = blockIdx.y, C = gridDim.y;
@@ -167,17 +175,23 @@ dwconv3x3_cm_rows_s2_kernel(const float* __restrict__ w, const float* __restrict
         for (int i = 0; i < 4; ++i) acc[o][i] = bias;
     const float* xc = x + (size_t)c * ldx + (size_t)(2 * f0) * W + strip * 8;   // input row 2*f0, first column of the strip
     const bool first = strip == 0;
+    float4 A[2 * RR + 1], B[2 * RR + 1];                           // all loads first: 2*RR + 1 rows in flight
+    float Le[2 * RR + 1];
 #pragma unroll
     for (int j = 0; j < 2 * RR + 1; ++j) {                         // input row 2*f0 - 1 + j
         const bool rowok = j > 0 || oy0 > 0;                       // only the row above an image is padding
         const float* row = xc + (j - 1) * W;
         const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float4 A = rowok ? __ldg(reinterpret_cast<const float4*>(row)) : z;
-        const float4 B = rowok ? __ldg(reinterpret_cast<const float4*>(row + 4)) : z;
-        float Lw = __shfl_up_sync(0xffffffffu, B.w, 1);
-        if (lane == 0 && !first && rowok) Lw = __ldg(row - 1);
+        A[j] = rowok ? __ldg(reinterpret_cast<const float4*>(row)) : z;
+        B[j] = rowok ? __ldg(reinterpret_cast<const float4*>(row + 4)) : z;
+        Le[j] = (lane == 0 && !first && rowok) ? __ldg(row - 1) : 0.0f;
+    }
+#pragma unroll
+    for (int j = 0; j < 2 * RR + 1; ++j) {
+        float Lw = __shfl_up_sync(0xffffffffu, B[j].w, 1);
+        if (lane == 0) Lw = Le[j];
         if (first) Lw = 0.0f;
-        const float in[9] = {Lw, A.x, A.y, A.z, A.w, B.x, B.y, B.z, B.w};
+        const float in[9] = {Lw, A[j].x, A[j].y, A[j].z, A[j].w, B[j].x, B[j].y, B[j].z, B[j].w};
 #pragma unroll
         for (int kh = 0; kh < 3; ++kh) {
             if ((j - kh) % 2 != 0) continue;
@@ -496,12 +510,12 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
         constexpr int RR = 4;
         const long long items = NHo / RR * (W / 4);
         if (stride == 1 && H % RR == 0 && items > 0 && items < 0x7fffffffLL / 2) {
-            dim3 gr((unsigned)((items + 255) / 256), C);
-            dwconv3x3_cm_rows_kernel<RR><<<gr, 256, 0, st>>>(w, b, x, ldx, y, ldy, (int)items, H, W, relu);
-        } else if (stride == 2 && Ho % RR == 0 && NHo / RR * (Wo / 4) > 0 && NHo / RR * (Wo / 4) < 0x7fffffffLL / 2) {
-            const long long items2 = NHo / RR * (Wo / 4);
-            dim3 gr((unsigned)((items2 + 255) / 256), C);
-            dwconv3x3_cm_rows_s2_kernel<RR><<<gr, 256, 0, st>>>(w, b, x, ldx, y, ldy, (int)items2, Ho, W, relu);
+            dim3 gr((unsigned)((items + 127) / 128), C);
+            dwconv3x3_cm_rows_kernel<RR><<<gr, 128, 0, st>>>(w, b, x, ldx, y, ldy, (int)items, H, W, relu);
+        } else if (stride == 2 && Ho % 2 == 0 && NHo / 2 * (Wo / 4) > 0 && NHo / 2 * (Wo / 4) < 0x7fffffffLL / 2) {
+            const long long items2 = NHo / 2 * (Wo / 4);
+            dim3 gr((unsigned)((items2 + 127) / 128), C);
+            dwconv3x3_cm_rows_s2_kernel<2><<<gr, 128, 0, st>>>(w, b, x, ldx, y, ldy, (int)items2, Ho, W, relu);
         } else if (stride == 1)
             dwconv3x3_cm_vec_kernel<1><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu);
         else
