@@ -88,7 +88,8 @@ namespace sbnn {
 sbnn_status prepare_default_1x1(const sbnn_packed* p);
 void free_streams_1x1(sbnn_packed* p);
 // conv1x1_cm.cu
-sbnn_status prepare_default_cm(const sbnn_packed* p);
+// Builds the weight stream of the tile shape that a launch on M pixels would pick (M <= 0: the many-pixel choice).
+sbnn_status prepare_default_cm(const sbnn_packed* p, long long M = 0);
 sbnn_status prepare_cm(const sbnn_packed* p, int P, int GPW, int NW, int KC);   // builds the stream of one tile shape
 void free_streams_cm(sbnn_packed* p);
 // Runs the NHWC call through the channel-major kernel if the shape profits; *done tells whether it did.

@@ -103,7 +103,9 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
     // The kernel-private weight layouts of the channel-major 1x1 kernel are built here, not in forward.
     for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
         if (pw[i]->device < 0) return fail(SBNN_ERR_CUDA, "pointwise layer %d was packed without a CUDA device", i + 1);
-        if ((st = prepare_default_cm(pw[i])) != SBNN_OK) return st;
+        const int hw = layer_table()[2 + 2 * i].hin;                 // the block's pointwise layer is entry 2 + 2*i
+        if ((st = prepare_default_cm(pw[i], (long long)max_batch * hw * hw)) != SBNN_OK) return st;
+        if ((st = prepare_default_cm(pw[i], (long long)hw * hw)) != SBNN_OK) return st;   // and the batch-1 choice
     }
     if (fc->device < 0) return fail(SBNN_ERR_CUDA, "the classifier was packed without a CUDA device");
     {
