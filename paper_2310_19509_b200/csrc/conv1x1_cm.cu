@@ -20,6 +20,7 @@
 #include <limits.h>
 
 #include <algorithm>
+#include <initializer_list>
 
 #include <cuda.h>   // CUtensorMap and the encode call's types only; the call itself is looked up at run time
 
@@ -536,6 +537,7 @@ sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, 
     X(2, 8, 2, 8, 32, 4)   \
     X(4, 8, 1, 16, 32, 4)  \
     X(4, 8, 2, 8, 32, 4)   \
+    X(4, 8, 2, 11, 32, 3)  \
     X(4, 8, 2, 12, 32, 3)  \
     X(4, 4, 1, 8, 32, 4)   \
     X(8, 8, 1, 8, 32, 4)   \
@@ -560,17 +562,27 @@ sbnn_status dispatch_cm(const sbnn_packed* p, const TileCfg& c, const float* x, 
 
 // Tile shape for a layer run on M pixels.  M <= 0 stands for "many pixels" (the choice made before M is known).
 TileCfg default_cfg_cm(const sbnn_packed* p, long long M) {
-    // Whole tiles are dealt to the SMs, so a launch takes ceil(tiles / SMs) rounds of one tile each.  Where 8 and
-    // 12 compute warps per CTA are both instantiated, take 12 when its larger tiles fill the rounds better
-    // (a 12-warp tile holds 1.5x the work and runs about 5 % more efficiently than 1.5 tiles of 8 warps).
-    auto rounds_cost = [&](int P, int GT, double work_per_tile) {
-        const long long ptiles = (M + 32 * P - 1) / (32 * P), gtiles = (p->ngroups + GT - 1) / GT;
+    // Whole tiles are dealt to the SMs, so a launch takes ceil(tiles / SMs) rounds of one tile each, and a tile's
+    // time grows with its compute warps.  Among the warp counts instantiated for the layer's G take the one with
+    // the cheapest rounds (CTAs of 11 or 12 compute warps run about 5 % more efficiently per warp than 8), and
+    // stay with 8 unless another is at least 3 % cheaper.
+    auto rounds_cost = [&](const TileCfg& c) {
+        const long long ptiles = (M + c.TM() - 1) / c.TM(), gtiles = (p->ngroups + c.GT() - 1) / c.GT();
         const long long sms = std::max(1, sm_count());
-        return (double)((ptiles * gtiles + sms - 1) / sms) * work_per_tile;
+        return (double)((ptiles * gtiles + sms - 1) / sms) * c.NW / (c.NW > 8 ? 1.05 : 1.0);
     };
-    auto pick = [&](const TileCfg& a, const TileCfg& b) {   // b is the 12-warp variant of a
-        if (M <= 0) return a;
-        return rounds_cost(b.P, b.GT(), 1.5 / 1.05) < 0.97 * rounds_cost(a.P, a.GT(), 1.0) ? b : a;
+    auto pick = [&](const TileCfg& base, std::initializer_list<TileCfg> others) {
+        if (M <= 0) return base;
+        TileCfg best = base;
+        double best_cost = 0.97 * rounds_cost(base);
+        for (const TileCfg& c : others) {
+            const double cost = rounds_cost(c);
+            if (cost < best_cost) {
+                best = c;
+                best_cost = cost;
+            }
+        }
+        return best;
     };
     switch (p->G) {
         case 1: return {8, 4, 8, 32};
@@ -580,8 +592,8 @@ TileCfg default_cfg_cm(const sbnn_packed* p, long long M) {
             // each hide the per-step latencies better than the shared activation fetch of two groups saves
             // (measured cross-over between 50 % and 70 % removed units).
             if ((double)p->nnz < 0.4 * (double)p->ngroups * p->Cin) return {8, 1, 16, 32};
-            return pick({8, 2, 8, 32}, {8, 2, 12, 32});
-        case 8: return pick({8, 1, 8, 32}, {8, 1, 12, 32});
+            return pick({8, 2, 8, 32}, {{8, 2, 11, 32}, {8, 2, 12, 32}});
+        case 8: return pick({8, 1, 8, 32}, {{8, 1, 12, 32}});
         default: return {4, 1, 8, 32};
     }
 }
