@@ -3,10 +3,11 @@
 //   Y[m][g*G + r] = act( bias[g*G + r] + sum_j val[g][j][r] * X[idx[g][j]][m] ),   X given as [Cin][ldx]
 //
 // With the pixels of one input channel contiguous in global memory, the [channel][pixel] shared
-// memory tile that the compute warps want is a set of plain row copies, so the staging is done by
+// memory tile that the compute warps want is a plain 2-D box of X, so the staging is done by
 // the copy engine and costs the SM no instructions:
-//   * warp NW (the producer) issues, per channel step, one bulk asynchronous copy per channel row
-//     and one for the step's weight block; their bytes complete a "full" mbarrier of the stage;
+//   * warp NW (the producer) issues, per channel step, one tiled tensor-map copy of the step's
+//     KC x TM box (one copy per channel row was measured to cap staging at a fifth of this rate)
+//     and one linear copy of the step's weight block; their bytes complete a "full" mbarrier of the stage;
 //   * the NW compute warps wait on "full", run their kept units out of the stage, and each
 //     releases it by arriving on the stage's "empty" mbarrier; STAGES stages are in flight, so warps
 //     whose groups keep more units in a step are not waited for until STAGES steps later
