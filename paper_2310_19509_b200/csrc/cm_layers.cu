@@ -4,6 +4,7 @@
 // The MobileNet chain keeps every intermediate activation in this layout so that the group-sparse
 // 1x1 kernel can fill its shared-memory tiles with plain row copies.
 #include "common.h"
+#include "pipeline.cuh"
 
 namespace sbnn {
 namespace {
@@ -393,7 +394,7 @@ conv3x3_thin_cm_kernel(const float* __restrict__ w, const float* __restrict__ b,
 
 // Wide variant for Cout % 32 == 0: one thread computes 2 consecutive output columns x 32 output
 // channels, so every input value is loaded once per pixel pair (not once per channel group) and each
-// broadcast float4 of weights feeds 8 FMAs.  Consecutive lanes take consecutive column pairs; a
+// broadcast float4 of weights feeds 4 packed FMAs (pairs of output channels, fma.rn.f32x2).  Consecutive lanes take consecutive column pairs; a
 // channel's stores are 8-byte pieces that are contiguous across the warp.
 template <int S>
 __global__ void __launch_bounds__(128)
@@ -417,12 +418,12 @@ conv3x3_thin_cm32_kernel(const float* __restrict__ w, const float* __restrict__ 
     const int n = (int)(f / Ho);
     const int ox0 = sx * TW, ix0 = ox0 * S - 1;
 
-    float acc[TW][32];
+    f32x2 acc[TW][16];                                             // packed pairs of output channels
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        const float bv = b ? __ldg(b + cg * 32 + j) : 0.f;
+    for (int j = 0; j < 16; ++j) {
+        const float b0 = b ? __ldg(b + cg * 32 + 2 * j) : 0.f, b1 = b ? __ldg(b + cg * 32 + 2 * j + 1) : 0.f;
 #pragma unroll
-        for (int i = 0; i < TW; ++i) acc[i][j] = bv;
+        for (int i = 0; i < TW; ++i) acc[i][j] = pack2(b0, b1);
     }
 #pragma unroll
     for (int kh = 0; kh < 3; ++kh) {
@@ -430,25 +431,22 @@ conv3x3_thin_cm32_kernel(const float* __restrict__ w, const float* __restrict__ 
         if (iy < 0 || iy >= H) continue;
         const float* row = x + ((size_t)n * H + iy) * W * Cin;
         for (int c = 0; c < Cin; ++c) {
-            float in[IW];
+            f32x2 in[IW];
 #pragma unroll
             for (int j = 0; j < IW; ++j) {
                 const int ix = ix0 + j;
-                in[j] = (ix >= 0 && ix < W) ? __ldg(row + (size_t)ix * Cin + c) : 0.f;
+                in[j] = dup2((ix >= 0 && ix < W) ? __ldg(row + (size_t)ix * Cin + c) : 0.f);
             }
 #pragma unroll
             for (int kw = 0; kw < 3; ++kw) {
-                const float4* wp = reinterpret_cast<const float4*>(ws + ((kh * 3 + kw) * Cin + c) * 32);
+                const ulonglong2* wp = reinterpret_cast<const ulonglong2*>(ws + ((kh * 3 + kw) * Cin + c) * 32);
 #pragma unroll
                 for (int v = 0; v < 8; ++v) {
-                    const float4 wv = wp[v];
+                    const ulonglong2 wv = wp[v];                   // channels (4v, 4v+1) and (4v+2, 4v+3)
 #pragma unroll
                     for (int i = 0; i < TW; ++i) {
-                        const float a = in[i * S + kw];
-                        acc[i][4 * v + 0] = fmaf(a, wv.x, acc[i][4 * v + 0]);
-                        acc[i][4 * v + 1] = fmaf(a, wv.y, acc[i][4 * v + 1]);
-                        acc[i][4 * v + 2] = fmaf(a, wv.z, acc[i][4 * v + 2]);
-                        acc[i][4 * v + 3] = fmaf(a, wv.w, acc[i][4 * v + 3]);
+                        fma2(acc[i][2 * v], in[i * S + kw], wv.x);
+                        fma2(acc[i][2 * v + 1], in[i * S + kw], wv.y);
                     }
                 }
             }
@@ -457,15 +455,21 @@ conv3x3_thin_cm32_kernel(const float* __restrict__ w, const float* __restrict__ 
     const long long p0 = f * Wo + ox0;
     const bool vec = (ox0 + 1 < Wo) && ((p0 & 1) == 0);
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        float v0 = acc[0][j], v1 = acc[1][j];
-        if (relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
-        float* yp = y + (size_t)(cg * 32 + j) * ldy + p0;
-        if (vec) {
-            *reinterpret_cast<float2*>(yp) = make_float2(v0, v1);
-        } else {
-            yp[0] = v0;
-            if (ox0 + 1 < Wo) yp[1] = v1;
+    for (int j = 0; j < 16; ++j) {
+        float v0[2], v1[2];
+        unpack2(acc[0][j], v0[0], v0[1]);
+        unpack2(acc[1][j], v1[0], v1[1]);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            float a0 = v0[e], a1 = v1[e];
+            if (relu) { a0 = fmaxf(a0, 0.f); a1 = fmaxf(a1, 0.f); }
+            float* yp = y + (size_t)(cg * 32 + 2 * j + e) * ldy + p0;
+            if (vec) {
+                *reinterpret_cast<float2*>(yp) = make_float2(a0, a1);
+            } else {
+                yp[0] = a0;
+                if (ox0 + 1 < Wo) yp[1] = a1;
+            }
         }
     }
 }
