@@ -197,14 +197,17 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
     const int tile = t % ntiles, m0 = (t / ntiles) * C::TM;
     f32x2 acc[GPW][P / 2][G];   // acc[q][p2][r]: pixels (2*p2, 2*p2+1) of the lane, channel r of group q
+    // The bias is fetched now and added in the epilogue: nothing waits for this global load until then,
+    // which matters for layers with few channel steps per tile.
+    float bv[GPW][G];
 #pragma unroll
     for (int q = 0; q < GPW; ++q) {
         const int g = tile * C::GT + warp * GPW + q;
 #pragma unroll
         for (int r = 0; r < G; ++r) {
-            const float b = (g < ngroups) ? bias[g * G + r] : 0.0f;
+            bv[q][r] = (g < ngroups) ? __ldg(bias + g * G + r) : 0.0f;
 #pragma unroll
-            for (int p = 0; p < P / 2; ++p) acc[q][p][r] = pack2(b, b);
+            for (int p = 0; p < P / 2; ++p) acc[q][p][r] = pack2(0.0f, 0.0f);
         }
     }
 
@@ -246,6 +249,8 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
             for (int rr = 0; rr < G; ++rr) {
                 unpack2(acc[q][2 * i][rr], v[0][rr], v[1][rr]);
                 unpack2(acc[q][2 * i + 1][rr], v[2][rr], v[3][rr]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) v[e][rr] += bv[q][rr];
             }
             if (relu) {
 #pragma unroll
