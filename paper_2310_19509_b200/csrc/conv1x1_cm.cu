@@ -199,13 +199,15 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
     f32x2 acc[GPW][P / 2][G];   // acc[q][p2][r]: pixels (2*p2, 2*p2+1) of the lane, channel r of group q
     // The bias is fetched now and added in the epilogue: nothing waits for this global load until then,
     // which matters for layers with few channel steps per tile.
+    // (Shapes whose main loop already uses every register fetch it at the start of the epilogue instead.)
+    constexpr bool BIAS_EARLY = G * GPW * P < 64 || G < 8;
     float bv[GPW][G];
 #pragma unroll
     for (int q = 0; q < GPW; ++q) {
         const int g = tile * C::GT + warp * GPW + q;
 #pragma unroll
         for (int r = 0; r < G; ++r) {
-            bv[q][r] = (g < ngroups) ? __ldg(bias + g * G + r) : 0.0f;
+            if constexpr (BIAS_EARLY) bv[q][r] = (g < ngroups) ? __ldg(bias + g * G + r) : 0.0f;
 #pragma unroll
             for (int p = 0; p < P / 2; ++p) acc[q][p][r] = pack2(0.0f, 0.0f);
         }
@@ -237,6 +239,14 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
     if (!ok) return;
 
     // epilogue
+    if constexpr (!BIAS_EARLY) {
+#pragma unroll
+        for (int q = 0; q < GPW; ++q) {
+            const int g = tile * C::GT + warp * GPW + q;
+#pragma unroll
+            for (int r = 0; r < G; ++r) bv[q][r] = (g < ngroups) ? __ldg(bias + g * G + r) : 0.0f;
+        }
+    }
 #pragma unroll
     for (int q = 0; q < GPW; ++q) {
         const int g = tile * C::GT + warp * GPW + q;
