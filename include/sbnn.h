@@ -89,6 +89,18 @@ typedef struct sbnn_packed sbnn_packed;
 SBNN_API sbnn_status sbnn_pack_weights(const float* W_host, const uint8_t* mask_host, const float* bias_host,
                                        int Cout, int KH, int KW, int Cin, int G, sbnn_packed** out);
 
+/*
+ * Kernel-pattern variant of packing (Section 3.3, last paragraph: pattern pruning of Conv3x3 in the manner of
+ * PatDNN, one pattern shared by adjacent filters; Section 3.2 for the patterns of a kernel).  Same arguments
+ * and layout as sbnn_pack_weights, but the taps of a unit may be masked individually: the mask must still be
+ * identical for the G filters of a group (the pattern is shared by the group), a unit is kept if any of its
+ * KH*KW taps is, pruned taps are stored as 0.0f in val, and the view's tap_mask records which taps were kept,
+ * so that sbnn_unpack_weights returns the mask exactly.  The convolution entry points take the result like
+ * any other packed layer (pruned taps are multiplied as zeros; they are not skipped).
+ */
+SBNN_API sbnn_status sbnn_pack_weights_pattern(const float* W_host, const uint8_t* mask_host, const float* bias_host,
+                                               int Cout, int KH, int KW, int Cin, int G, sbnn_packed** out);
+
 typedef struct {
     int Cout, KH, KW, Cin, G, ngroups;
     int64_t nnz_units;
@@ -96,6 +108,8 @@ typedef struct {
     const int32_t* idx;       /* host, borrowed */
     const float* val;         /* host, borrowed */
     const float* bias;        /* host, borrowed */
+    const uint16_t* tap_mask; /* host, borrowed: [nnz_units], bit t = tap t of the unit is kept; NULL unless the layer
+                                 was packed by sbnn_pack_weights_pattern */
 } sbnn_packed_view;
 
 /* Borrow the canonical host arrays; they stay valid until sbnn_packed_free. */

@@ -146,6 +146,37 @@ def pack(w, mask, g):
     return np.array(group_ptr, dtype=np.int32), np.array(idx, dtype=np.int32), val
 
 
+def pack_pattern(w, mask, g):
+    """Packing when the taps of a kernel are pruned individually (kernel patterns shared by the g filters of a
+    group; Section 3.3's Conv3x3 pattern pruning).
+
+    A unit (group, input channel) is kept iff any of its taps is; its pruned taps are stored as zeros.  Returns
+    (group_ptr, idx, val, tap_mask) with tap_mask uint16 [nnzU], bit t set iff tap t = kh*KW + kw is kept.
+    """
+    w = np.asarray(w, dtype=np.float32)
+    mask = np.asarray(mask, dtype=np.uint8)
+    cout, kh, kw, cin = w.shape
+    if cout % g:
+        raise ValueError("Cout % G != 0")
+    group_ptr, idx, val, tap_mask = [0], [], [], []
+    for gi in range(cout // g):
+        rows = mask[gi * g:(gi + 1) * g].reshape(g, kh * kw, cin)
+        if np.any(rows != rows[0][None]) or np.any(rows > 1):
+            raise MaskNotGroupUniform(f"group {gi}")
+        wg = w[gi * g:(gi + 1) * g].reshape(g, kh * kw, cin)
+        for c in range(cin):
+            taps = rows[0, :, c]
+            if not taps.any():
+                continue
+            idx.append(c)
+            tap_mask.append(sum(1 << t for t in range(kh * kw) if taps[t]))
+            val.append(np.where(taps[None, :] != 0, wg[:, :, c], np.float32(0)).T)   # [taps][g]
+        group_ptr.append(len(idx))
+    val = np.array(val, dtype=np.float32).reshape(len(idx), kh * kw, g)
+    return (np.array(group_ptr, dtype=np.int32), np.array(idx, dtype=np.int32), val,
+            np.array(tap_mask, dtype=np.uint16))
+
+
 def unpack(group_ptr, idx, val, cout, kh, kw, cin, g):
     """Inverse of pack: returns (W (.) M, M)."""
     w = np.zeros((cout, kh, kw, cin), dtype=np.float32)

@@ -20,7 +20,7 @@ class SbnnError(RuntimeError):
 class _View(C.Structure):
     _fields_ = [("Cout", C.c_int), ("KH", C.c_int), ("KW", C.c_int), ("Cin", C.c_int), ("G", C.c_int),
                 ("ngroups", C.c_int), ("nnz_units", C.c_int64), ("group_ptr", C.c_void_p), ("idx", C.c_void_p),
-                ("val", C.c_void_p), ("bias", C.c_void_p)]
+                ("val", C.c_void_p), ("bias", C.c_void_p), ("tap_mask", C.c_void_p)]
 
 
 def lib_path() -> str:
@@ -40,6 +40,7 @@ def lib():
     P, I = C.c_void_p, C.c_int
     sig = {
         "sbnn_pack_weights": [P, P, P, I, I, I, I, I, P],
+        "sbnn_pack_weights_pattern": [P, P, P, I, I, I, I, I, P],
         "sbnn_packed_get": [P, P],
         "sbnn_unpack_weights": [P, P, P],
         "sbnn_packed_free": [P],
@@ -123,7 +124,8 @@ class Packed:
         return dict(Cout=v.Cout, KH=v.KH, KW=v.KW, Cin=v.Cin, G=v.G, ngroups=v.ngroups, nnz_units=v.nnz_units,
                     group_ptr=arr(v.group_ptr, v.ngroups + 1, np.int32), idx=arr(v.idx, v.nnz_units, np.int32),
                     val=arr(v.val, v.nnz_units * taps * v.G, np.float32).reshape(v.nnz_units, taps, v.G),
-                    bias=arr(v.bias, v.Cout, np.float32))
+                    bias=arr(v.bias, v.Cout, np.float32),
+                    tap_mask=arr(v.tap_mask, v.nnz_units, np.uint16) if v.tap_mask else None)
 
     def unpack(self):
         v = _View()
@@ -145,7 +147,8 @@ class Packed:
             pass
 
 
-def pack_weights(w, mask, bias, g) -> Packed:
+def pack_weights(w, mask, bias, g, tap_patterns=False) -> Packed:
+    """tap_patterns=True packs through sbnn_pack_weights_pattern (taps of a unit masked individually)."""
     w = np.ascontiguousarray(w, dtype=np.float32)
     mask = np.ascontiguousarray(mask, dtype=np.uint8)
     if w.ndim != 4 or mask.shape != w.shape:
@@ -153,8 +156,8 @@ def pack_weights(w, mask, bias, g) -> Packed:
     cout, kh, kw, cin = w.shape
     b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
     h = C.c_void_p()
-    _check(lib().sbnn_pack_weights(w.ctypes.data, mask.ctypes.data, None if b is None else b.ctypes.data,
-                                   cout, kh, kw, cin, int(g), C.byref(h)))
+    fn = lib().sbnn_pack_weights_pattern if tap_patterns else lib().sbnn_pack_weights
+    _check(fn(w.ctypes.data, mask.ctypes.data, None if b is None else b.ctypes.data, cout, kh, kw, cin, int(g), C.byref(h)))
     return Packed(h)
 
 

@@ -69,6 +69,7 @@ struct sbnn_packed {
     int64_t nnz = 0;
     std::vector<int32_t> group_ptr, idx;
     std::vector<float> val, bias;
+    std::vector<uint16_t> tap_mask;   // per kept unit, bit t = tap t kept; empty unless packed with tap patterns
     // device side (valid when device >= 0)
     int device = -1;
     int32_t* d_group_ptr = nullptr;

@@ -85,8 +85,12 @@ extern "C" const char* sbnn_status_str(sbnn_status s) {
 
 extern "C" const char* sbnn_last_error(void) { return g_err; }
 
-extern "C" sbnn_status sbnn_pack_weights(const float* W, const uint8_t* mask, const float* bias, int Cout, int KH,
-                                         int KW, int Cin, int G, sbnn_packed** out) {
+namespace {
+// tap_patterns = false: a unit's mask is one value for all taps (connectivity pruning only).
+// tap_patterns = true: the taps of a unit may differ (kernel patterns), but not between the G filters of the group;
+// a unit is kept if any of its taps is, pruned taps are stored as zeros and remembered in tap_mask.
+sbnn_status pack_impl(const float* W, const uint8_t* mask, const float* bias, int Cout, int KH, int KW, int Cin, int G,
+                      bool tap_patterns, sbnn_packed** out) {
     clear_error();
     if (!W || !mask || !out) return fail(SBNN_ERR_NULL, "W_host, mask_host and out must not be NULL");
     *out = nullptr;
@@ -105,41 +109,53 @@ extern "C" sbnn_status sbnn_pack_weights(const float* W, const uint8_t* mask, co
         p->group_ptr.assign(p->ngroups + 1, 0);
         p->bias.assign(Cout, 0.0f);
         if (bias) memcpy(p->bias.data(), bias, sizeof(float) * Cout);
-        // Pass 1: validate that a unit is kept or removed as a whole, and count.
+        // Pass 1: validate the mask's structure and count the kept units.
+        std::vector<uint16_t> unit_taps((size_t)p->ngroups * Cin, 0);   // bit t = tap t of the unit is kept
         for (int g = 0; g < p->ngroups; ++g) {
             const uint8_t* m0 = mask + (int64_t)g * G * row;  // first row, first tap
             int kept = 0;
             for (int c = 0; c < Cin; ++c) {
-                const uint8_t ref = m0[c];
-                if (ref > 1) {
-                    delete p;
-                    return fail(SBNN_ERR_MASK_NOT_GROUP_UNIFORM, "mask value %d at group %d channel %d is not 0/1", ref, g, c);
-                }
-                for (int r = 0; r < G; ++r)
-                    for (int t = 0; t < taps; ++t)
+                unsigned bits = 0;
+                for (int t = 0; t < taps; ++t) {
+                    const uint8_t ref = m0[(int64_t)t * Cin + c];
+                    if (ref > 1) {
+                        delete p;
+                        return fail(SBNN_ERR_MASK_NOT_GROUP_UNIFORM, "mask value %d at group %d channel %d is not 0/1", ref, g, c);
+                    }
+                    if (!tap_patterns && ref != m0[c]) {
+                        delete p;
+                        return fail(SBNN_ERR_MASK_NOT_GROUP_UNIFORM, "mask of group %d differs at row 0 tap %d channel %d", g, t, c);
+                    }
+                    for (int r = 1; r < G; ++r)
                         if (m0[(int64_t)r * row + (int64_t)t * Cin + c] != ref) {
                             delete p;
                             return fail(SBNN_ERR_MASK_NOT_GROUP_UNIFORM,
                                         "mask of group %d differs at row %d tap %d channel %d", g, r, t, c);
                         }
-                kept += ref;
+                    bits |= (unsigned)ref << t;
+                }
+                unit_taps[(size_t)g * Cin + c] = (uint16_t)bits;
+                kept += bits != 0;
             }
             p->group_ptr[g + 1] = p->group_ptr[g] + kept;
         }
         p->nnz = p->group_ptr[p->ngroups];
         p->idx.resize(p->nnz);
         p->val.resize((size_t)p->nnz * taps * G);
+        if (tap_patterns) p->tap_mask.resize(p->nnz);
         // Pass 2: emit ascending indices and the [taps][G] value block of every kept unit.
         for (int g = 0; g < p->ngroups; ++g) {
-            const uint8_t* m0 = mask + (int64_t)g * G * row;
             const float* w0 = W + (int64_t)g * G * row;
             int64_t u = p->group_ptr[g];
             for (int c = 0; c < Cin; ++c) {
-                if (!m0[c]) continue;
+                const unsigned bits = unit_taps[(size_t)g * Cin + c];
+                if (!bits) continue;
                 p->idx[u] = c;
+                if (tap_patterns) p->tap_mask[u] = (uint16_t)bits;
                 float* v = p->val.data() + (size_t)u * taps * G;
                 for (int t = 0; t < taps; ++t)
-                    for (int r = 0; r < G; ++r) v[t * G + r] = w0[(int64_t)r * row + (int64_t)t * Cin + c];
+                    for (int r = 0; r < G; ++r)
+                        v[t * G + r] = ((bits >> t) & 1u) ? w0[(int64_t)r * row + (int64_t)t * Cin + c] : 0.0f;
                 ++u;
             }
         }
@@ -170,6 +186,17 @@ extern "C" sbnn_status sbnn_pack_weights(const float* W, const uint8_t* mask, co
     *out = p;
     return SBNN_OK;
 }
+}  // namespace
+
+extern "C" sbnn_status sbnn_pack_weights(const float* W, const uint8_t* mask, const float* bias, int Cout, int KH,
+                                         int KW, int Cin, int G, sbnn_packed** out) {
+    return pack_impl(W, mask, bias, Cout, KH, KW, Cin, G, false, out);
+}
+
+extern "C" sbnn_status sbnn_pack_weights_pattern(const float* W, const uint8_t* mask, const float* bias, int Cout, int KH,
+                                                 int KW, int Cin, int G, sbnn_packed** out) {
+    return pack_impl(W, mask, bias, Cout, KH, KW, Cin, G, true, out);
+}
 
 extern "C" sbnn_status sbnn_packed_get(const sbnn_packed* p, sbnn_packed_view* v) {
     clear_error();
@@ -180,6 +207,7 @@ extern "C" sbnn_status sbnn_packed_get(const sbnn_packed* p, sbnn_packed_view* v
     v->idx = p->idx.data();
     v->val = p->val.data();
     v->bias = p->bias.data();
+    v->tap_mask = p->tap_mask.empty() ? nullptr : p->tap_mask.data();
     return SBNN_OK;
 }
 
@@ -198,7 +226,7 @@ extern "C" sbnn_status sbnn_unpack_weights(const sbnn_packed* p, float* W, uint8
                 for (int r = 0; r < G; ++r) {
                     int64_t o = ((int64_t)g * G + r) * row + (int64_t)t * p->Cin + c;
                     if (W) W[o] = v[t * G + r];
-                    if (mask) mask[o] = 1;
+                    if (mask) mask[o] = p->tap_mask.empty() ? 1 : (uint8_t)((p->tap_mask[u] >> t) & 1u);
                 }
         }
     return SBNN_OK;

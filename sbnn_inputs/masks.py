@@ -72,3 +72,22 @@ def expand_mask(unit_mask: np.ndarray, g: int, kh: int, kw: int) -> np.ndarray:
     ngroups, cin = unit_mask.shape
     m = np.broadcast_to(unit_mask[:, None, None, None, :], (ngroups, g, kh, kw, cin))
     return np.ascontiguousarray(m.reshape(ngroups * g, kh, kw, cin)).astype(np.uint8)
+
+
+def tap_pattern_mask(seed: int, stream: int, unit_mask: np.ndarray, g: int, kept_taps: int = 4) -> np.ndarray:
+    """3x3 kernel patterns on top of a unit mask: every kept unit keeps the centre tap and `kept_taps - 1` of the
+    other eight (those with the largest random keys), the same pattern for the g filters of the group.
+
+    With kept_taps = 4 these are the C(8,3) = 56 four-entry patterns of pattern-based pruning.  Returns a uint8
+    mask of shape [ngroups*g][3][3][Cin].
+    """
+    if not 1 <= kept_taps <= 9:
+        raise ValueError("kept_taps must be in [1, 9]")
+    ngroups, cin = unit_mask.shape
+    keys = u64_stream(seed, stream, ngroups * cin * 8).reshape(ngroups, cin, 8)
+    others = _ranks(keys) >= 8 - (kept_taps - 1)                      # [ngroups][cin][8]: taps 0-3 and 5-8
+    taps = np.ones((ngroups, cin, 9), dtype=bool)
+    taps[:, :, [0, 1, 2, 3, 5, 6, 7, 8]] = others
+    taps &= unit_mask[:, :, None]
+    m = np.broadcast_to(taps.transpose(0, 2, 1).reshape(ngroups, 1, 3, 3, cin), (ngroups, g, 3, 3, cin))
+    return np.ascontiguousarray(m.reshape(ngroups * g, 3, 3, cin)).astype(np.uint8)

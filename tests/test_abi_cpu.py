@@ -10,7 +10,7 @@ import pytest
 import paper_2310_19509_b200 as sbnn
 from paper_2310_19509_b200 import build as sbnn_build
 from oracle import reference as R
-from sbnn_inputs import expand_mask, group_mask_balanced, group_mask_layer_global
+from sbnn_inputs import expand_mask, group_mask_balanced, group_mask_layer_global, tap_pattern_mask
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -56,6 +56,43 @@ def test_pack_is_bit_identical_to_oracle_pack(k, g, cin, cout, mode):
     w2, m2 = p.unpack()
     assert np.array_equal(m2, m) and (w2.tobytes() == np.where(m != 0, w, np.float32(0)).tobytes())
     p.free()
+
+
+@pytest.mark.parametrize("g,cin,cout,kept_taps", [(4, 16, 32, 4), (2, 8, 8, 4), (1, 6, 5, 6), (8, 8, 16, 1)])
+def test_pattern_pack_is_bit_identical_to_oracle_pack(g, cin, cout, kept_taps):
+    """3x3 kernels pruned tap by tap (one pattern per group and input channel): kept taps, zeros elsewhere, and the
+    tap masks must equal the oracle's own packing; unpacking returns the mask exactly."""
+    rng = np.random.default_rng(17)
+    w = rng.standard_normal((cout, 3, 3, cin)).astype(np.float32)
+    ng = cout // g
+    um = group_mask_balanced(2, 3, ng, cin, 50)
+    m = tap_pattern_mask(2, 19, um, g, kept_taps)
+    assert m.reshape(ng, g, 9, cin).sum(axis=2).max() == kept_taps and m[:, 1, 1, :].sum() == um.sum() * g
+    p = sbnn.pack_weights(w, m, None, g, tap_patterns=True)
+    v = p.view()
+    gp, idx, val, tm = R.pack_pattern(w, m, g)
+    assert np.array_equal(v["group_ptr"], gp) and np.array_equal(v["idx"], idx)
+    assert v["val"].tobytes() == val.tobytes()
+    assert v["tap_mask"].dtype == np.uint16 and np.array_equal(v["tap_mask"], tm)
+    assert all(bin(int(t)).count("1") == kept_taps and (int(t) >> 4) & 1 for t in tm)
+    w2, m2 = p.unpack()
+    assert np.array_equal(m2, m) and (w2.tobytes() == np.where(m != 0, w, np.float32(0)).tobytes())
+    p.free()
+    # the connectivity-only packer refuses such a mask, and a plain unit mask packs the same either way
+    with pytest.raises(sbnn.SbnnError) as e:
+        sbnn.pack_weights(w, m, None, g)
+    assert e.value.code == 4
+    if g > 1:
+        bad = m.copy()
+        c0 = int(np.flatnonzero(um[0])[0])
+        bad[1, 0, 0, c0] ^= 1                      # one filter of the group deviates from the shared pattern
+        with pytest.raises(sbnn.SbnnError) as e:
+            sbnn.pack_weights(w, bad, None, g, tap_patterns=True)
+        assert e.value.code == 4
+    mu = expand_mask(um, g, 3, 3)
+    a, b = sbnn.pack_weights(w, mu, None, g).view(), sbnn.pack_weights(w, mu, None, g, tap_patterns=True).view()
+    assert a["val"].tobytes() == b["val"].tobytes() and np.array_equal(a["idx"], b["idx"]) and a["tap_mask"] is None
+    assert np.all(b["tap_mask"] == 0x1FF)
 
 
 def test_pack_edge_cases():

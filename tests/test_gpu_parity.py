@@ -219,6 +219,24 @@ def test_3x3_shapes_and_groups(g, hw):
         assert_within(y, ref, s, what=f"3x3 G={g} {hw} relu={relu}")
 
 
+@pytest.mark.parametrize("g,kept_taps", [(4, 4), (2, 4), (8, 6), (1, 1)])
+def test_3x3_kernel_patterns(g, kept_taps):
+    """Kernels pruned tap by tap (centre + kept_taps - 1 others, one pattern per group and input channel, packed by
+    sbnn_pack_weights_pattern) on top of 50 % removed kernels: same result as the oracle's masked dense convolution."""
+    from sbnn_inputs import tap_pattern_mask, group_mask_balanced
+    d = WL.single_conv_inputs(2, 9, 28, 24, 32, 3, g, 50, seed=14, w_sigma=0.1)
+    um = group_mask_balanced(14, 3, 32 // g, 24, 50)
+    m = tap_pattern_mask(14, 19, um, g, kept_taps)
+    p = sbnn.pack_weights(d["w"], m, d["bias"], g, tap_patterns=True)
+    n, h, w, _ = d["x"].shape
+    yd = torch.full((n, h, w, 32), float("nan"), device="cuda")
+    sbnn.conv3x3_gs(p, dev(d["x"]), yd, n, h, w, sbnn.SBNN_RELU)
+    sbnn.get_async_status()
+    ref, s = R.conv2d(d["x"], d["w"], m, d["bias"], relu=True)
+    assert_within(yd.cpu().numpy(), ref, s, what=f"3x3 patterns G={g} taps={kept_taps}")
+    p.free()
+
+
 def test_3x3_dense_and_empty_masks():
     for sp in (0, 100):
         d = WL.single_conv_inputs(1, 8, 8, 8, 8, 3, 4, sp, seed=6)
@@ -228,8 +246,8 @@ def test_3x3_dense_and_empty_masks():
 
 
 CM_CFGS = {1: [(8, 4, 8, 32)], 2: [(8, 2, 8, 32)],
-           4: [(8, 1, 16, 32), (8, 2, 8, 32), (4, 1, 8, 32)],
-           8: [(8, 1, 8, 32), (4, 1, 16, 32)], 16: [(4, 1, 8, 32)]}
+           4: [(8, 1, 16, 32), (8, 2, 8, 32), (8, 2, 11, 32), (8, 2, 12, 32), (4, 1, 8, 32)],
+           8: [(8, 1, 8, 32), (8, 1, 12, 32), (4, 1, 16, 32)], 16: [(4, 1, 8, 32)]}
 
 
 def run_cm(d, flags, tile, out_cm):
