@@ -318,6 +318,69 @@ dwconv3x3_cm_col7_kernel(const float* __restrict__ w, const float* __restrict__ 
     }
 }
 
+// 14 x 14 maps, stride 1: seven consecutive lanes own the seven column pairs of a row strip (7 output rows of one
+// channel), so a lane needs one 8-byte load per input row and takes the columns left and right of its pair from
+// its neighbours by shuffle: 9 load requests for 14 outputs.  (With one scalar load per tap the kernel above
+// was limited by the number of load requests in flight, not by bytes.)  A warp holds 4 such strips in 28 lanes;
+// lanes 28-31 only take part in the shuffles.  A CTA of 4 warps covers 8 channels x 2 strips.
+template <int NI>
+__global__ void __launch_bounds__(128)
+dwconv3x3_cm_w14_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
+                        float* __restrict__ y, int ldy, int N, int C, int relu) {
+    constexpr int W = 14, H = 14;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int grp = lane / 7, j = lane - grp * 7;                  // strip within the warp, column pair
+    const int gidx = warp * 4 + (grp & 3);
+    const int cl = gidx >> 1, vs = gidx & 1;
+    const int c0 = blockIdx.y * 8 + cl;
+    const bool live = grp < 4 && c0 < C;
+    const int c = c0 < C ? c0 : C - 1;
+    const int oy0 = vs * 7, n0 = blockIdx.x * NI;
+    float wk[9];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);
+    const float bias = b ? __ldg(b + c) : 0.0f;
+    const float* pc = x + (size_t)c * ldx + (size_t)n0 * H * W + (oy0 - 1) * W + 2 * j;   // input row oy0 - 1, own pair
+    float* yc = y + (size_t)c * ldy + (size_t)n0 * H * W + oy0 * W + 2 * j;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        if (n0 + i >= N) break;                                    // uniform over the CTA
+        float2 v[9];
+#pragma unroll
+        for (int r = 0; r < 9; ++r) {                              // input rows oy0-1 .. oy0+7; row -1 and row 14 are padding
+            const bool rowok = (r > 0 || vs == 1) && (r < 8 || vs == 0);
+            v[r] = rowok ? __ldg(reinterpret_cast<const float2*>(pc + r * W)) : make_float2(0.f, 0.f);
+        }
+        float acc[7][2];
+#pragma unroll
+        for (int o = 0; o < 7; ++o) acc[o][0] = acc[o][1] = bias;
+#pragma unroll
+        for (int r = 0; r < 9; ++r) {
+            float L = __shfl_up_sync(0xffffffffu, v[r].y, 1), R = __shfl_down_sync(0xffffffffu, v[r].x, 1);
+            if (j == 0) L = 0.0f;
+            if (j == 6) R = 0.0f;
+#pragma unroll
+            for (int kh = 0; kh < 3; ++kh) {
+                const int o = r - kh;                              // output row fed through tap row kh
+                if (o >= 0 && o < 7) {
+                    acc[o][0] = fmaf(v[r].y, wk[kh * 3 + 2], fmaf(v[r].x, wk[kh * 3 + 1], fmaf(L, wk[kh * 3], acc[o][0])));
+                    acc[o][1] = fmaf(R, wk[kh * 3 + 2], fmaf(v[r].y, wk[kh * 3 + 1], fmaf(v[r].x, wk[kh * 3], acc[o][1])));
+                }
+            }
+        }
+        if (live) {
+#pragma unroll
+            for (int o = 0; o < 7; ++o) {
+                float2 out = make_float2(acc[o][0], acc[o][1]);
+                if (relu) out = make_float2(fmaxf(out.x, 0.f), fmaxf(out.y, 0.f));
+                *reinterpret_cast<float2*>(yc + o * W) = out;
+            }
+        }
+        pc += H * W;
+        yc += H * W;
+    }
+}
+
 // ---- first layer: NHWC image with Cin <= 4 in, channel-major out --------------------------------
 // One thread: 4 consecutive output columns of one row x 8 output channels; consecutive lanes take
 // consecutive column strips, so each channel's stores are contiguous across the warp.
@@ -538,7 +601,11 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
         dwconv3x3_cm_col7_kernel<NI, WT_><<<g7, 128, 0, st>>>(w, b, x, ldx, y, ldy, N, H, C, relu);            \
     }
         if (stride == 1) {
-            if (W == 14 && H % 7 == 0) SBNN_DW_C7(14)
+            if (W == 14 && H == 14 && ldx % 2 == 0 && ldy % 2 == 0) {
+                constexpr int NI2 = 2;
+                dim3 g14((unsigned)((N + NI2 - 1) / NI2), (C + 7) / 8);
+                dwconv3x3_cm_w14_kernel<NI2><<<g14, 128, 0, st>>>(w, b, x, ldx, y, ldy, N, C, relu);
+            } else if (W == 14 && H % 7 == 0) SBNN_DW_C7(14)
             else if (W == 7 && H % 7 == 0) SBNN_DW_C7(7)
             else SBNN_DW_PX(1, 0);
         } else {
