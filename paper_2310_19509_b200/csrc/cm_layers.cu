@@ -538,18 +538,37 @@ conv3x3_thin_cm32_kernel(const float* __restrict__ w, const float* __restrict__ 
 }
 
 // ---- global average pool: channel-major in ([C][ld], pixel index n*HW + p), channel-major [C][ldy] out --
-// One warp per (channel, image): the HW values are contiguous; lanes stride over them and reduce.
+// Eight lanes per (channel, image): the HW values are contiguous; the lanes stride over them (all loads issued
+// before the adds) and reduce by shuffle.  (A whole warp per pair left most lanes with two loads and five
+// shuffle steps for 49 values.)
 __global__ void __launch_bounds__(256)
 avgpool_cm_kernel(const float* __restrict__ x, int ldx, float* __restrict__ y, int ldy, int N, int HW, int C) {
-    const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (wid >= N * C) return;
-    const int n = wid % N, c = wid / N;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int sub = threadIdx.x & 7;
+    const long long pair0 = t >> 3, pairs = (long long)N * C;
+    const bool live = pair0 < pairs;
+    const long long pair = live ? pair0 : pairs - 1;               // every lane stays for the shuffles
+    const int n = (int)(pair % N), c = (int)(pair / N);
     const float* p = x + (size_t)c * ldx + (size_t)n * HW;
     float s = 0.f;
-    for (int i = lane; i < HW; i += 32) s += __ldg(p + i);
+    int i = sub;
+    for (; i + 56 < HW; i += 64) {                                 // 8 loads in flight per lane
+        float v[8];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (lane == 0) y[(size_t)c * ldy + n] = s * (1.0f / (float)HW);
+        for (int k = 0; k < 8; ++k) v[k] = __ldg(p + i + 8 * k);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s += v[k];
+    }
+    {
+        float v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = (i + 8 * k < HW) ? __ldg(p + i + 8 * k) : 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s += v[k];
+    }
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (live && sub == 0) y[(size_t)c * ldy + n] = s * (1.0f / (float)HW);
 }
 
 }  // namespace
@@ -650,7 +669,7 @@ sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* 
 }
 
 sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int ldy, int N, int HW, int C, cudaStream_t st) {
-    const long long threads = (long long)N * C * 32;
+    const long long threads = (long long)N * C * 8;
     avgpool_cm_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(x, ldx, y, ldy, N, HW, C);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;

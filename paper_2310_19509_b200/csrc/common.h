@@ -105,6 +105,9 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
 sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* x, float* y, int ldy, int N, int H, int W,
                                    int Cin, int Cout, int stride, int relu, cudaStream_t st);
 sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int ldy, int N, int HW, int C, cudaStream_t st);
+// conv1x1_small.cu: kernel for launches with few pixels; reads the canonical packed arrays (no private layout)
+sbnn_status conv1x1_small(const sbnn_packed* p, const float* x, int ldx, float* y, int ldy, int M, int relu, bool out_cm,
+                          cudaStream_t st);
 // conv1x1_bf16.cu
 sbnn_status conv1x1_bf16(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st);
 void free_stream_bf16(sbnn_packed* p);

@@ -614,6 +614,13 @@ TileCfg default_cfg_cm(const sbnn_packed* p, long long M) {
     }
 }
 
+// True when the pipelined kernel would get fewer tiles than half the SMs: such launches go to the few-pixel kernel.
+bool few_tiles(const sbnn_packed* p, long long M) {
+    const TileCfg c = default_cfg_cm(p, 0);
+    const long long tiles = ((M + c.TM() - 1) / c.TM()) * ((p->ngroups + c.GT() - 1) / c.GT());
+    return 2 * tiles < sm_count();
+}
+
 // Per-device scratch for the channel-major copy of X made on behalf of NHWC callers.  Grows on demand
 // (synchronously) and is kept until the process exits.
 struct Workspace {
@@ -729,6 +736,8 @@ extern "C" sbnn_status sbnn_conv1x1_gs_cm(const sbnn_packed* w, const float* xt_
     if (M == 0) return SBNN_OK;
     sbnn_status st = check_device();
     if (st != SBNN_OK) return st;
+    if (!(P | GPW | NW | KC) && few_tiles(w, M))
+        return conv1x1_small(w, xt_dev, ldx, y_dev, ldy, M, flags & SBNN_RELU, out_cm, static_cast<cudaStream_t>(cuda_stream));
     const TileCfg c = (P | GPW | NW | KC) ? TileCfg{P, GPW, NW, KC} : default_cfg_cm(w, M);
     return dispatch_cm(w, c, xt_dev, ldx, y_dev, ldy, M, flags & SBNN_RELU, out_cm, static_cast<cudaStream_t>(cuda_stream));
 }

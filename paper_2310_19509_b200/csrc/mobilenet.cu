@@ -43,13 +43,6 @@ const LayerShape* layer_table() {
 
 inline int round4(long long v) { return (int)((v + 3) / 4 * 4); }
 
-// Tile of the channel-major 1x1 kernel used for the classifier (0s = the layer's default).
-inline void fc_tile(int G, int* P, int* GPW, int* NW, int* KC) {
-    *P = *GPW = *NW = *KC = 0;
-    if (G == 4 || G == 16) { *P = 4; *GPW = 1; *NW = 8; *KC = 32; }
-    if (G == 8) { *P = 4; *GPW = 1; *NW = 16; *KC = 32; }
-}
-
 }  // namespace
 }  // namespace sbnn
 
@@ -108,11 +101,7 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
         if ((st = prepare_default_cm(pw[i], (long long)hw * hw)) != SBNN_OK) return st;   // and the batch-1 choice
     }
     if (fc->device < 0) return fail(SBNN_ERR_CUDA, "the classifier was packed without a CUDA device");
-    {
-        int P, GPW, NW, KC;
-        fc_tile(fc->G, &P, &GPW, &NW, &KC);
-        if ((st = P ? prepare_cm(fc, P, GPW, NW, KC) : prepare_default_cm(fc)) != SBNN_OK) return st;
-    }
+    if ((st = prepare_default_cm(fc, max_batch)) != SBNN_OK) return st;
     sbnn_mbv1* n = new (std::nothrow) sbnn_mbv1;
     if (!n) return fail(SBNN_ERR_ALLOC, "out of host memory");
     for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
@@ -152,10 +141,8 @@ sbnn_status run_cm(sbnn_mbv1* net, int layer, const float* in, float* out, int N
         case 1: return launch_dwconv3x3_cm(net->dw_w[blk], net->dw_b[blk], in, ld_in, out, ld_out, N, L.hin, L.hin, L.cin, L.stride, 1, st);
         case 2: return sbnn_conv1x1_gs_cm(net->pw[blk], in, ld_in, out, ld_out, N * L.hin * L.hin, SBNN_RELU | SBNN_OUT_CM, 0, 0, 0, 0, stream);
         case 3: return launch_avgpool_cm(in, ld_in, out, round4(N), N, L.hin * L.hin, L.cin, st);
-        default: {   // classifier: pooled features [1024][ld] in, logits [N][1000] out; few pixels, so a narrow tile
-            int P, GPW, NW, KC;
-            fc_tile(net->fc->G, &P, &GPW, &NW, &KC);
-            return sbnn_conv1x1_gs_cm(net->fc, in, round4(N), out, L.cout, N, 0, P, GPW, NW, KC, stream);
+        default: {   // classifier: pooled features [1024][ld] in, logits [N][1000] out (few pixels: the entry point picks the kernel)
+            return sbnn_conv1x1_gs_cm(net->fc, in, round4(N), out, L.cout, N, 0, 0, 0, 0, 0, stream);
         }
     }
 }

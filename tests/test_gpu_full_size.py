@@ -71,14 +71,23 @@ def test_mobilenet_batch64_matches_oracle_on_two_images_and_is_batch_invariant()
     sbnn.get_async_status()
     y = logits.cpu().numpy().astype(np.float64)
     assert np.all(np.isfinite(y))
+    refs = {}
     for img in (0, 63):                         # the oracle's chain with its propagated error bound
         outs = R.mobilenet_v1_forward(x[img:img + 1], layers)
         ref, e = outs[-1]["ref"].reshape(-1), outs[-1]["E"].reshape(-1)
+        refs[img] = (ref, e)
         assert np.all(np.abs(y[img] - ref) <= e), f"image {img}: worst ratio {np.max(np.abs(y[img] - ref) / e)}"
-    # an image's logits do not depend on its position in the batch or on the batch size
+    # an image's logits do not depend on its position in the batch (bit for bit: same kernels, same order of sums)
+    flipped = torch.full((64, 1000), float("nan"), device="cuda")
+    net.forward(dev(np.ascontiguousarray(x[::-1])), flipped, 64)
+    sbnn.get_async_status()
+    assert torch.equal(flipped.flip(0), logits)
+    # nor, within the oracle's bound, on the batch size (a batch of one runs the few-pixel kernels, which sum in
+    # another order)
     one = torch.full((1, 1000), float("nan"), device="cuda")
-    for img in (0, 17, 63):
+    for img in (0, 63):
         net.forward(dev(x[img:img + 1]), one, 1)
         sbnn.get_async_status()
-        assert torch.equal(one[0], logits[img])
+        ref, e = refs[img]
+        assert np.all(np.abs(one[0].cpu().numpy().astype(np.float64) - ref) <= e)
     net.free()

@@ -176,12 +176,15 @@ def test_mobilenet_v1_batch1_layer_isolated_and_end_to_end(sparsity):
     y = logits.cpu().numpy().astype(np.float64).reshape(outs[-1]["ref"].shape)
     err = np.abs(y - outs[-1]["ref"])
     assert np.all(err <= outs[-1]["E"]), f"worst ratio {np.max(err / outs[-1]['E'])}"
-    # two images in one call give the single-image result twice
+    # two copies of the image in one call give the same logits twice, bit for bit, and the single-image result
+    # within the bound (the kernel picked for a layer, hence the order of its sums, depends on the pixel count)
     x2 = np.concatenate([x, x])
     l2 = torch.full((2, 1000), float("nan"), device="cuda")
     net.forward(dev(x2), l2, 2)
     sbnn.get_async_status()
-    assert torch.equal(l2[0], l2[1]) and torch.equal(l2[0], logits[0])
+    assert torch.equal(l2[0], l2[1])
+    err2 = np.abs(l2[0].cpu().numpy().astype(np.float64).reshape(outs[-1]["ref"].shape) - outs[-1]["ref"])
+    assert np.all(err2 <= outs[-1]["E"])
     net.free()
 
 
