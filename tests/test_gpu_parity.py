@@ -297,6 +297,19 @@ def test_channel_major_kernel_instances(g):
             assert_within(y, ref, s, what=f"cm G={g} cfg={cfg} relu={relu} out_cm={out_cm}")
 
 
+@pytest.mark.parametrize("g", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("cin,sp", [(40, 50), (160, 50), (320, 40), (1024, 50)])
+def test_few_pixel_kernel(g, cin, sp):
+    """Launches with few pixels take the kernel that gives a CTA 32 pixels of one group and splits the group's list
+    over 1, 2, 4 or 8 warps (by list length): ragged pixel count, variable list lengths (layer-global masks, empty
+    quarters), both output layouts."""
+    d = WL.single_conv_inputs(1, 3, 37, cin, 48, 1, g, sp, seed=21, mask_mode="layer_global")
+    for relu, out_cm in ((True, False), (False, True)):
+        y = run_cm(d, sbnn.SBNN_RELU if relu else 0, (0, 0, 0, 0), out_cm)
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
+        assert_within(y, ref, s, what=f"few-pixel G={g} cin={cin} relu={relu} out_cm={out_cm}")
+
+
 def test_channel_major_kernel_edge_cases():
     for sp in (0, 100):
         d = WL.single_conv_inputs(1, 3, 5, 40, 24, 1, 4, sp, seed=10)
