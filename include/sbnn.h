@@ -160,7 +160,10 @@ SBNN_API sbnn_status sbnn_conv1x1_gs_tuned(const sbnn_packed* w, const float* x_
  * filled by bulk asynchronous copies, which is the fast path for layers bound by arithmetic.
  *   output: y_dev [M][ldy] (pixel-major rows of ldy >= Cout floats), or, with SBNN_OUT_CM, [Cout][ldy]
  *   with ldy >= M; ldy a multiple of 4 in both cases.
- *   P, GPW, NW, KC: tile shape as in sbnn_conv1x1_gs_tuned, or all 0 for the default of the layer.
+ *   P, GPW, NW, KC: tile shape as in sbnn_conv1x1_gs_tuned, or all 0 to let the library choose: the tile
+ *   shape whose tiles fill the SMs best for this M, or, when M is so small that even that leaves most SMs
+ *   idle (the classifier, batch-1 layers), a kernel that splits the work by 32 pixels x one group instead.
+ *   The order of the sums, hence the last bits of the result, can therefore depend on M.
  * sbnn_conv1x1_gs itself takes this path for wide layers (Cin >= 128, M >= 2048): it first copies X
  * into a channel-major scratch buffer kept per device, which it allocates or grows (synchronously) the
  * first time a size is seen.
