@@ -537,6 +537,85 @@ conv3x3_thin_cm32_kernel(const float* __restrict__ w, const float* __restrict__ 
     }
 }
 
+// The network's first layer proper (stride 2, 3 input channels, W a multiple of 4): the 5 input columns x 3
+// channels a thread needs from one image row are 15 consecutive floats that start one float after a 16-byte
+// boundary, so four aligned 16-byte loads per row fetch them, and all twelve are issued before the first FMA
+// (the generic kernel above issues 45 scalar loads in nine dependent batches).  Otherwise as above: 2 output
+// columns x 32 output channels per thread, packed FMAs over channel pairs, weights broadcast from shared memory.
+__global__ void __launch_bounds__(128)
+conv3x3_first_s2c3_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x,
+                          float* __restrict__ y, int ldy, int N, int H, int W, int Cout, int Ho, int Wo, int relu) {
+    constexpr int Cin = 3;
+    extern __shared__ __align__(16) float ws[];   // [9][3][32] of this CTA's channel group
+    const int cg = blockIdx.y;
+    for (int i = threadIdx.x; i < 9 * Cin * 32; i += blockDim.x) {
+        const int o = i & 31, tc = i >> 5;
+        ws[i] = w[(size_t)(cg * 32 + o) * 9 * Cin + tc];
+    }
+    __syncthreads();
+    const int strips = Wo >> 1;
+    const long long total = (long long)N * Ho * strips;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= total) return;
+    const int sx = (int)(t % strips);
+    const long long f = t / strips;
+    const int oy = (int)(f % Ho);
+    const int n = (int)(f / Ho);
+    float v[3][16];                                                // per row: floats 12*sx - 4 .. 12*sx + 11
+#pragma unroll
+    for (int kh = 0; kh < 3; ++kh) {
+        const int iy = oy * 2 + kh - 1;
+        const bool rowok = iy >= 0 && iy < H;
+        const float4* row = reinterpret_cast<const float4*>(x + ((size_t)n * H + (rowok ? iy : 0)) * W * Cin) + 3 * sx;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const bool ok = rowok && (q > 0 || sx > 0);            // the piece left of the row holds only the padding column
+            const float4 t4 = ok ? __ldg(row + q - 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[kh][4 * q] = t4.x; v[kh][4 * q + 1] = t4.y; v[kh][4 * q + 2] = t4.z; v[kh][4 * q + 3] = t4.w;
+        }
+    }
+    f32x2 acc[2][16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const float b0 = b ? __ldg(b + cg * 32 + 2 * j) : 0.f, b1 = b ? __ldg(b + cg * 32 + 2 * j + 1) : 0.f;
+        acc[0][j] = acc[1][j] = pack2(b0, b1);
+    }
+#pragma unroll
+    for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+        for (int c = 0; c < Cin; ++c) {
+            f32x2 in[5];
+#pragma unroll
+            for (int j = 0; j < 5; ++j) in[j] = dup2(v[kh][1 + 3 * j + c]);   // column 4*sx - 1 + j, channel c
+#pragma unroll
+            for (int kw = 0; kw < 3; ++kw) {
+                const ulonglong2* wp = reinterpret_cast<const ulonglong2*>(ws + ((kh * 3 + kw) * Cin + c) * 32);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const ulonglong2 wv = wp[q];
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        fma2(acc[i][2 * q], in[i * 2 + kw], wv.x);
+                        fma2(acc[i][2 * q + 1], in[i * 2 + kw], wv.y);
+                    }
+                }
+            }
+        }
+    const long long p0 = f * Wo + 2 * sx;                          // even, so the pair of columns is one 8-byte store
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float v0[2], v1[2];
+        unpack2(acc[0][j], v0[0], v0[1]);
+        unpack2(acc[1][j], v1[0], v1[1]);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            float a0 = v0[e], a1 = v1[e];
+            if (relu) { a0 = fmaxf(a0, 0.f); a1 = fmaxf(a1, 0.f); }
+            *reinterpret_cast<float2*>(y + (size_t)(cg * 32 + 2 * j + e) * ldy + p0) = make_float2(a0, a1);
+        }
+    }
+}
+
 // ---- global average pool: channel-major in ([C][ld], pixel index n*HW + p), channel-major [C][ldy] out --
 // Eight lanes per (channel, image): the HW values are contiguous; the lanes stride over them (all loads issued
 // before the adds) and reduce by shuffle.  (A whole warp per pair left most lanes with two loads and five
@@ -648,7 +727,9 @@ sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* 
         if (blocks > 0x7fffffff) return fail(SBNN_ERR_SHAPE, "tensor too large");
         dim3 grid((unsigned)blocks, Cout / 32);
         const size_t smem = sizeof(float) * 9 * Cin * 32;
-        if (stride == 1)
+        if (stride == 2 && Cin == 3 && W % 4 == 0 && H % 2 == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0)
+            conv3x3_first_s2c3_kernel<<<grid, 128, smem, st>>>(w, b, x, y, ldy, N, H, W, Cout, Ho, Wo, relu);
+        else if (stride == 1)
             conv3x3_thin_cm32_kernel<1><<<grid, 128, smem, st>>>(w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu);
         else
             conv3x3_thin_cm32_kernel<2><<<grid, 128, smem, st>>>(w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu);
