@@ -48,7 +48,10 @@ struct K2 {
     static constexpr int QUAD = 1 + G;                     // 4 row offsets + 4*G weights
     static constexpr int QUAD2 = 1 + 2 * G;                // the same for a unit that feeds two groups
     static constexpr int NQ = KC / 4 + 1;                  // quads of a full list incl. its all-zero end quad
-    static constexpr int WS_U4 = UNION ? HDR + NW * (NQ * QUAD2 + 2 * NQ * QUAD) : HDR + GT * NQ * QUAD;
+    // Largest weight block of a step.  Union lists partition the step's KC channels, and a unit kept by both
+    // groups is the most expensive, so the worst case is all KC channels in the first list and the other two empty
+    // (one all-zero end quad each).
+    static constexpr int WS_U4 = UNION ? HDR + NW * (NQ * QUAD2 + 2 * QUAD) : HDR + GT * NQ * QUAD;
     static constexpr int WS_BYTES = WS_U4 * 16;
     static constexpr size_t SMEM = (size_t)STAGES * (XS_BYTES + WS_BYTES) + 2 * STAGES * 8 + 16;
     static_assert(P % 4 == 0 && KC % 4 == 0, "tile shape");
