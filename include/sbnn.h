@@ -241,6 +241,12 @@ SBNN_API sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, cons
  * conv0 -> 13 x (depthwise 3x3 -> group-sparse 1x1) -> average pool -> classifier.
  *   x_dev [N][224][224][3] fp32 (4-byte aligned is enough), logits_dev [N][1000] fp32.
  * Every conv but the classifier applies ReLU.  No host synchronisation.
+ * The second call with the same (x_dev, logits_dev, N) records the 29 launches into a CUDA graph (captured on a
+ * stream the network owns; nothing of the caller's stream is touched) and from then on such calls launch that
+ * graph on cuda_stream, which shortens the gaps between the kernels; up to 8 triples are kept.  If recording
+ * fails, or if cuda_stream is itself being captured, the launches are issued one by one as on the first call.
+ * Calls on one network are serialised on the host by a lock; the workspaces make concurrent forwards of one
+ * network on different streams invalid in any case.
  */
 SBNN_API sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_dev, float* logits_dev,
                                                int N, void* cuda_stream);

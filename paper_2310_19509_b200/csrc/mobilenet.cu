@@ -56,6 +56,27 @@ struct sbnn_mbv1 {
     int max_batch;
     int device;
     float* ws[2];  // ping-pong activation buffers
+    // Forward calls replay a CUDA graph of the 29 launches once a (x, logits, N) triple has been seen twice:
+    // the first call runs plainly (and builds whatever is built lazily), the second is captured on a private
+    // stream and instantiated, later ones only launch the graph on the caller's stream.
+    struct GraphKey {
+        const float* x;
+        float* y;
+        int n;
+        bool operator<(const GraphKey& o) const {
+            if (x != o.x) return x < o.x;
+            if (y != o.y) return y < o.y;
+            return n < o.n;
+        }
+    };
+    struct GraphEntry {
+        cudaGraphExec_t exec = nullptr;
+        int seen = 0;
+        bool failed = false;
+    };
+    std::mutex mu;
+    std::map<GraphKey, GraphEntry> graphs;
+    cudaStream_t capture_stream = nullptr;
 };
 
 using namespace sbnn;
@@ -112,6 +133,10 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
     n->fc = fc; n->c0_w = conv0_w_dev; n->c0_b = conv0_b_dev; n->max_batch = max_batch;
     n->ws[0] = n->ws[1] = nullptr;
     cudaGetDevice(&n->device);
+    if (cudaStreamCreateWithFlags(&n->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        cudaGetLastError();
+        n->capture_stream = nullptr;   // forward then always launches plainly
+    }
     // Largest activation: pw1's output, 112*112*64 floats per image (+ row padding of the layout).
     const size_t bytes = ((size_t)max_batch * 112 * 112 * 64 + 4 * 1024) * sizeof(float);
     for (int i = 0; i < 2; ++i) {
@@ -184,13 +209,9 @@ extern "C" sbnn_status sbnn_mobilenet_v1_run_layer_cm(sbnn_mbv1* net, int layer,
     return run_cm(net, layer, in, outp, N, stream);
 }
 
-extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_dev, float* logits_dev, int N,
-                                                 void* stream) {
-    clear_error();
-    if (!net || !x_dev || !logits_dev) return fail(SBNN_ERR_NULL, "net, x_dev and logits_dev must not be NULL");
-    if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
-    if (!aligned16(logits_dev)) return fail(SBNN_ERR_ALIGN, "logits_dev must be 16-byte aligned");
-    if (N == 0) return SBNN_OK;
+namespace {
+
+sbnn_status forward_plain(sbnn_mbv1* net, const float* x_dev, float* logits_dev, int N, void* stream) {
     const float* cur = x_dev;
     for (int l = 0; l < SBNN_MBV1_NUM_LAYERS; ++l) {
         float* dst = (l == SBNN_MBV1_NUM_LAYERS - 1) ? logits_dev : net->ws[l & 1];
@@ -201,9 +222,64 @@ extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_
     return SBNN_OK;
 }
 
+void drop_graphs(sbnn_mbv1* net) {
+    for (auto& kv : net->graphs)
+        if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+    net->graphs.clear();
+}
+
+constexpr size_t kMaxGraphs = 8;
+
+}  // namespace
+
+extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_dev, float* logits_dev, int N,
+                                                 void* stream) {
+    clear_error();
+    if (!net || !x_dev || !logits_dev) return fail(SBNN_ERR_NULL, "net, x_dev and logits_dev must not be NULL");
+    if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
+    if (!aligned16(logits_dev)) return fail(SBNN_ERR_ALIGN, "logits_dev must be 16-byte aligned");
+    if (N == 0) return SBNN_OK;
+    cudaStream_t user = static_cast<cudaStream_t>(stream);
+    // A caller that is itself capturing gets the plain launches recorded into its own graph.
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(user, &cs) != cudaSuccess) cudaGetLastError();
+    if (cs != cudaStreamCaptureStatusNone) return forward_plain(net, x_dev, logits_dev, N, stream);
+
+    std::lock_guard<std::mutex> lk(net->mu);
+    if (net->graphs.size() >= kMaxGraphs && !net->graphs.count({x_dev, logits_dev, N})) drop_graphs(net);
+    sbnn_mbv1::GraphEntry& e = net->graphs[{x_dev, logits_dev, N}];
+    if (e.exec) {
+        SBNN_CUDA_TRY(cudaGraphLaunch(e.exec, user));
+        return SBNN_OK;
+    }
+    if (e.failed || e.seen++ == 0 || !net->capture_stream) return forward_plain(net, x_dev, logits_dev, N, stream);
+    // second call with these buffers: record the launches on the private stream (nothing runs there)
+    cudaGraph_t graph = nullptr;
+    sbnn_status r = SBNN_ERR_CUDA;
+    if (cudaStreamBeginCapture(net->capture_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+        r = forward_plain(net, x_dev, logits_dev, N, net->capture_stream);
+        if (cudaStreamEndCapture(net->capture_stream, &graph) != cudaSuccess || !graph) r = SBNN_ERR_CUDA;
+    }
+    if (r == SBNN_OK && cudaGraphInstantiate(&e.exec, graph, 0) != cudaSuccess) {
+        e.exec = nullptr;
+        r = SBNN_ERR_CUDA;
+    }
+    if (graph) cudaGraphDestroy(graph);
+    if (r != SBNN_OK) {          // no graph for these buffers: keep launching plainly
+        cudaGetLastError();
+        clear_error();
+        e.failed = true;
+        return forward_plain(net, x_dev, logits_dev, N, stream);
+    }
+    SBNN_CUDA_TRY(cudaGraphLaunch(e.exec, user));
+    return SBNN_OK;
+}
+
 extern "C" sbnn_status sbnn_mobilenet_v1_free(sbnn_mbv1* net) {
     clear_error();
     if (!net) return SBNN_OK;
+    drop_graphs(net);
+    if (net->capture_stream) cudaStreamDestroy(net->capture_stream);
     cudaFree(net->ws[0]);
     cudaFree(net->ws[1]);
     cudaGetLastError();

@@ -188,6 +188,41 @@ def test_mobilenet_v1_batch1_layer_isolated_and_end_to_end(sparsity):
     net.free()
 
 
+def test_forward_graph_replay_matches_plain_launches():
+    """forward records a CUDA graph on its second call with the same buffers and replays it afterwards: replays
+    must give, bit for bit, what the plain first call gave, follow the current contents of the input buffer, and a
+    different batch size on the same buffers must not reuse the recording."""
+    x, layers = mobilenet_v1_inputs(2, 50, 4, seed=5)
+    net = build_net(layers, 2)
+    xd = dev(x)
+    logits = torch.full((2, 1000), float("nan"), device="cuda")
+    net.forward(xd, logits, 2)                       # plain
+    sbnn.get_async_status()
+    first = logits.clone()
+    for _ in range(3):                               # recorded, then replayed twice
+        logits.fill_(float("nan"))
+        net.forward(xd, logits, 2)
+        sbnn.get_async_status()
+        assert torch.equal(logits, first)
+    xd.copy_(xd.flip(0))                             # same buffer, other contents: the two images swapped
+    net.forward(xd, logits, 2)
+    sbnn.get_async_status()
+    assert torch.equal(logits, first.flip(0))
+    one = torch.full((2, 1000), float("nan"), device="cuda")
+    for _ in range(3):                               # N = 1 on the same input buffer: its own recording
+        net.forward(xd, one, 1)
+        sbnn.get_async_status()
+        assert bool(torch.isfinite(one[0]).all()) and bool(torch.isnan(one[1]).all())
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):                    # replay on another stream than the one it was first used on
+        side.wait_stream(torch.cuda.current_stream())
+        logits.fill_(float("nan"))
+        net.forward(xd, logits, 2, stream=side)
+        side.synchronize()
+    assert torch.equal(logits, first.flip(0))
+    net.free()
+
+
 def run_3x3(d, flags=sbnn.SBNN_RELU):
     x = d["x"]
     n, h, w, cin = x.shape
