@@ -201,6 +201,28 @@ SBNN_API sbnn_status sbnn_dwconv3x3(const float* w_dev, const float* b_dev, cons
                                     int N, int H, int W, int C, int stride, int flags, void* cuda_stream);
 
 /*
+ * Depthwise 3x3 with 3:9 kernel patterns (Section 3.2, DwConv3x3; Algorithm 2): in every row of a kernel the
+ * middle weight stays and either the first or the third column is pruned, one pattern per block of go
+ * consecutive channels (the paper's PatternInfo; go = 16, or 8 or 4 for channel counts that need it).
+ *
+ * sbnn_pack_dw_pattern (host only): from dense weights W_host [3][3][C] and mask_host [3][3][C] (1 = kept)
+ * writes pattern_host_out [C/go] (bit kh set = the THIRD column of row kh is pruned and the first is kept;
+ * clear = the first is pruned) and w6_host_out [3][2][C] (per row: the surviving side weight, then the
+ * middle weight).  A mask that is not such a pattern, or that differs inside a block, gives
+ * SBNN_ERR_MASK_NOT_GROUP_UNIFORM.  The paper's additional dense ("full-1") pattern is not part of this format:
+ * dense channels go through sbnn_dwconv3x3.
+ *
+ * sbnn_dwconv3x3_pattern: Y as in sbnn_dwconv3x3 with the pruned weights taken as zero; six loads and six
+ * FMAs per output.  w6_dev, b_dev, x_dev, y_dev 16-byte aligned device pointers, pattern_dev a device byte array;
+ * x_dev [N][H][W][C], y_dev [N][Ho][Wo][C]; stride 1 or 2; go in {4, 8, 16}, C a multiple of go.
+ */
+SBNN_API sbnn_status sbnn_pack_dw_pattern(const float* W_host, const uint8_t* mask_host, int C, int go,
+                                          uint8_t* pattern_host_out, float* w6_host_out);
+SBNN_API sbnn_status sbnn_dwconv3x3_pattern(const float* w6_dev, const uint8_t* pattern_dev, int go, const float* b_dev,
+                                            const float* x_dev, float* y_dev, int N, int H, int W, int C, int stride,
+                                            int flags, void* cuda_stream);
+
+/*
  * Dense 3x3, pad 1, stride 1 or 2, for thin inputs (the network's first layer, Cin = 3):
  *   w_dev [Cout][3][3][Cin], b_dev [Cout] or NULL, x_dev [N][H][W][Cin], y_dev [N][Ho][Wo][Cout].
  * Cin <= 4 and Cout a multiple of 8 and <= 64; other shapes return SBNN_ERR_UNSUPPORTED.

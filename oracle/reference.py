@@ -177,6 +177,34 @@ def pack_pattern(w, mask, g):
             np.array(tap_mask, dtype=np.uint16))
 
 
+def pack_dw_pattern(w, mask, go):
+    """Compact form of 3:9 pattern-pruned depthwise weights (Section 3.2, DwConv3x3; Algorithm 2's PatternInfo).
+
+    w, mask: [3][3][C].  In every row the middle weight is kept and exactly one of the two side columns is
+    pruned, identically for the `go` channels of a block.  Returns (pattern uint8 [C/go] with bit kh set iff the
+    third column of row kh is pruned, w6 float32 [3][2][C] = per row the surviving side weight, then the middle).
+    """
+    w = np.asarray(w, dtype=np.float32)
+    mask = np.asarray(mask, dtype=np.uint8)
+    c = w.shape[2]
+    if c % go:
+        raise ValueError("C % go != 0")
+    pattern = np.zeros(c // go, dtype=np.uint8)
+    w6 = np.zeros((3, 2, c), dtype=np.float32)
+    for blk in range(c // go):
+        sl = slice(blk * go, (blk + 1) * go)
+        for kh in range(3):
+            rows = mask[kh, :, sl]                      # [kw][go]
+            if np.any(rows != rows[:, :1]) or rows[1, 0] != 1 or int(rows[0, 0]) + int(rows[2, 0]) != 1:
+                raise MaskNotGroupUniform(f"block {blk} row {kh}")
+            third_pruned = rows[2, 0] == 0
+            if third_pruned:
+                pattern[blk] |= 1 << kh
+            w6[kh, 0, sl] = w[kh, 0 if third_pruned else 2, sl]
+            w6[kh, 1, sl] = w[kh, 1, sl]
+    return pattern, w6
+
+
 def unpack(group_ptr, idx, val, cout, kh, kw, cin, g):
     """Inverse of pack: returns (W (.) M, M)."""
     w = np.zeros((cout, kh, kw, cin), dtype=np.float32)

@@ -19,11 +19,13 @@ from .binding import (  # noqa: F401
     conv3x3_dense,
     conv3x3_gs,
     dwconv3x3,
+    dwconv3x3_pattern,
     get_async_status,
     head_noalloc,
     lib,
     lib_path,
     mobilenet_v1_layer_shape,
+    pack_dw_pattern,
     pack_weights,
     selftest_wait_timeout,
     status_str,

@@ -50,6 +50,8 @@ def lib():
         "sbnn_conv1x1_gs_cm": [P, P, I, P, I, I, I, I, I, I, I, P],
         "sbnn_to_channel_major": [P, P, I, I, I, P],
         "sbnn_dwconv3x3": [P, P, P, P, I, I, I, I, I, I, P],
+        "sbnn_pack_dw_pattern": [P, P, I, I, P, P],
+        "sbnn_dwconv3x3_pattern": [P, P, I, P, P, P, I, I, I, I, I, I, P],
         "sbnn_conv3x3_dense": [P, P, P, P, I, I, I, I, I, I, I, P],
         "sbnn_avgpool": [P, P, I, I, I, P],
         "sbnn_mobilenet_v1_create": [P, P, P, P, P, P, I, P],
@@ -183,6 +185,24 @@ def conv3x3_gs(w: Packed, x, y, n, h, wd, flags=SBNN_RELU, stream=None):
 
 def dwconv3x3(w, b, x, y, n, h, wd, c, stride, flags=SBNN_RELU, stream=None):
     _check(lib().sbnn_dwconv3x3(_ptr(w), _ptr(b), _ptr(x), _ptr(y), n, h, wd, c, stride, flags, _stream(stream)))
+
+
+def pack_dw_pattern(w, mask, go):
+    """Host-side: dense depthwise weights [3][3][C] and a 3:9 pattern mask -> (pattern uint8 [C/go], w6 fp32 [3][2][C])."""
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    if w.ndim != 3 or w.shape[:2] != (3, 3) or mask.shape != w.shape:
+        raise ValueError("w and mask must both be [3][3][C]")
+    c = w.shape[2]
+    pattern = np.zeros(max(c // max(int(go), 1), 1), dtype=np.uint8)
+    w6 = np.zeros((3, 2, c), dtype=np.float32)
+    _check(lib().sbnn_pack_dw_pattern(w.ctypes.data, mask.ctypes.data, c, int(go), pattern.ctypes.data, w6.ctypes.data))
+    return pattern, w6
+
+
+def dwconv3x3_pattern(w6, pattern, go, b, x, y, n, h, wd, c, stride, flags=SBNN_RELU, stream=None):
+    _check(lib().sbnn_dwconv3x3_pattern(_ptr(w6), _ptr(pattern), int(go), _ptr(b), _ptr(x), _ptr(y), n, h, wd, c, stride,
+                                        flags, _stream(stream)))
 
 
 def conv3x3_dense(w, b, x, y, n, h, wd, cin, cout, stride, flags=SBNN_RELU, stream=None):

@@ -5,7 +5,7 @@ arithmetic of the convolution path and imports neither the CUDA library
 nor the CPU oracle, so both can be fed the very same arrays.
 """
 from .rng import uniform01, normal, u64_stream
-from .masks import removed_units, group_mask_balanced, group_mask_layer_global, group_mask_magnitude, expand_mask, tap_pattern_mask
+from .masks import removed_units, group_mask_balanced, group_mask_layer_global, group_mask_magnitude, expand_mask, tap_pattern_mask, dw_pattern_mask
 from .workloads import (
     single_conv_inputs,
     mobilenet_v1_shapes,
@@ -15,6 +15,6 @@ from .workloads import (
 __all__ = [
     "uniform01", "normal", "u64_stream",
     "removed_units", "group_mask_balanced", "group_mask_layer_global",
-    "group_mask_magnitude", "expand_mask", "tap_pattern_mask",
+    "group_mask_magnitude", "expand_mask", "tap_pattern_mask", "dw_pattern_mask",
     "single_conv_inputs", "mobilenet_v1_shapes", "mobilenet_v1_inputs",
 ]

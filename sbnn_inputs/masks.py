@@ -91,3 +91,24 @@ def tap_pattern_mask(seed: int, stream: int, unit_mask: np.ndarray, g: int, kept
     taps &= unit_mask[:, :, None]
     m = np.broadcast_to(taps.transpose(0, 2, 1).reshape(ngroups, 1, 3, 3, cin), (ngroups, g, 3, 3, cin))
     return np.ascontiguousarray(m.reshape(ngroups * g, 3, 3, cin)).astype(np.uint8)
+
+
+def dw_pattern_mask(seed: int, stream: int, c: int, go: int, w: np.ndarray | None = None) -> np.ndarray:
+    """3:9 patterns for depthwise 3x3 weights [3][3][C]: in every kernel row the middle weight stays and either the
+    first or the third column goes, one choice per row and per block of `go` consecutive channels.
+
+    With w given, a block keeps in each row the side whose weights have the larger l1 norm over the block (the
+    pattern that maximises the remaining l1 norm); otherwise the side is drawn at random.  Returns uint8 [3][3][C].
+    """
+    if c % go:
+        raise ValueError("C must be a multiple of go")
+    nblk = c // go
+    if w is None:
+        drop_third = (u64_stream(seed, stream, 3 * nblk).reshape(3, nblk) >> np.uint64(63)).astype(bool)
+    else:
+        l1 = np.abs(np.asarray(w, dtype=np.float64)).reshape(3, 3, nblk, go).sum(axis=3)   # [kh][kw][blk]
+        drop_third = l1[:, 0, :] >= l1[:, 2, :]
+    m = np.ones((3, 3, nblk, go), dtype=np.uint8)
+    m[:, 2][drop_third] = 0
+    m[:, 0][~drop_third] = 0
+    return m.reshape(3, 3, c)

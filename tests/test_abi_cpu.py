@@ -10,7 +10,7 @@ import pytest
 import paper_2310_19509_b200 as sbnn
 from paper_2310_19509_b200 import build as sbnn_build
 from oracle import reference as R
-from sbnn_inputs import expand_mask, group_mask_balanced, group_mask_layer_global, tap_pattern_mask
+from sbnn_inputs import expand_mask, group_mask_balanced, group_mask_layer_global, tap_pattern_mask, dw_pattern_mask
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -93,6 +93,44 @@ def test_pattern_pack_is_bit_identical_to_oracle_pack(g, cin, cout, kept_taps):
     a, b = sbnn.pack_weights(w, mu, None, g).view(), sbnn.pack_weights(w, mu, None, g, tap_patterns=True).view()
     assert a["val"].tobytes() == b["val"].tobytes() and np.array_equal(a["idx"], b["idx"]) and a["tap_mask"] is None
     assert np.all(b["tap_mask"] == 0x1FF)
+
+
+@pytest.mark.parametrize("c,go,by_magnitude", [(64, 16, False), (24, 8, True), (12, 4, False), (160, 16, True)])
+def test_dw_pattern_pack_is_bit_identical_to_oracle_pack(c, go, by_magnitude):
+    """3:9 depthwise patterns: PatternInfo and the six surviving weights per channel equal the oracle's own packing."""
+    rng = np.random.default_rng(23)
+    w = rng.standard_normal((3, 3, c)).astype(np.float32)
+    m = dw_pattern_mask(3, 5, c, go, w if by_magnitude else None)
+    assert np.all(m.sum(axis=(0, 1)) == 6) and np.all(m[:, 1] == 1)
+    if c // go >= 8 and not by_magnitude:
+        assert len({tuple(m[:, :, b * go].reshape(-1)) for b in range(c // go)}) > 1      # blocks differ
+    pat, w6 = sbnn.pack_dw_pattern(w, m, go)
+    rpat, rw6 = R.pack_dw_pattern(w, m, go)
+    assert np.array_equal(pat, rpat) and w6.tobytes() == rw6.tobytes()
+    # what the compact form stands for: the masked dense weights
+    dense = np.zeros_like(w)
+    for b in range(c // go):
+        for kh in range(3):
+            side = 0 if (pat[b] >> kh) & 1 else 2
+            dense[kh, side, b * go:(b + 1) * go] = w6[kh, 0, b * go:(b + 1) * go]
+            dense[kh, 1, b * go:(b + 1) * go] = w6[kh, 1, b * go:(b + 1) * go]
+    assert dense.tobytes() == np.where(m != 0, w, np.float32(0)).tobytes()
+    # not a 3:9 pattern / not uniform inside a block / bad block size
+    for bad in ("middle", "both", "deviate"):
+        mb = m.copy()
+        if bad == "middle":
+            mb[1, 1, 0] = 0
+        elif bad == "both":
+            mb[0, 0, :go] = 1
+            mb[0, 2, :go] = 1
+        else:
+            mb[2, 0, 1], mb[2, 2, 1] = mb[2, 2, 1], mb[2, 0, 1]
+        with pytest.raises(sbnn.SbnnError) as e:
+            sbnn.pack_dw_pattern(w, mb, go)
+        assert e.value.code == 4
+    with pytest.raises(sbnn.SbnnError) as e:
+        sbnn.pack_dw_pattern(w, m, 5)
+    assert e.value.code == 3
 
 
 def test_pack_edge_cases():

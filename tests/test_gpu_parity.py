@@ -123,6 +123,27 @@ def test_depthwise(stride, shape):
     assert_within(yd.cpu().numpy(), ref, s, what=f"dw {shape} s{stride}")
 
 
+@pytest.mark.parametrize("stride", [1, 2])
+@pytest.mark.parametrize("shape,go", [((2, 9, 11, 32), 16), ((1, 14, 14, 48), 8), ((1, 1, 1, 4), 4), ((3, 7, 7, 64), 16)])
+def test_depthwise_3of9_patterns(stride, shape, go):
+    """Depthwise 3x3 with 3:9 kernel patterns (compact weights + PatternInfo through the C interface) against the
+    oracle's dense depthwise convolution on the masked weights."""
+    from sbnn_inputs import dw_pattern_mask
+    n, h, w, c = shape
+    rng = np.random.default_rng(31)
+    x = rng.random((n, h, w, c), dtype=np.float32)
+    wt = rng.standard_normal((3, 3, c)).astype(np.float32)
+    b = rng.standard_normal(c).astype(np.float32)
+    m = dw_pattern_mask(7, 5, c, go)
+    pat, w6 = sbnn.pack_dw_pattern(wt, m, go)
+    ho, wo = (h - 1) // stride + 1, (w - 1) // stride + 1
+    yd = torch.full((n, ho, wo, c), float("nan"), device="cuda")
+    sbnn.dwconv3x3_pattern(dev(w6), torch.from_numpy(pat).cuda(), go, dev(b), dev(x), yd, n, h, w, c, stride)
+    sbnn.get_async_status()
+    ref, s = R.dwconv3x3(x, np.where(m != 0, wt, np.float32(0)), b, stride=stride, relu=True)
+    assert_within(yd.cpu().numpy(), ref, s, what=f"dw 3:9 {shape} go={go} s{stride}")
+
+
 @pytest.mark.parametrize("stride,shape", [(2, (2, 32, 32, 3, 32)), (1, (1, 9, 7, 3, 32)), (2, (1, 15, 17, 4, 8))])
 def test_thin_dense_conv(stride, shape):
     n, h, w, cin, cout = shape
