@@ -490,28 +490,52 @@ int sm_count() {
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-sbnn_status encode_x_map(const float* x, int ldx, int M, int Cin, int box_px, int box_rows, CUtensorMap* out) {
+sbnn_status get_encode(EncodeTiledFn* out) {
     static std::mutex mu;
     static EncodeTiledFn encode = nullptr;
-    {
-        std::lock_guard<std::mutex> lk(mu);
-        if (!encode) {
-            void* fn = nullptr;
-            cudaDriverEntryPointQueryResult q;
-            SBNN_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
-            if (!fn || q != cudaDriverEntryPointSuccess) return fail(SBNN_ERR_CUDA, "driver has no cuTensorMapEncodeTiled");
-            encode = reinterpret_cast<EncodeTiledFn>(fn);
+    std::lock_guard<std::mutex> lk(mu);
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        SBNN_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (!fn || q != cudaDriverEntryPointSuccess) return fail(SBNN_ERR_CUDA, "driver has no cuTensorMapEncodeTiled");
+        encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    *out = encode;
+    return SBNN_OK;
+}
+
+// fp32 tensor of `rank` dimensions (innermost first), tiled copies of `box` elements, zeros outside the tensor.
+sbnn_status encode_generic(void* out, const float* base, int rank, const unsigned long long* dims,
+                           const unsigned long long* strides_bytes, const unsigned* box) {
+    EncodeTiledFn encode = nullptr;
+    sbnn_status r = get_encode(&encode);
+    if (r != SBNN_OK) return r;
+    if (!aligned16(base)) return fail(SBNN_ERR_ALIGN, "tensor base must be 16-byte aligned");
+    cuuint64_t d[5], st[4];
+    cuuint32_t b[5], es[5];
+    for (int i = 0; i < rank; ++i) {
+        d[i] = dims[i];
+        b[i] = box[i];
+        es[i] = 1;
+        if (i + 1 < rank) {
+            st[i] = strides_bytes[i];
+            if (st[i] % 16) return fail(SBNN_ERR_ALIGN, "tensor stride %llu is not a multiple of 16 bytes", (unsigned long long)st[i]);
         }
     }
-    if (!aligned16(x) || ldx % 4) return fail(SBNN_ERR_ALIGN, "channel-major activations need a 16-byte aligned base and ld %% 4 == 0");
-    const cuuint64_t dims[2] = {(cuuint64_t)M, (cuuint64_t)Cin};
-    const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(float)};
-    const cuuint32_t box[2] = {(cuuint32_t)box_px, (cuuint32_t)box_rows}, elem_strides[2] = {1, 1};
-    const CUresult cr = encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(x), dims, strides, box, elem_strides,
-                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (cr != CUDA_SUCCESS) return fail(SBNN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for M=%d Cin=%d ld=%d", (int)cr, M, Cin, ldx);
+    const CUresult cr = encode(static_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank,
+                               const_cast<float*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return fail(SBNN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)cr);
     return SBNN_OK;
+}
+
+sbnn_status encode_x_map(const float* x, int ldx, int M, int Cin, int box_px, int box_rows, CUtensorMap* out) {
+    if (ldx % 4) return fail(SBNN_ERR_ALIGN, "channel-major activations need ld %% 4 == 0");
+    const unsigned long long dims[2] = {(unsigned long long)M, (unsigned long long)Cin};
+    const unsigned long long strides[1] = {(unsigned long long)ldx * sizeof(float)};
+    const unsigned box[2] = {(unsigned)box_px, (unsigned)box_rows};
+    return encode_generic(out, x, 2, dims, strides, box);
 }
 
 template <class C>
@@ -651,6 +675,13 @@ sbnn_status workspace(size_t bytes, float** out) {
 }  // namespace
 
 sbnn_status scratch_workspace(size_t bytes, float** out) { return workspace(bytes, out); }
+
+sbnn_status async_status_word(int** out) { return status_word(out); }
+
+sbnn_status encode_tiled_map(void* out, const float* base, int rank, const unsigned long long* dims,
+                             const unsigned long long* strides_bytes, const unsigned* box) {
+    return encode_generic(out, base, rank, dims, strides_bytes, box);
+}
 
 sbnn_status prepare_default_cm(const sbnn_packed* p, long long M) {
     Stream1x1 s;

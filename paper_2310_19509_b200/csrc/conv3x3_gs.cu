@@ -354,6 +354,177 @@ conv3x3_gs_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y
     }
 }
 
+// ---- channel-major variant with a copy-engine pipeline ------------------------------------------------
+// Same decomposition and inner loop as conv3x3_gs_cm_kernel, but the staging is taken off the compute warps: the
+// planes of X are a 3-D tensor [Cin][N*H][W], and one tiled copy per channel step brings the box
+// (pitch columns from x = -4, R + 2 rows from f0 - 1, KC channels) into a stage; columns and rows outside the
+// tensor arrive as zeros, which is exactly the horizontal padding.  A producer warp issues that copy and the
+// linear copy of the step's weight block onto the stage's "full" mbarrier; the compute warps release a stage
+// through its "empty" mbarrier, so a warp whose groups keep more kernels in one step is not waited for at a
+// CTA-wide barrier (ncu had 19 % of the stall cycles of the two-buffer version there).  Vertical padding between
+// images: rows of a neighbouring image are replaced by a row of zeros kept beside the stages.  Waits are bounded.
+struct Map3 { alignas(64) unsigned char bytes[128]; };
+
+template <class C>
+__global__ void __launch_bounds__(C::NT + 32, 1)
+conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, const float* __restrict__ bias,
+                      const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, Geo3 geo, int relu, int S,
+                      int stage_bytes, int* status) {
+    constexpr int G = C::G, CW = C::CW, GPW = C::GPW, KC = C::KC, NW = C::NW;
+    constexpr int GP = (G + 1) / 2;
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int xs_bytes = KC * geo.plane * 4;                       // one stage: KC planes, then the weight block
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
+    uint64_t* empty = full + S;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + S);
+    float* zrow = reinterpret_cast<float*>(empty + S) + 4;         // geo.pitch zeros
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int f0 = blockIdx.x * geo.R;
+    const int tile = blockIdx.y;
+    const int NH = geo.N * geo.H, W = geo.W;
+    const int32_t* bp = blk_ptr + (size_t)tile * (geo.nchunks + 1);
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, NW);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    for (int i = tid; i < geo.pitch; i += blockDim.x) zrow[i] = 0.0f;
+    __syncthreads();
+
+    if (warp == NW) {
+        // ---------------- producer warp ----------------
+        bool ok = true;
+        int k = 0;
+        for (; k < geo.nchunks && ok; ++k) {
+            const int s = k % S;
+            if (k >= S) ok = mbar_wait(empty + s, ((k / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+            if (!ok) break;
+            if (lane == 0) {
+                const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
+                unsigned char* st = smem + (size_t)s * stage_bytes;
+                mbar_arrive_expect_tx(full + s, (uint32_t)xs_bytes + (uint32_t)wn * 16u);
+                tensor_g2s_3d(st, &xmap, -4, f0 - 1, k * KC, full + s);
+                bulk_g2s(st + xs_bytes, rec + wbeg, (uint32_t)wn * 16u, full + s);
+            }
+        }
+        if (!ok) {   // gave up: let the copies already issued land before the CTA's shared memory is released
+            for (int j = max(0, k - S); j < k; ++j) {
+                bool landed = false;
+                for (uint32_t i = 0; i < kWaitLimit && !landed; ++i) landed = mbar_try_wait(full + j % S, (j / S) & 1);
+            }
+        }
+        return;
+    }
+
+    // ---------------- compute warps ----------------
+    const int pw = warp % C::NPW, gw = warp / C::NPW;
+    const int lrow = pw * geo.RPW + lane / geo.LPR;
+    const int lx = (lane % geo.LPR) * CW;
+    const int f = f0 + lrow;
+    const int y = f % geo.H;
+    // plane row j holds image row f0 - 1 + j; column c holds x = c - 4
+    int rowoff[3];
+    bool rowok[3];
+#pragma unroll
+    for (int kh = 0; kh < 3; ++kh) {
+        rowoff[kh] = (lrow + kh) * geo.pitch + lx + 3;             // column of x = lx - 1
+        rowok[kh] = (kh == 0) ? (y > 0) : (kh == 2 ? (y < geo.H - 1) : true);
+    }
+    const float* zr = zrow + lx + 3;
+
+    f32x2 acc[GPW][CW][GP];
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * C::GT + gw * GPW + q;
+#pragma unroll
+        for (int r = 0; r < GP; ++r) {
+            const float b0 = (g < geo.ngroups) ? bias[g * G + 2 * r] : 0.0f;
+            const float b1 = (g < geo.ngroups && 2 * r + 1 < G) ? bias[g * G + 2 * r + 1] : 0.0f;
+#pragma unroll
+            for (int p = 0; p < CW; ++p) acc[q][p][r] = pack2(b0, b1);
+        }
+    }
+
+    for (int k = 0; k < geo.nchunks; ++k) {
+        const int s = k % S;
+        if (!mbar_wait(full + s, (k / S) & 1, abort_flag, status, SBNN_ERR_TIMEOUT)) return;
+        const float* xs = reinterpret_cast<const float*>(smem + (size_t)s * stage_bytes);
+        const uint4* ws = reinterpret_cast<const uint4*>(smem + (size_t)s * stage_bytes + xs_bytes);
+#pragma unroll
+        for (int q = 0; q < GPW; ++q) {
+            const int2 hd = reinterpret_cast<const int2*>(ws)[gw * GPW + q];
+            const uint4* r = ws + hd.x;
+            for (int it = 0; it < hd.y; ++it, r += C::UNIT) {
+                const float* plane = xs + r[0].x;
+                const float* wq = reinterpret_cast<const float*>(r + 1);   // [9][G]
+#pragma unroll
+                for (int kh = 0; kh < 3; ++kh) {
+                    const float* arow = rowok[kh] ? plane + rowoff[kh] : zr;
+                    f32x2 a[CW + 2];
+#pragma unroll
+                    for (int i = 0; i < CW + 2; ++i) a[i] = dup2(arow[i]);
+#pragma unroll
+                    for (int kw = 0; kw < 3; ++kw) {
+                        f32x2 w[GP];
+                        if constexpr (G % 4 == 0) {
+#pragma unroll
+                            for (int v = 0; v < G / 4; ++v) {
+                                const ulonglong2 t = reinterpret_cast<const ulonglong2*>(wq + (kh * 3 + kw) * G)[v];
+                                w[2 * v] = t.x;
+                                w[2 * v + 1] = t.y;
+                            }
+                        } else if constexpr (G == 2) {
+                            w[0] = *reinterpret_cast<const unsigned long long*>(wq + (kh * 3 + kw) * 2);
+                        } else {
+                            w[0] = pack2(wq[kh * 3 + kw], 0.0f);
+                        }
+#pragma unroll
+                        for (int p = 0; p < CW; ++p)
+#pragma unroll
+                            for (int rr = 0; rr < GP; ++rr) fma2(acc[q][p][rr], a[p + kw], w[rr]);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty + s);
+    }
+
+    if (f >= NH) return;
+#pragma unroll
+    for (int q = 0; q < GPW; ++q) {
+        const int g = tile * C::GT + gw * GPW + q;
+        if (g >= geo.ngroups) continue;
+#pragma unroll
+        for (int p = 0; p < CW; ++p) {
+            const int x = lx + p;
+            if (x >= W) continue;
+            float* yp = Y + ((size_t)f * W + x) * geo.Cout + g * G;
+            float v[2 * GP];
+#pragma unroll
+            for (int rr = 0; rr < GP; ++rr) unpack2(acc[q][p][rr], v[2 * rr], v[2 * rr + 1]);
+            if (relu) {
+#pragma unroll
+                for (int rr = 0; rr < 2 * GP; ++rr) v[rr] = fmaxf(v[rr], 0.0f);
+            }
+            if constexpr (G >= 4) {
+#pragma unroll
+                for (int vv = 0; vv < G / 4; ++vv)
+                    reinterpret_cast<float4*>(yp)[vv] = make_float4(v[4 * vv], v[4 * vv + 1], v[4 * vv + 2], v[4 * vv + 3]);
+            } else if constexpr (G == 2) {
+                *reinterpret_cast<float2*>(yp) = make_float2(v[0], v[1]);
+            } else {
+                yp[0] = v[0];
+            }
+        }
+    }
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 int pow2_ceil(int v) {
@@ -539,6 +710,70 @@ sbnn_status launch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y,
     return SBNN_OK;
 }
 
+// Launches the copy-engine variant; *done = false (and SBNN_OK) if the shape does not fit it.
+template <class C>
+sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
+                        cudaStream_t st, bool* done) {
+    *done = false;
+    Geo3 g;
+    g.N = N; g.H = H; g.W = W; g.Cin = p->Cin; g.Cout = p->Cout; g.ngroups = p->ngroups;
+    g.LPR = lanes_per_row(W, C::CW);
+    g.RPW = 32 / g.LPR;
+    g.R = C::NPW * g.RPW;
+    g.pitch = pick_pitch4(g.LPR, C::CW);
+    g.plane = (g.R + 2) * g.pitch;                                 // the copied box: no padding between planes
+    g.nchunks = (p->Cin + C::KC - 1) / C::KC;
+    g.dpp_row = g.dpp_x = 0;
+    if (g.pitch > 256 || g.R + 2 > 256 || W % 4 || ldx % 4) return SBNN_OK;
+    const int stage_bytes = (C::KC * g.plane * 4 + C::WS_U4 * 16 + 127) / 128 * 128;
+    const size_t tail = (size_t)2 * 3 * 8 + 16 + (size_t)g.pitch * 4;
+    int S = 3;
+    if ((size_t)S * stage_bytes + tail > 227 * 1024) S = 2;
+    const size_t smem = (size_t)S * stage_bytes + tail;
+    if (smem > 227 * 1024) return SBNN_OK;
+    Stream3x3 s;
+    {
+        std::lock_guard<std::mutex> lk(p->mu);
+        const int key = (g.plane << 8) | (C::GT << 4) | (C::KC / 4);
+        auto it = p->streams3x3.find(key);
+        if (it == p->streams3x3.end()) {
+            sbnn_status r = build_stream3(p, C::GT, C::KC, g.plane, &s);
+            if (r != SBNN_OK) return r;
+            p->streams3x3[key] = s;
+        } else {
+            s = it->second;
+        }
+    }
+    if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
+    const long long NH = (long long)N * H;
+    Map3 xmap;
+    const unsigned long long dims[3] = {(unsigned long long)W, (unsigned long long)NH, (unsigned long long)p->Cin};
+    const unsigned long long strides[2] = {(unsigned long long)W * 4, (unsigned long long)ldx * 4};
+    const unsigned box[3] = {(unsigned)g.pitch, (unsigned)(g.R + 2), (unsigned)C::KC};
+    sbnn_status r = encode_tiled_map(&xmap, xt, 3, dims, strides, box);
+    if (r != SBNN_OK) return r;
+    int* status = nullptr;
+    if ((r = async_status_word(&status)) != SBNN_OK) return r;
+    SBNN_CUDA_TRY(cudaFuncSetAttribute(conv3x3_gs_tma_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid((unsigned)((NH + g.R - 1) / g.R), s.ntiles);
+    conv3x3_gs_tma_kernel<C><<<grid, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    *done = true;
+    return SBNN_OK;
+}
+
+template <int CW>
+sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
+                          cudaStream_t st, bool* done) {
+    switch (p->G) {
+        case 1: return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        case 2: return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        case 4: return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        case 8: return launch3_tma<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        default: return launch3_tma<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+    }
+}
+
 template <int CW>
 sbnn_status dispatch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
                          cudaStream_t st, bool* done) {
@@ -610,6 +845,9 @@ extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev,
         if ((st = scratch_workspace((size_t)w->Cin * ld * sizeof(float), &xt)) != SBNN_OK) return st;
         if ((st = launch_transpose(x_dev, w->Cin, xt, ld, M, w->Cin, s)) != SBNN_OK) return st;
         bool done = false;
+        st = cw == 7 ? dispatch3_tma<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
+                     : dispatch3_tma<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);
+        if (st != SBNN_OK || done) return st;
         st = cw == 7 ? dispatch3_cm<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
                      : dispatch3_cm<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);
         if (st != SBNN_OK || done) return st;

@@ -91,4 +91,11 @@ __device__ __forceinline__ void tensor_g2s_2d(void* dst_smem, const void* tensor
                  : "memory");
 }
 
+// The same for a 3-D tensor map: box origin (x, y, z), x along the contiguous dimension.
+__device__ __forceinline__ void tensor_g2s_3d(void* dst_smem, const void* tensor_map, int x, int y, int z, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(smem_u32(dst_smem)), "l"(tensor_map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+                 : "memory");
+}
+
 }  // namespace sbnn
