@@ -98,10 +98,10 @@ sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M
 sbnn_status read_async_status(int* value);
 // Device address of the status word that bounded waits report into (per device).
 sbnn_status async_status_word(int** out);
-// Fills a 128-byte tensor-map descriptor (CUtensorMap) for tiled copies out of an fp32 tensor: `rank` dimensions,
-// innermost first, `strides_bytes` for dimensions 1.. (multiples of 16), `box` = elements copied per dimension.
-// Elements outside the tensor are delivered as zeros.
-sbnn_status encode_tiled_map(void* out, const float* base, int rank, const unsigned long long* dims,
+// Fills a 128-byte tensor-map descriptor (CUtensorMap) for tiled copies out of an fp32 (elem_bytes 4) or bf16 (2)
+// tensor: `rank` dimensions, innermost first, `strides_bytes` for dimensions 1.. (multiples of 16), `box` = elements
+// copied per dimension.  Elements outside the tensor are delivered as zeros.
+sbnn_status encode_tiled_map(void* out, const void* base, int elem_bytes, int rank, const unsigned long long* dims,
                              const unsigned long long* strides_bytes, const unsigned* box);
 // Per-device scratch buffer for channel-major copies made on behalf of NHWC callers (grows on demand, synchronously).
 sbnn_status scratch_workspace(size_t bytes, float** out);

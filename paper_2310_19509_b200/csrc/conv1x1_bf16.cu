@@ -16,8 +16,10 @@
 //
 // CTA = 128 pixels x 8 warps; a warp owns GPW groups over all 128 pixels (8 row blocks of 16), i.e.
 // 32 fp32 accumulators per N-tile.  A pre-pass converts X once to bf16 in channel-major order
-// ([Cin][ld], pixels contiguous); the kernel then fills its [channel][pixel] tile with 16-byte
-// cp.async pieces into two buffers, so the copies of step k+1 run under the MMAs of step k.  The
+// ([Cin][ld], pixels contiguous); a ninth warp then fills the [channel][pixel] tile of every channel
+// step with one tiled tensor-map copy (plus a linear copy of the step's weight block) onto a "full"
+// mbarrier, and the MMA warps hand a stage back through an "empty" mbarrier, so no CTA-wide barrier
+// makes warps with fewer kept channels in a step wait for the others (two stages, bounded waits).  The
 // weight stream holds, per 16 kept channels, 16 row offsets and the B fragments in register order.
 #include <cuda_bf16.h>
 #include <string.h>
@@ -26,6 +28,7 @@
 #include <new>
 
 #include "common.h"
+#include "pipeline.cuh"
 
 namespace sbnn {
 namespace {
@@ -57,20 +60,63 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+struct MapB { alignas(64) unsigned char bytes[128]; };
+
+constexpr int STAGE_X = KC * ROWB;         // bytes of activations per stage (a multiple of 128)
+
 template <int G, int GPW>
-__global__ void __launch_bounds__(NWARP * 32)
-conv1x1_bf16_kernel(const __nv_bfloat16* __restrict__ Xb, int ldb, float* __restrict__ Y, const float* __restrict__ bias,
+__global__ void __launch_bounds__((NWARP + 1) * 32)
+conv1x1_bf16_kernel(const __grid_constant__ MapB xmap, float* __restrict__ Y, const float* __restrict__ bias,
                     const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout,
-                    int ngroups, int nchunks, int ntiles, int ws_u4, int relu) {
+                    int ngroups, int nchunks, int ntiles, int ws_u4, int S, int stage_bytes, int relu, int* status) {
     constexpr int NT8 = (G + 7) / 8;
     constexpr int GT = NWARP * GPW;
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* xs0 = smem;                                         // two buffers of [KC][ROWB]
-    uint4* ws0 = reinterpret_cast<uint4*>(smem + 2 * KC * ROWB);       // two weight blocks of ws_u4 units
+    // S stages of [KC][ROWB] activations + the step's weight block, then the stages' "full" and "empty" mbarriers
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
+    uint64_t* empty = full + S;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + S);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tile = blockIdx.x % ntiles;
     const int m0 = (blockIdx.x / ntiles) * TM;
     const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, NWARP);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == NWARP) {
+        // producer warp: per channel step one tiled copy of the [KC][TM + 8] box of X (the 8 extra pixels are the row
+        // padding that spreads the rows over the banks; channels past Cin and pixels past the tensor arrive as zeros)
+        // and one linear copy of the step's weight block, both onto the stage's "full" barrier
+        bool ok = true;
+        int k = 0;
+        for (; k < nchunks && ok; ++k) {
+            const int s = k % S;
+            if (k >= S) ok = mbar_wait(empty + s, ((k / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+            if (!ok) break;
+            if (lane == 0) {
+                const int beg = bp[k], n = bp[k + 1] - beg;
+                unsigned char* st = smem + (size_t)s * stage_bytes;
+                mbar_arrive_expect_tx(full + s, (uint32_t)STAGE_X + (uint32_t)n * 16u);
+                tensor_g2s_2d(st, &xmap, m0, k * KC, full + s);
+                bulk_g2s(st + STAGE_X, rec + beg, (uint32_t)n * 16u, full + s);
+            }
+        }
+        if (!ok) {   // gave up: let the copies already issued land before the CTA's shared memory is released
+            for (int j = max(0, k - S); j < k; ++j) {
+                bool landed = false;
+                for (uint32_t i = 0; i < kWaitLimit && !landed; ++i) landed = mbar_try_wait(full + j % S, (j / S) & 1);
+            }
+        }
+        return;
+    }
+
     const int gq = lane >> 2, tq = lane & 3;
 
     float acc[GPW][NT8][8][4];
@@ -90,36 +136,13 @@ conv1x1_bf16_kernel(const __nv_bfloat16* __restrict__ Xb, int ldb, float* __rest
     }
     // ldmatrix: lane l addresses row (l & 7) of sub-matrix (l >> 3): channels 8*(l>>4) + (l&7), pixels 8*((l>>3)&1)..
     const int off_idx = 8 * (lane >> 4) + (lane & 7);
-    const uint32_t xs_base = static_cast<uint32_t>(__cvta_generic_to_shared(xs0)) + ((lane >> 3) & 1) * 16;
+    const uint32_t xs_base = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + ((lane >> 3) & 1) * 16;
 
-    auto cp16 = [](void* dst, const void* src) {
-        const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(dst));
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(src) : "memory");
-    };
-    auto issue = [&](int k, int buf) {   // rows of 128 pixels = 16 pieces of 16 bytes; then the weight block
-        unsigned char* xd = xs0 + buf * (KC * ROWB);
-        for (int i = tid; i < KC * 16; i += NWARP * 32) {
-            const int c = i >> 4, pc = i & 15;
-            if (k * KC + c < Cin) cp16(xd + c * ROWB + pc * 16, Xb + (size_t)(k * KC + c) * ldb + m0 + pc * 8);
-        }
-        uint4* wd = ws0 + buf * ws_u4;
-        const int beg = bp[k], n = bp[k + 1] - beg;
-        for (int i = tid; i < n; i += NWARP * 32) cp16(wd + i, rec + beg + i);
-        asm volatile("cp.async.commit_group;\n" ::: "memory");
-    };
-
-    issue(0, 0);
     for (int k = 0; k < nchunks; ++k) {
-        const int cur = k & 1;
-        if (k + 1 < nchunks) {
-            issue(k + 1, cur ^ 1);
-            asm volatile("cp.async.wait_group 1;\n" ::: "memory");
-        } else {
-            asm volatile("cp.async.wait_group 0;\n" ::: "memory");
-        }
-        __syncthreads();
-        const uint4* ws = ws0 + cur * ws_u4;
-        const uint32_t xs_lane = xs_base + cur * (KC * ROWB);
+        const int s = k % S;
+        if (!mbar_wait(full + s, (k / S) & 1, abort_flag, status, SBNN_ERR_TIMEOUT)) return;
+        const uint4* ws = reinterpret_cast<const uint4*>(smem + (size_t)s * stage_bytes + STAGE_X);
+        const uint32_t xs_lane = xs_base + s * stage_bytes;
 #pragma unroll
         for (int q = 0; q < GPW; ++q) {
             const int2 hd = reinterpret_cast<const int2*>(ws)[warp * GPW + q];   // (start, 16-channel blocks)
@@ -141,7 +164,8 @@ conv1x1_bf16_kernel(const __nv_bfloat16* __restrict__ Xb, int ldb, float* __rest
                 }
             }
         }
-        __syncthreads();   // done with this buffer before the copies of step k+2 are issued
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty + s);   // the warp is done with the stage
     }
 #pragma unroll
     for (int q = 0; q < GPW; ++q) {
@@ -306,13 +330,25 @@ sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, const float* 
     to_channel_major_bf16_kernel<<<tg, 256, 0, st>>>(x, xb, M, p->Cin, ldb);
     SBNN_CUDA_TRY(cudaGetLastError());
 
-    const size_t smem = (size_t)2 * KC * ROWB + (size_t)2 * s.max_blk * 16;
+    const int stage_bytes = (STAGE_X + s.max_blk * 16 + 127) / 128 * 128;
+    // Two stages: with about 38 KB per stage that leaves room for two or three CTAs per SM, which measured faster
+    // than one CTA with four stages (config 5, G = 8, dense: 577 us against 722 us).
+    const int S = 2;
+    const size_t smem = (size_t)S * stage_bytes + 2 * S * 8 + 16;
     if (smem > 200 * 1024) return fail(SBNN_ERR_UNSUPPORTED, "internal: bf16 tile needs %zu bytes of shared memory", smem);
+    MapB xmap;
+    const unsigned long long dims[2] = {(unsigned long long)ldb, (unsigned long long)p->Cin};
+    const unsigned long long strides[1] = {(unsigned long long)ldb * sizeof(__nv_bfloat16)};
+    const unsigned box[2] = {(unsigned)(ROWB / 2), (unsigned)KC};
+    if ((r = encode_tiled_map(&xmap, xb, 2, 2, dims, strides, box)) != SBNN_OK) return r;
+    int* status = nullptr;
+    if ((r = async_status_word(&status)) != SBNN_OK) return r;
     SBNN_CUDA_TRY(cudaFuncSetAttribute(conv1x1_bf16_kernel<G, GPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const long long nblk = (long long)(ldb / TM) * s.ntiles;
     if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
-    conv1x1_bf16_kernel<G, GPW><<<(unsigned)nblk, NWARP * 32, smem, st>>>(xb, ldb, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin,
-                                                                          p->Cout, p->ngroups, s.nchunks, s.ntiles, s.max_blk, relu);
+    conv1x1_bf16_kernel<G, GPW><<<(unsigned)nblk, (NWARP + 1) * 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin,
+                                                                                p->Cout, p->ngroups, s.nchunks, s.ntiles, s.max_blk,
+                                                                                S, stage_bytes, relu, status);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
 }

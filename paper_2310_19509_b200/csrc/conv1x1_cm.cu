@@ -505,8 +505,9 @@ sbnn_status get_encode(EncodeTiledFn* out) {
     return SBNN_OK;
 }
 
-// fp32 tensor of `rank` dimensions (innermost first), tiled copies of `box` elements, zeros outside the tensor.
-sbnn_status encode_generic(void* out, const float* base, int rank, const unsigned long long* dims,
+// fp32 (elem_bytes 4) or bf16 (2) tensor of `rank` dimensions (innermost first), tiled copies of `box` elements,
+// zeros outside the tensor.
+sbnn_status encode_generic(void* out, const void* base, int elem_bytes, int rank, const unsigned long long* dims,
                            const unsigned long long* strides_bytes, const unsigned* box) {
     EncodeTiledFn encode = nullptr;
     sbnn_status r = get_encode(&encode);
@@ -523,8 +524,9 @@ sbnn_status encode_generic(void* out, const float* base, int rank, const unsigne
             if (st[i] % 16) return fail(SBNN_ERR_ALIGN, "tensor stride %llu is not a multiple of 16 bytes", (unsigned long long)st[i]);
         }
     }
-    const CUresult cr = encode(static_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank,
-                               const_cast<float*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+    const CUresult cr = encode(static_cast<CUtensorMap*>(out),
+                               elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                               (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return fail(SBNN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)cr);
     return SBNN_OK;
@@ -535,7 +537,7 @@ sbnn_status encode_x_map(const float* x, int ldx, int M, int Cin, int box_px, in
     const unsigned long long dims[2] = {(unsigned long long)M, (unsigned long long)Cin};
     const unsigned long long strides[1] = {(unsigned long long)ldx * sizeof(float)};
     const unsigned box[2] = {(unsigned)box_px, (unsigned)box_rows};
-    return encode_generic(out, x, 2, dims, strides, box);
+    return encode_generic(out, x, 4, 2, dims, strides, box);
 }
 
 template <class C>
@@ -678,9 +680,9 @@ sbnn_status scratch_workspace(size_t bytes, float** out) { return workspace(byte
 
 sbnn_status async_status_word(int** out) { return status_word(out); }
 
-sbnn_status encode_tiled_map(void* out, const float* base, int rank, const unsigned long long* dims,
+sbnn_status encode_tiled_map(void* out, const void* base, int elem_bytes, int rank, const unsigned long long* dims,
                              const unsigned long long* strides_bytes, const unsigned* box) {
-    return encode_generic(out, base, rank, dims, strides_bytes, box);
+    return encode_generic(out, base, elem_bytes, rank, dims, strides_bytes, box);
 }
 
 sbnn_status prepare_default_cm(const sbnn_packed* p, long long M) {

@@ -750,7 +750,7 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     const unsigned long long dims[3] = {(unsigned long long)W, (unsigned long long)NH, (unsigned long long)p->Cin};
     const unsigned long long strides[2] = {(unsigned long long)W * 4, (unsigned long long)ldx * 4};
     const unsigned box[3] = {(unsigned)g.pitch, (unsigned)(g.R + 2), (unsigned)C::KC};
-    sbnn_status r = encode_tiled_map(&xmap, xt, 3, dims, strides, box);
+    sbnn_status r = encode_tiled_map(&xmap, xt, 4, 3, dims, strides, box);
     if (r != SBNN_OK) return r;
     int* status = nullptr;
     if ((r = async_status_word(&status)) != SBNN_OK) return r;
