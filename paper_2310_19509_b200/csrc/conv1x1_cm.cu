@@ -132,6 +132,102 @@ __device__ __forceinline__ void run_list(const uint4* r, int n, const unsigned c
     }
 }
 
+// ---- second form of the list loop, for G >= 8 ---------------------------------------------------------------
+// The same loop with every shared-memory load written as a volatile instruction on a 32-bit shared address, which
+// pins the loads to program order (the order the look-ahead was written in).  Measured: the one-group-per-warp
+// G = 8 kernels gain 2-3 % from the pinned order (config 5 at 50 %: 0.594 -> 0.609 of roofline), the union-list
+// G = 4 kernels lose about as much, so each keeps its own form.
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ ulonglong2 lds128_pairs(uint32_t addr) {
+    ulonglong2 v;
+    asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+// The G weights of unit u of a quad whose weights start at shared address wq.
+template <int G>
+__device__ __forceinline__ void unit_weights_v(uint32_t wq, int u, float (&w)[G]) {
+    if constexpr (G >= 4) {
+#pragma unroll
+        for (int v = 0; v < G / 4; ++v) {
+            const uint4 t = lds128(wq + (u * (G / 4) + v) * 16);
+            w[4 * v + 0] = __uint_as_float(t.x); w[4 * v + 1] = __uint_as_float(t.y);
+            w[4 * v + 2] = __uint_as_float(t.z); w[4 * v + 3] = __uint_as_float(t.w);
+        }
+    } else if constexpr (G == 2) {
+        const uint2 t = lds64(wq + u * 8);
+        w[0] = __uint_as_float(t.x); w[1] = __uint_as_float(t.y);
+    } else {
+        w[0] = __uint_as_float(lds32(wq + u * 4));
+    }
+}
+
+// run_list with shared addresses: r = the list's first quad, xs = the lane's first pixels in the stage.
+template <int P, int G, int NG>
+__device__ __forceinline__ void run_list_v(uint32_t r, int n, uint32_t xs, f32x2 (&acc0)[P / 2][G],
+                                           f32x2 (&acc1)[P / 2][G]) {
+    constexpr int QUAD = 1 + NG * G;
+    ulonglong2 aA[P / 4], aB[P / 4];
+    float wA[NG * G], wB[NG * G];
+    auto load_unit = [&](uint32_t quad, unsigned off, int u, ulonglong2 (&a)[P / 4], float (&w)[NG * G]) {
+#pragma unroll
+        for (int i = 0; i < P / 4; ++i) a[i] = lds128_pairs(xs + off + i * 512);
+        unit_weights_v<NG * G>(quad + 16, u, w);
+    };
+    auto fma_unit = [&](const ulonglong2 (&a)[P / 4], const float (&w)[NG * G]) {
+#pragma unroll
+        for (int rr = 0; rr < NG * G; ++rr) {
+            const f32x2 ww = dup2(w[rr]);
+#pragma unroll
+            for (int i = 0; i < P / 4; ++i) {
+                if (rr < G) {
+                    fma2(acc0[2 * i][rr], a[i].x, ww);
+                    fma2(acc0[2 * i + 1][rr], a[i].y, ww);
+                } else {
+                    fma2(acc1[2 * i][rr - G], a[i].x, ww);
+                    fma2(acc1[2 * i + 1][rr - G], a[i].y, ww);
+                }
+            }
+        }
+    };
+    uint4 off = lds128(r);
+    load_unit(r, off.x, 0, aA, wA);
+    const int nfull = n >> 2, rem = n & 3;
+    for (int it = 0; it < nfull; ++it) {
+        const uint4 off_next = lds128(r + QUAD * 16);
+        load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+        load_unit(r, off.z, 2, aA, wA); fma_unit(aB, wB);
+        load_unit(r, off.w, 3, aB, wB); fma_unit(aA, wA);
+        load_unit(r + QUAD * 16, off_next.x, 0, aA, wA); fma_unit(aB, wB);
+        off = off_next;
+        r += QUAD * 16;
+    }
+    if (rem == 1) {   // last, short quad (warp-uniform)
+        fma_unit(aA, wA);
+    } else if (rem == 2) {
+        load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+        fma_unit(aB, wB);
+    } else if (rem == 3) {
+        load_unit(r, off.y, 1, aB, wB); fma_unit(aA, wA);
+        load_unit(r, off.z, 2, aA, wA); fma_unit(aB, wB);
+        fma_unit(aA, wA);
+    }
+}
+
 template <class C, bool OUT_CM>
 __global__ void __launch_bounds__(C::NT, 1)
 conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ Y, int ldy,
@@ -221,19 +317,31 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
         const int s = consumed % S;
         ok = mbar_wait(full + s, (consumed / S) & 1, abort_flag, status, SBNN_ERR_TIMEOUT);
         if (!ok) break;
-        const unsigned char* xs = xs0 + (size_t)s * C::XS_BYTES + lane_off;
-        const uint4* ws = reinterpret_cast<const uint4*>(ws0 + (size_t)s * C::WS_BYTES);
-        const int2* hdr = reinterpret_cast<const int2*>(ws) + warp * C::NL;   // (start, kept units) per list
-        if constexpr (C::UNION) {
-            const int2 hb = hdr[0], h0 = hdr[1], h1 = hdr[2];
-            run_list<P, G, 2>(ws + hb.x, hb.y, xs, acc[0], acc[1]);   // channels both groups keep
-            run_list<P, G, 1>(ws + h0.x, h0.y, xs, acc[0], acc[0]);   // only the first group
-            run_list<P, G, 1>(ws + h1.x, h1.y, xs, acc[1], acc[1]);   // only the second group
-        } else {
+        if constexpr (G >= 8) {
+            const uint32_t xs = smem_u32(xs0) + (uint32_t)s * C::XS_BYTES + lane_off;
+            const uint32_t ws = smem_u32(ws0) + (uint32_t)s * C::WS_BYTES;
+            const uint32_t hdr = ws + warp * C::NL * 8;             // (start in 16-byte units, kept units) per list
+            static_assert(G < 8 || !C::UNION, "the G >= 8 instances have one list per group");
 #pragma unroll
             for (int q = 0; q < GPW; ++q) {
-                const int2 hd = hdr[q];
-                run_list<P, G, 1>(ws + hd.x, hd.y, xs, acc[q], acc[q]);
+                const uint2 hd = lds64(hdr + q * 8);
+                run_list_v<P, G, 1>(ws + hd.x * 16, (int)hd.y, xs, acc[q], acc[q]);
+            }
+        } else {
+            const unsigned char* xs = xs0 + (size_t)s * C::XS_BYTES + lane_off;
+            const uint4* ws = reinterpret_cast<const uint4*>(ws0 + (size_t)s * C::WS_BYTES);
+            const int2* hdr = reinterpret_cast<const int2*>(ws) + warp * C::NL;   // (start, kept units) per list
+            if constexpr (C::UNION) {
+                const int2 hb = hdr[0], h0 = hdr[1], h1 = hdr[2];
+                run_list<P, G, 2>(ws + hb.x, hb.y, xs, acc[0], acc[1]);   // channels both groups keep
+                run_list<P, G, 1>(ws + h0.x, h0.y, xs, acc[0], acc[0]);   // only the first group
+                run_list<P, G, 1>(ws + h1.x, h1.y, xs, acc[1], acc[1]);   // only the second group
+            } else {
+#pragma unroll
+                for (int q = 0; q < GPW; ++q) {
+                    const int2 hd = hdr[q];
+                    run_list<P, G, 1>(ws + hd.x, hd.y, xs, acc[q], acc[q]);
+                }
             }
         }
         __syncwarp();
