@@ -28,7 +28,7 @@ import numpy as np  # noqa: E402
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FP32 lanes x 2 flop x max SM clock
 HBM_FALLBACK_GBS = 6650.0
 METRIC = "mobilenet_v1_images_per_s"
-PW_DRAM_BYTES_PER_STEP = 746.9e6
+PW_DRAM_BYTES_PER_STEP = 746.5e6
 
 
 def measured_peaks():
