@@ -201,6 +201,16 @@ SBNN_API sbnn_status sbnn_dwconv3x3(const float* w_dev, const float* b_dev, cons
                                     int N, int H, int W, int C, int stride, int flags, void* cuda_stream);
 
 /*
+ * The same depthwise convolution on channel-major tensors, as the MobileNet chain runs it: xt_dev [C][ldx] with the
+ * pixels of a channel contiguous (index (n*H + y)*W + x), yt_dev [C][ldy] likewise for the output; ldx >= N*H*W,
+ * ldy >= N*Ho*Wo, both multiples of 4, both tensors 16-byte aligned; H and W must be divisible by the stride
+ * (else SBNN_ERR_UNSUPPORTED).  w_dev [3][3][C], b_dev [C] or NULL.  Any C.  The kernel is chosen by shape
+ * (row blocks of 4 for wide maps, column strips for the 14- and 7-wide maps, one output per thread otherwise).
+ */
+SBNN_API sbnn_status sbnn_dwconv3x3_cm(const float* w_dev, const float* b_dev, const float* xt_dev, int ldx, float* yt_dev,
+                                       int ldy, int N, int H, int W, int C, int stride, int flags, void* cuda_stream);
+
+/*
  * Depthwise 3x3 with 3:9 kernel patterns (Section 3.2, DwConv3x3; Algorithm 2): in every row of a kernel the
  * middle weight stays and either the first or the third column is pruned, one pattern per block of go
  * consecutive channels (the paper's PatternInfo; go = 16, or 8 or 4 for channel counts that need it).

@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     conv3x3_dense,
     conv3x3_gs,
     dwconv3x3,
+    dwconv3x3_cm,
     dwconv3x3_pattern,
     get_async_status,
     head_noalloc,

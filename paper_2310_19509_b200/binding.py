@@ -50,6 +50,7 @@ def lib():
         "sbnn_conv1x1_gs_cm": [P, P, I, P, I, I, I, I, I, I, I, P],
         "sbnn_to_channel_major": [P, P, I, I, I, P],
         "sbnn_dwconv3x3": [P, P, P, P, I, I, I, I, I, I, P],
+        "sbnn_dwconv3x3_cm": [P, P, P, I, P, I, I, I, I, I, I, I, P],
         "sbnn_pack_dw_pattern": [P, P, I, I, P, P],
         "sbnn_dwconv3x3_pattern": [P, P, I, P, P, P, I, I, I, I, I, I, P],
         "sbnn_conv3x3_dense": [P, P, P, P, I, I, I, I, I, I, I, P],
@@ -185,6 +186,10 @@ def conv3x3_gs(w: Packed, x, y, n, h, wd, flags=SBNN_RELU, stream=None):
 
 def dwconv3x3(w, b, x, y, n, h, wd, c, stride, flags=SBNN_RELU, stream=None):
     _check(lib().sbnn_dwconv3x3(_ptr(w), _ptr(b), _ptr(x), _ptr(y), n, h, wd, c, stride, flags, _stream(stream)))
+
+
+def dwconv3x3_cm(w, b, xt, ldx, yt, ldy, n, h, wd, c, stride, flags=SBNN_RELU, stream=None):
+    _check(lib().sbnn_dwconv3x3_cm(_ptr(w), _ptr(b), _ptr(xt), ldx, _ptr(yt), ldy, n, h, wd, c, stride, flags, _stream(stream)))
 
 
 def pack_dw_pattern(w, mask, go):

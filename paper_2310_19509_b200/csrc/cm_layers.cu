@@ -757,3 +757,25 @@ sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int ldy, int N,
 }
 
 }  // namespace sbnn
+
+using namespace sbnn;
+
+extern "C" sbnn_status sbnn_dwconv3x3_cm(const float* w_dev, const float* b_dev, const float* xt_dev, int ldx, float* yt_dev,
+                                         int ldy, int N, int H, int W, int C, int stride, int flags, void* cuda_stream) {
+    clear_error();
+    if (!w_dev || !xt_dev || !yt_dev) return fail(SBNN_ERR_NULL, "w_dev, xt_dev and yt_dev must not be NULL");
+    if (N < 0 || H < 0 || W < 0 || C <= 0) return fail(SBNN_ERR_SHAPE, "bad shape N=%d H=%d W=%d C=%d", N, H, W, C);
+    if (stride != 1 && stride != 2) return fail(SBNN_ERR_SHAPE, "stride %d: only 1 and 2", stride);
+    if (flags & ~SBNN_RELU) return fail(SBNN_ERR_UNSUPPORTED, "unknown flag bits 0x%x", flags);
+    if ((long long)N * H * W > 0x7fffffffLL / 2) return fail(SBNN_ERR_SHAPE, "N*H*W too large");
+    const int Ho = stride ? (H - 1) / stride + 1 : 0, Wo = stride ? (W - 1) / stride + 1 : 0;
+    if (ldx < N * H * W || ldy < N * Ho * Wo || ldx % 4 || ldy % 4)
+        return fail(SBNN_ERR_SHAPE, "ldx=%d / ldy=%d must cover the pixels of a channel and be multiples of 4", ldx, ldy);
+    if (!aligned16(xt_dev) || !aligned16(yt_dev)) return fail(SBNN_ERR_ALIGN, "xt_dev and yt_dev must be 16-byte aligned");
+    if ((long long)N * H * W == 0) return SBNN_OK;
+    sbnn_status st = check_device();
+    if (st != SBNN_OK) return st;
+    return launch_dwconv3x3_cm(w_dev, b_dev, xt_dev, ldx, yt_dev, ldy, N, H, W, C, stride, flags & SBNN_RELU,
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+

@@ -123,6 +123,31 @@ def test_depthwise(stride, shape):
     assert_within(yd.cpu().numpy(), ref, s, what=f"dw {shape} s{stride}")
 
 
+@pytest.mark.parametrize("stride,hw", [(1, (8, 8)), (1, (6, 8)), (1, (14, 14)), (1, (7, 14)), (1, (7, 7)), (1, (5, 6)),
+                                       (2, (8, 16)), (2, (6, 8)), (2, (28, 28)), (2, (14, 14)), (2, (6, 6))])
+@pytest.mark.parametrize("n,c", [(3, 5), (2, 37)])
+def test_depthwise_channel_major_variants(stride, hw, n, c):
+    """Every kernel behind the channel-major depthwise entry point (row blocks, the stride-2 row blocks, the one-row
+    fallbacks, the 14 x 14 kernel, column strips, one output per thread), several images and channel counts that do
+    not fill a CTA's channel slots, leading dimensions with padding."""
+    h, w = hw
+    rng = np.random.default_rng(41)
+    x = rng.random((n, h, w, c), dtype=np.float32)
+    wt = rng.standard_normal((3, 3, c)).astype(np.float32)
+    b = rng.standard_normal(c).astype(np.float32)
+    ho, wo = (h - 1) // stride + 1, (w - 1) // stride + 1
+    ldx, ldy = (n * h * w + 3) // 4 * 4 + 4, (n * ho * wo + 3) // 4 * 4 + 8
+    xt = torch.zeros((c, ldx), device="cuda")
+    xt[:, :n * h * w] = dev(x).reshape(n * h * w, c).t()
+    yt = torch.full((c, ldy), float("nan"), device="cuda")
+    sbnn.dwconv3x3_cm(dev(wt), dev(b), xt, ldx, yt, ldy, n, h, w, c, stride)
+    sbnn.get_async_status()
+    y = yt[:, :n * ho * wo].t().reshape(n, ho, wo, c).cpu().numpy()
+    ref, s = R.dwconv3x3(x, wt, b, stride=stride, relu=True)
+    assert_within(y, ref, s, what=f"dw cm {hw} s{stride} n={n} c={c}")
+    assert bool(torch.isnan(yt[:, n * ho * wo:]).all())          # nothing written past the last pixel
+
+
 @pytest.mark.parametrize("stride", [1, 2])
 @pytest.mark.parametrize("shape,go", [((2, 9, 11, 32), 16), ((1, 14, 14, 48), 8), ((1, 1, 1, 4), 4), ((3, 7, 7, 64), 16)])
 def test_depthwise_3of9_patterns(stride, shape, go):
