@@ -321,6 +321,14 @@ def test_3x3_kernel_patterns(g, kept_taps):
     p.free()
 
 
+def test_3x3_row_too_wide_for_the_tiled_copy():
+    """A 252-pixel row needs a plane pitch above the copy engine's 256-element box limit: the cp.async variant runs."""
+    d = WL.single_conv_inputs(1, 3, 252, 12, 16, 3, 4, 50, seed=15, w_sigma=0.1)
+    y = run_3x3(d)
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    assert_within(y, ref, s, what="3x3 W=252")
+
+
 def test_3x3_dense_and_empty_masks():
     for sp in (0, 100):
         d = WL.single_conv_inputs(1, 8, 8, 8, 8, 3, 4, sp, seed=6)
