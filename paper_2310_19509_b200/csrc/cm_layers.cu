@@ -382,80 +382,8 @@ dwconv3x3_cm_w14_kernel(const float* __restrict__ w, const float* __restrict__ b
 }
 
 // ---- first layer: NHWC image with Cin <= 4 in, channel-major out --------------------------------
-// One thread: 4 consecutive output columns of one row x 8 output channels; consecutive lanes take
-// consecutive column strips, so each channel's stores are contiguous across the warp.
-template <int S>
-__global__ void __launch_bounds__(256)
-conv3x3_thin_cm_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x,
-                       float* __restrict__ y, int ldy, int N, int H, int W, int Cin, int Cout, int Ho, int Wo, int relu) {
-    extern __shared__ __align__(16) float ws[];   // [9][Cin][Cout]
-    for (int i = threadIdx.x; i < 9 * Cin * Cout; i += blockDim.x) {
-        const int o = i % Cout, tc = i / Cout;
-        ws[i] = w[(size_t)o * 9 * Cin + tc];
-    }
-    __syncthreads();
-    constexpr int TW = 4, IW = S * (TW - 1) + 3;
-    const int strips = (Wo + TW - 1) / TW;
-    const long long total = (long long)N * Ho * strips;
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= total) return;
-    const int cg = blockIdx.y;
-    const int sx = (int)(t % strips);
-    const long long f = t / strips;                      // n*Ho + oy
-    const int oy = (int)(f % Ho);
-    const int n = (int)(f / Ho);
-    const int ox0 = sx * TW, ix0 = ox0 * S - 1;
-
-    float acc[TW][8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const float bv = b ? __ldg(b + cg * 8 + j) : 0.f;
-#pragma unroll
-        for (int i = 0; i < TW; ++i) acc[i][j] = bv;
-    }
-#pragma unroll
-    for (int kh = 0; kh < 3; ++kh) {
-        const int iy = oy * S + kh - 1;
-        if (iy < 0 || iy >= H) continue;
-        const float* row = x + ((size_t)n * H + iy) * W * Cin;
-        for (int c = 0; c < Cin; ++c) {
-            float in[IW];
-#pragma unroll
-            for (int j = 0; j < IW; ++j) {
-                const int ix = ix0 + j;
-                in[j] = (ix >= 0 && ix < W) ? __ldg(row + (size_t)ix * Cin + c) : 0.f;
-            }
-#pragma unroll
-            for (int kw = 0; kw < 3; ++kw) {
-                const float4* wp = reinterpret_cast<const float4*>(ws + ((kh * 3 + kw) * Cin + c) * Cout + cg * 8);
-                const float4 w0 = wp[0], w1 = wp[1];
-                const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-                for (int i = 0; i < TW; ++i)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(in[i * S + kw], wv[j], acc[i][j]);
-            }
-        }
-    }
-    const long long p0 = f * Wo + ox0;
-    const bool vec = (ox0 + 3 < Wo) && ((p0 & 3) == 0);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        float v[TW];
-#pragma unroll
-        for (int i = 0; i < TW; ++i) v[i] = relu ? fmaxf(acc[i][j], 0.f) : acc[i][j];
-        float* yp = y + (size_t)(cg * 8 + j) * ldy + p0;
-        if (vec) {
-            *reinterpret_cast<float4*>(yp) = make_float4(v[0], v[1], v[2], v[3]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < TW; ++i)
-                if (ox0 + i < Wo) yp[i] = v[i];
-        }
-    }
-}
-
-// Wide variant for Cout % 32 == 0: one thread computes 2 consecutive output columns x 32 output
+// Weights [Cout][3][3][Cin]; a CTA stages the 32 output channels of its channel group as [tap][Cin][32].
+// Generic kernel (Cout % 32 == 0): one thread computes 2 consecutive output columns x 32 output
 // channels, so every input value is loaded once per pixel pair (not once per channel group) and each
 // broadcast float4 of weights feeds 4 packed FMAs (pairs of output channels, fma.rn.f32x2).  Consecutive lanes take consecutive column pairs; a
 // channel's stores are 8-byte pieces that are contiguous across the warp.
@@ -736,17 +664,7 @@ sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* 
         SBNN_CUDA_TRY(cudaGetLastError());
         return SBNN_OK;
     }
-    const long long total = (long long)N * Ho * ((Wo + 3) / 4);
-    const long long blocks = (total + 255) / 256;
-    if (blocks > 0x7fffffff) return fail(SBNN_ERR_SHAPE, "tensor too large");
-    dim3 grid((unsigned)blocks, Cout / 8);
-    const size_t smem = sizeof(float) * 9 * Cin * Cout;
-    if (stride == 1)
-        conv3x3_thin_cm_kernel<1><<<grid, 256, smem, st>>>(w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu);
-    else
-        conv3x3_thin_cm_kernel<2><<<grid, 256, smem, st>>>(w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu);
-    SBNN_CUDA_TRY(cudaGetLastError());
-    return SBNN_OK;
+    return fail(SBNN_ERR_UNSUPPORTED, "channel-major first layer needs Cout %% 32 == 0 and an even leading dimension");
 }
 
 sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int ldy, int N, int HW, int C, cudaStream_t st) {

@@ -269,6 +269,23 @@ def test_forward_graph_replay_matches_plain_launches():
     net.free()
 
 
+def test_forward_accepts_an_image_that_is_only_4_byte_aligned():
+    """The first layer's fast kernel needs 16-byte aligned rows; an input at an odd float offset takes the generic
+    first-layer kernel and must give the same logits (same order of sums: compared closely, not bit for bit)."""
+    x, layers = mobilenet_v1_inputs(1, 50, 4, seed=6)
+    net = build_net(layers, 1)
+    flat = torch.zeros(x.size + 1, device="cuda")
+    flat[1:] = dev(x).reshape(-1)
+    a = torch.full((1, 1000), float("nan"), device="cuda")
+    b = torch.full((1, 1000), float("nan"), device="cuda")
+    net.forward(dev(x), a, 1)
+    net.forward(flat[1:], b, 1)
+    sbnn.get_async_status()
+    assert bool(torch.isfinite(b).all())
+    assert torch.allclose(a, b, rtol=1e-4, atol=1e-5)
+    net.free()
+
+
 def run_3x3(d, flags=sbnn.SBNN_RELU):
     x = d["x"]
     n, h, w, cin = x.shape
