@@ -194,6 +194,29 @@ def time_layers(sbnn, torch, net, layers, batch, reps, flush):
     return res
 
 
+def time_layers_in_chain(sbnn, torch, net, layers, batch, xd, reps):
+    """The 29 launches in forward's order on forward-sized ping-pong buffers, a CUDA event between consecutive
+    launches: what each kernel takes inside a step (its input just written by its predecessor, no L2 flush)."""
+    r4 = lambda v: (v + 3) // 4 * 4  # noqa: E731
+    bufs = [torch.empty(64 * r4(batch * 112 * 112) + 4096, device="cuda") for _ in range(2)]
+    logits = torch.empty((batch, 1000), device="cuda")
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(layers) + 1)]
+    samples = [[] for _ in layers]
+    for rep in range(reps + 2):
+        src = xd
+        for li, L in enumerate(layers):
+            dst = logits if L["kind"] == "fc" else bufs[li & 1]
+            evs[li].record()
+            net.run_layer_cm(li, src, dst, batch)
+            src = dst
+        evs[len(layers)].record()
+        evs[len(layers)].synchronize()
+        if rep >= 2:
+            for li in range(len(layers)):
+                samples[li].append(evs[li].elapsed_time(evs[li + 1]) * 1e-3)
+    return [float(np.median(v)) for v in samples]
+
+
 def max_over_ranks(values, world, device="cpu"):
     """Element-wise maximum of per-rank timings over the process group (the job is as slow as its slowest replica)."""
     if world <= 1:
@@ -290,15 +313,22 @@ def run_gpu(args, rank, world, local_rank):
     # per-layer timings for the roofline of the dominant kernel (the group-sparse 1x1)
     flush = torch.zeros(64 * 1024 * 1024, device="cuda")     # 256 MB > L2
     per = time_layers(sbnn, torch, net, layers, batch, args.layer_reps, flush)
+    chain_t = time_layers_in_chain(sbnn, torch, net, layers, batch, xd, max(args.layer_reps, 5))
+    for r, t in zip(per, chain_t):
+        r["s_cold"], r["s"] = r["s"], t          # the roofline uses the in-step durations; the cold ones are reported beside
     hbm_gbs, peak_kind = measured_peaks()
     pw = [r for r in per if r["kind"] == "pw"]
     pw_t, pw_fl, pw_by = sum(r["s"] for r in pw), sum(r["flops"] for r in pw), sum(r["bytes"] for r in pw)
+    pw_t_cold = sum(r["s_cold"] for r in pw)
     t_roof = lambda r: max(r["flops"] / (FP32_PEAK_TFLOPS * 1e12), r["bytes"] / (hbm_gbs * 1e9))  # noqa: E731
     total_layer_t = sum(r["s"] for r in per)
     roofline = {
         "bound": "alu", "kernel": "conv1x1_cm_kernel (13 pointwise launches per step)",
         "achieved": pw_fl / pw_t / 1e12, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s",
         "frac": pw_fl / pw_t / 1e12 / FP32_PEAK_TFLOPS,
+        "timing": "CUDA events between the consecutive launches of a step (forward's order and buffers, no flush)",
+        "frac_cold": pw_fl / pw_t_cold / 1e12 / FP32_PEAK_TFLOPS,
+        "frac_cold_note": "each layer launched alone after a 256 MB write has flushed L2",
         "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz (no measured FP32 peak on file)",
         # dram__bytes_read.sum + dram__bytes_write.sum of the 13 launches of one step from the ncu capture in
         # profiles/bench_mobilenet_v1_b64_s50_launch_list.md; valid for the default workload and this kernel only
@@ -310,7 +340,7 @@ def run_gpu(args, rank, world, local_rank):
         "share_of_step": pw_t / total_layer_t,
         "whole_chain_frac": sum(t_roof(r) for r in per) / total_layer_t,
     }
-    layers_out = [{"name": r["name"], "us": round(r["s"] * 1e6, 2), "tflops": round(r["flops"] / r["s"] / 1e12, 2),
+    layers_out = [{"name": r["name"], "us": round(r["s"] * 1e6, 2), "us_cold": round(r["s_cold"] * 1e6, 2), "tflops": round(r["flops"] / r["s"] / 1e12, 2),
                    "gbs": round(r["bytes"] / r["s"] / 1e9, 1), "frac": round(t_roof(r) / r["s"], 3)} for r in per]
 
     cpu = cpu_baseline(x, layers) if world == 1 and not args.no_cpu else None
@@ -324,7 +354,8 @@ def run_gpu(args, rank, world, local_rank):
                                f"group-sparse G=4 at {args.sparsity}% (balanced random masks), rest dense",
                    "global_batch": batch * world, "parallelism": f"batch-sharded replicas x{world}, no collective",
                    "l2": "one step streams about 2.6 GB of activations through two ping-pong buffers (far above the "
-                         "126 MB L2); per-layer timings flush L2 with a 256 MB write before every launch"},
+                         "126 MB L2); per-layer timings: in step order without a flush (roofline), and alone after a 256 MB "
+                         "write has flushed L2 (us_cold)"},
         "effective_gflops_nonzero": sum(r["flops"] for r in per) / (elapsed / args.steps) / 1e9,
         "e2e": {"value": imgs / e2e_elapsed, "unit": "images/s", "h2d_bytes_per_step": int(x.nbytes),
                 "d2h_bytes_per_step": int(batch * 1000 * 4)},
