@@ -217,6 +217,23 @@ def time_layers_in_chain(sbnn, torch, net, layers, batch, xd, reps):
     return [float(np.median(v)) for v in samples]
 
 
+def sweep_oracle_lines():
+    """The oracle timed on the host cores for each distinct single-layer shape of the sweep (it does not skip zeros,
+    so sparsity and G do not change its work): one warm-up, one timed run, on a bounded number of images and scaled
+    to the configuration's batch.  A baseline beside the GPU lines, nothing more."""
+    from oracle import reference as R
+    from sbnn_inputs import workloads as WL
+    cases = [("config1", WL.config1(), 1, 1), ("config4", WL.config4(n=4), 4, 32),
+             ("config5", WL.config5(4, 50, n=8), 8, 256)]
+    for name, d, n_timed, n_full in cases:
+        for rep in range(2):
+            t0 = time.perf_counter()
+            R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+            dt = time.perf_counter() - t0
+        print(json.dumps({"case": name, "impl": "oracle (fp64, dense over masked weights)", "cores": R.num_threads(),
+                          "sample": f"{n_timed} of {n_full} images, scaled", "us": dt * 1e6 * n_full / n_timed}), flush=True)
+
+
 def max_over_ranks(values, world, device="cpu"):
     """Element-wise maximum of per-rank timings over the process group (the job is as slow as its slowest replica)."""
     if world <= 1:
@@ -390,6 +407,8 @@ def main():
     if args.sweep:
         from paper_2310_19509_b200 import sweep
         sweep.main()
+        if rank == 0 and not args.no_cpu:
+            sweep_oracle_lines()
         return
     run_gpu(args, rank, world, local_rank)
 
