@@ -22,6 +22,7 @@
 // makes warps with fewer kept channels in a step wait for the others (two stages, bounded waits).  The
 // weight stream holds, per 16 kept channels, 16 row offsets and the B fragments in register order.
 #include <cuda_bf16.h>
+#include <stdint.h>
 #include <string.h>
 
 #include <algorithm>
@@ -126,8 +127,8 @@ conv1x1_bf16_kernel(const __grid_constant__ MapB xmap, float* __restrict__ Y, co
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
             const int c0 = n * 8 + 2 * tq;
-            const float b0 = (g < ngroups && c0 < G) ? bias[g * G + c0] : 0.f;
-            const float b1 = (g < ngroups && c0 + 1 < G) ? bias[g * G + c0 + 1] : 0.f;
+            const float b0 = (g < ngroups && c0 < G && g * G + c0 < Cout) ? bias[g * G + c0] : 0.f;
+            const float b1 = (g < ngroups && c0 + 1 < G && g * G + c0 + 1 < Cout) ? bias[g * G + c0 + 1] : 0.f;
 #pragma unroll
             for (int pb = 0; pb < 8; ++pb) {
                 acc[q][n][pb][0] = b0; acc[q][n][pb][1] = b1; acc[q][n][pb][2] = b0; acc[q][n][pb][3] = b1;
@@ -183,9 +184,15 @@ conv1x1_bf16_kernel(const __grid_constant__ MapB xmap, float* __restrict__ Y, co
                     if (m >= M) continue;
                     float v0 = acc[q][n][pb][2 * h], v1 = acc[q][n][pb][2 * h + 1];
                     if (relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
-                    float* yp = Y + (size_t)m * Cout + g * G + c0;
-                    if (G >= 2) *reinterpret_cast<float2*>(yp) = make_float2(v0, v1);
-                    else yp[0] = v0;
+                    const int ch = g * G + c0;                      // merged groups may reach past Cout
+                    if (ch >= Cout) continue;
+                    float* yp = Y + (size_t)m * Cout + ch;
+                    if (G >= 2 && ch + 1 < Cout && (Cout & 1) == 0) {
+                        *reinterpret_cast<float2*>(yp) = make_float2(v0, v1);
+                    } else {
+                        yp[0] = v0;
+                        if (G >= 2 && ch + 1 < Cout) yp[1] = v1;
+                    }
                 }
         }
     }
@@ -224,7 +231,59 @@ uint16_t bf16_bits(float f) {
 // Stream: block (tile t, step k) = GT (start, blocks) pairs, then per group its 16-channel blocks:
 // 16 byte offsets of the channels' shared-memory rows, then per N-tile the B fragment of m16n8k16 in
 // register order (lane l: {B[2t][g], B[2t+1][g]}, {B[2t+8][g], B[2t+9][g]}, g = l/4, t = l%4).
-sbnn_status build_stream_bf16(const sbnn_packed* p, StreamBf16* out) {
+// The layer as the kernel sees it.  An MMA has 8 output columns, so groups of fewer than 8 channels are merged, 8 / G
+// neighbours at a time, into one group of 8 whose kept set is the union of theirs and whose weights are zero where a
+// member does not keep the channel: one activation fragment then serves all 8 columns instead of leaving most of
+// them as padding (G = 4, dense: half the MMAs and fragment loads).
+struct LayerView {
+    int G = 0, ngroups = 0;
+    std::vector<int32_t> group_ptr, idx;
+    std::vector<float> val;
+};
+
+LayerView view_for_mma(const sbnn_packed* p) {
+    LayerView v;
+    if (p->G >= 8) {
+        v.G = p->G; v.ngroups = p->ngroups; v.group_ptr = p->group_ptr; v.idx = p->idx; v.val = p->val;
+        return v;
+    }
+    const int G = p->G, per = 8 / G;
+    v.G = 8;
+    v.ngroups = (p->ngroups + per - 1) / per;
+    v.group_ptr.assign(v.ngroups + 1, 0);
+    std::vector<int32_t> pos(per);
+    for (int sg = 0; sg < v.ngroups; ++sg) {
+        const int g0 = sg * per, g1 = std::min(p->ngroups, g0 + per);
+        for (int g = g0; g < g1; ++g) pos[g - g0] = p->group_ptr[g];
+        for (;;) {                                                   // merge the members' ascending lists
+            int32_t c = INT32_MAX;
+            for (int g = g0; g < g1; ++g)
+                if (pos[g - g0] < p->group_ptr[g + 1]) c = std::min(c, p->idx[pos[g - g0]]);
+            if (c == INT32_MAX) break;
+            v.idx.push_back(c);
+            const size_t base = v.val.size();
+            v.val.resize(base + 8, 0.0f);
+            for (int g = g0; g < g1; ++g)
+                if (pos[g - g0] < p->group_ptr[g + 1] && p->idx[pos[g - g0]] == c) {
+                    for (int r = 0; r < G; ++r) v.val[base + (size_t)(g - g0) * G + r] = p->val[(size_t)pos[g - g0] * G + r];
+                    ++pos[g - g0];
+                }
+        }
+        v.group_ptr[sg + 1] = (int32_t)v.idx.size();
+    }
+    return v;
+}
+
+sbnn_status build_stream_bf16(const sbnn_packed* pk, StreamBf16* out) {
+    LayerView lv;
+    try {
+        lv = view_for_mma(pk);
+    } catch (const std::bad_alloc&) {
+        return fail(SBNN_ERR_ALLOC, "out of host memory building the bf16 weight stream");
+    }
+    struct { int G, ngroups, Cin; std::vector<int32_t>&group_ptr, &idx; std::vector<float>& val; }
+        view{lv.G, lv.ngroups, pk->Cin, lv.group_ptr, lv.idx, lv.val};
+    auto* p = &view;
     const int G = p->G, NT8 = (G + 7) / 8, GT = NWARP * (G <= 8 ? 2 : 1), BLK = 4 + NT8 * 16;
     const int ntiles = (p->ngroups + GT - 1) / GT, nchunks = (p->Cin + KC - 1) / KC;
     const int HDR = (GT * 2 + 3) / 4;
@@ -318,7 +377,8 @@ sbnn_status build_stream_bf16(const sbnn_packed* p, StreamBf16* out) {
 }
 
 template <int G>
-sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, const float* x, float* y, int M, int relu, cudaStream_t st) {
+sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, int ngroups, const float* x, float* y, int M, int relu,
+                        cudaStream_t st) {
     constexpr int GPW = (G <= 8) ? 2 : 1;
     // bf16 channel-major copy of X in the per-device scratch buffer; rows padded to whole pixel tiles
     const int ldb = (M + TM - 1) / TM * TM;
@@ -347,7 +407,7 @@ sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, const float* 
     const long long nblk = (long long)(ldb / TM) * s.ntiles;
     if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
     conv1x1_bf16_kernel<G, GPW><<<(unsigned)nblk, (NWARP + 1) * 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin,
-                                                                                p->Cout, p->ngroups, s.nchunks, s.ntiles, s.max_blk,
+                                                                                p->Cout, ngroups, s.nchunks, s.ntiles, s.max_blk,
                                                                                 S, stage_bytes, relu, status);
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
@@ -372,11 +432,11 @@ sbnn_status conv1x1_bf16(const sbnn_packed* p, const float* x, float* y, int M, 
         s = static_cast<StreamBf16*>(p->bf16_stream);
     }
     switch (p->G) {
-        case 1: return launch_bf16<1>(p, *s, x, y, M, relu, st);
-        case 2: return launch_bf16<2>(p, *s, x, y, M, relu, st);
-        case 4: return launch_bf16<4>(p, *s, x, y, M, relu, st);
-        case 8: return launch_bf16<8>(p, *s, x, y, M, relu, st);
-        default: return launch_bf16<16>(p, *s, x, y, M, relu, st);
+        case 16: return launch_bf16<16>(p, *s, p->ngroups, x, y, M, relu, st);
+        default: {   // G <= 8: groups merged into groups of 8 output channels (see view_for_mma)
+            const int per = 8 / p->G;
+            return launch_bf16<8>(p, *s, (p->ngroups + per - 1) / per, x, y, M, relu, st);
+        }
     }
 }
 

@@ -449,6 +449,16 @@ def test_bf16_tensor_core_mode(g):
         assert_within(y, ref, s, tol=1e-2, what=f"bf16 G={g} relu={relu} vs fp32 oracle")
 
 
+@pytest.mark.parametrize("g,cout", [(4, 12), (2, 6), (1, 5), (1, 16), (2, 22)])
+def test_bf16_mode_merged_groups_ragged_channel_count(g, cout):
+    """Groups of fewer than 8 channels are merged into 8-column groups for the tensor cores; the last merged group
+    may reach past Cout, and an odd Cout forces scalar stores."""
+    d = WL.single_conv_inputs(1, 5, 37, 72, cout, 1, g, 50, seed=13, mask_mode="layer_global")
+    y = run_1x1(d, sbnn.SBNN_BF16_TC | sbnn.SBNN_RELU)
+    ref16, s16 = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True, bf16=True)
+    assert_within(y, ref16, s16, tol=1e-5, what=f"bf16 merged G={g} Cout={cout}")
+
+
 def test_bf16_mode_on_config5_shape_reduced_batch():
     d = WL.config5(8, 50, n=6)
     y = run_1x1(d, sbnn.SBNN_BF16_TC | sbnn.SBNN_RELU)
