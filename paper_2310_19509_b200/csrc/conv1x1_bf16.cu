@@ -12,7 +12,7 @@
 // (arbitrary) channel.  So one `ldmatrix.x4.trans` with gathered row addresses yields the 16x16 A
 // fragment of an m16n8k16 MMA at 4 shared-memory wavefronts per 2048 MACs, against 9 per 1024 in
 // the fp32 kernel.  The N = 8 columns of the MMA are the group's output channels (G = 8 fills them,
-// G = 4 uses half, G = 16 takes two MMAs per A fragment).
+// G = 16 takes two MMAs per A fragment, smaller groups are merged into 8-column groups at pack time).
 //
 // CTA = 128 pixels x 8 warps; a warp owns GPW groups over all 128 pixels (8 row blocks of 16), i.e.
 // 32 fp32 accumulators per N-tile.  A pre-pass converts X once to bf16 in channel-major order
