@@ -8,7 +8,7 @@ import pytest
 import torch
 
 from oracle import reference as R
-from sbnn_inputs import expand_mask, group_mask_balanced
+from sbnn_inputs import dw_pattern_mask, expand_mask, group_mask_balanced, tap_pattern_mask
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
 rng = np.random.default_rng(1234)
@@ -186,6 +186,51 @@ def test_p4_pack_rejects_non_uniform_mask():
     m3[0:4, 1, 1, 2] = 0        # one tap removed for a whole group: not a whole-kernel mask
     with pytest.raises(R.MaskNotGroupUniform):
         R.pack(np.ones((8, 3, 3, 8), np.float32), m3, 4)
+
+
+def test_p4_pattern_packers_reconstruct_the_masked_weights():
+    """The two pattern formats, checked by writing the dense masked weights back out of them by hand (not through
+    the oracle's own unpack): kernel patterns of a 3x3 layer, and the 3:9 patterns of depthwise weights; the
+    convolution with the reconstructed weights is the masked convolution."""
+    g, cin, cout = 4, 10, 8
+    wt = rng.standard_normal((cout, 3, 3, cin)).astype(np.float32)
+    um = rng.random((cout // g, cin)) < 0.6
+    m = tap_pattern_mask(5, 19, um, g, 4)
+    assert np.all(m.reshape(cout // g, g, 9, cin).sum(axis=2)[:, 0][um] == 4) and np.all(m[:, 1, 1].reshape(cout // g, g, cin)[:, 0] == um)
+    gp, idx, val, tm = R.pack_pattern(wt, m, g)
+    dense = np.zeros_like(wt)
+    for gi in range(cout // g):
+        for u in range(gp[gi], gp[gi + 1]):
+            for t in range(9):
+                kept = (int(tm[u]) >> t) & 1
+                assert kept or not val[u, t].any()                      # pruned taps are stored as zeros
+                dense[gi * g:(gi + 1) * g, t // 3, t % 3, idx[u]] = val[u, t]
+                assert np.all(m[gi * g:(gi + 1) * g, t // 3, t % 3, idx[u]] == kept)
+    assert np.array_equal(dense, wt * m) and gp[-1] == um.sum()
+    x = rng.standard_normal((1, 4, 5, cin)).astype(np.float32)
+    a, _ = R.conv2d(x, wt, m, None, relu=False)
+    b, _ = R.conv2d(x, dense, np.ones_like(m), None, relu=False)
+    assert np.array_equal(a, b)
+
+    c, go = 32, 8
+    wd = rng.standard_normal((3, 3, c)).astype(np.float32)
+    md = dw_pattern_mask(5, 7, c, go, wd)
+    pat, w6 = R.pack_dw_pattern(wd, md, go)
+    dd = np.zeros_like(wd)
+    for blk in range(c // go):
+        sl = slice(blk * go, (blk + 1) * go)
+        for kh in range(3):
+            third_pruned = (int(pat[blk]) >> kh) & 1
+            dd[kh, 0 if third_pruned else 2, sl] = w6[kh, 0, sl]
+            dd[kh, 1, sl] = w6[kh, 1, sl]
+            # the l1 rule: the kept side is the heavier one over the block
+            l1 = np.abs(wd[kh, :, sl].astype(np.float64)).sum(axis=1)
+            assert (l1[0] >= l1[2]) == bool(third_pruned)
+    assert np.array_equal(dd, wd * md) and np.all(md.sum(axis=(0, 1)) == 6)
+    with pytest.raises(R.MaskNotGroupUniform):
+        bad = md.copy()
+        bad[0, 0, 0] ^= 1
+        R.pack_dw_pattern(wd, bad, go)
 
 
 def test_p5_mobilenet_mac_counts_match_table3():
