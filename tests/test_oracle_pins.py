@@ -287,3 +287,116 @@ def test_sample_outputs_agrees_with_the_full_loops():
     r2, s2 = R.sample_outputs(x, wt, m, b, pos, relu=True)
     for i, (n, y, xx, o) in enumerate(pos):
         assert abs(r2[i] - ref[n, y, xx, o]) < 1e-12 and abs(s2[i] - s[n, y, xx, o]) < 1e-12
+
+
+# ---------------------------------------------------------------------------
+# The chained MobileNet-v1 oracle (all 29 table entries) against an independent chain built here from
+# torch's fp64 library convolution and mean, and its propagated bound E pinned from below and from above.
+# ---------------------------------------------------------------------------
+
+def _torch_layer(L, cur, tol_sign=None, tol=1e-5):
+    """One layer of the network from library routines in fp64: NHWC in, (out, S) NHWC out.  Pointwise weights are
+    multiplied by their mask; ReLU after every convolution but the classifier; the pool is a plain mean."""
+    import torch.nn.functional as F
+    kind = L["kind"]
+    t = torch.from_numpy(np.ascontiguousarray(cur, dtype=np.float64)).permute(0, 3, 1, 2)
+    if kind == "pool":
+        out = t.mean(dim=(2, 3), keepdim=True)
+        s = t.abs().mean(dim=(2, 3), keepdim=True)
+        return out.permute(0, 2, 3, 1).numpy(), s.permute(0, 2, 3, 1).numpy()
+    b = torch.from_numpy(L["bias"].astype(np.float64))
+    if kind == "dw":
+        w = torch.from_numpy(L["w"].astype(np.float64)).permute(2, 0, 1).unsqueeze(1)          # [C][1][3][3]
+        conv = lambda a, ww, bb: F.conv2d(a, ww, bb, stride=L["stride"], padding=1, groups=a.shape[1])  # noqa: E731
+    else:
+        wm = L["w"].astype(np.float64)
+        if "mask" in L:
+            wm = wm * L["mask"]
+        w = torch.from_numpy(wm).permute(0, 3, 1, 2)                                           # [Cout][Cin][KH][KW]
+        pad = (w.shape[2] - 1) // 2
+        conv = lambda a, ww, bb: F.conv2d(a, ww, bb, stride=L["stride"], padding=pad)          # noqa: E731
+    out = conv(t, w, b)
+    s = conv(t.abs(), w.abs(), b.abs())
+    if kind != "fc":
+        out = out.clamp_min(0)
+    return out.permute(0, 2, 3, 1).numpy(), s.permute(0, 2, 3, 1).numpy()
+
+
+def _small_network(seed, side=64, sparsity=50):
+    """MobileNet-v1's 29 table entries on a side x side crop (the shapes scale with the image; 64 leaves a 2x2 map
+    for the pool to average)."""
+    from sbnn_inputs import mobilenet_v1_inputs
+    x, layers = mobilenet_v1_inputs(1, sparsity, 4, seed=seed)
+    return np.ascontiguousarray(x[:, :side, :side]), layers
+
+
+def test_chain_every_layer_against_an_independent_fp64_chain():
+    x, layers = _small_network(seed=3)
+    outs = R.mobilenet_v1_forward(x, layers)
+    assert [o["name"] for o in outs] == [L["name"] for L in layers] and len(outs) == 29
+    # (i) layer by layer on the oracle's own fp32 inputs: value and S, tightly
+    for L, rec in zip(layers, outs):
+        ref, s = _torch_layer(L, rec["in"])
+        assert rec["ref"].shape == ref.shape, L["name"]
+        np.testing.assert_allclose(rec["ref"], ref, rtol=0, atol=1e-11 * float(np.max(s)), err_msg=L["name"])
+        np.testing.assert_allclose(rec["S"], s, rtol=1e-12, atol=1e-300, err_msg=L["name"])
+    # (ii) the chaining itself: each layer is fed the fp32 rounding of the previous result
+    for prev, rec in zip(outs, outs[1:]):
+        assert rec["in"].dtype == np.float32
+        np.testing.assert_array_equal(rec["in"].reshape(-1), prev["ref"].astype(np.float32).reshape(-1))
+    # (iii) a chain that never looks at the oracle's intermediates ends at the same logits (fp32 rounding between
+    # layers may flip a last bit here and there, hence the looser comparison)
+    cur = x
+    for L in layers:
+        cur = _torch_layer(L, cur)[0].astype(np.float32)
+    assert cur.shape == (1, 1, 1, 1000) == outs[-1]["ref"].shape
+    scale = float(np.max(np.abs(outs[-1]["ref"])))
+    assert scale > 1e-3
+    np.testing.assert_allclose(cur.astype(np.float64), outs[-1]["ref"], rtol=0, atol=2e-5 * scale)
+    # the classifier has no ReLU (negative logits exist), the pool no ReLU either and it does average
+    assert (outs[-1]["ref"] < 0).any()
+    pool_in = outs[27]["in"].astype(np.float64)
+    np.testing.assert_allclose(outs[27]["ref"].reshape(-1), pool_in.reshape(4, 1024).mean(axis=0), rtol=1e-13)
+
+
+def _perturbed_chain(x, layers, tol, sign_of):
+    """The independent fp64 chain with every layer's result moved by sign * tol * S (an implementation that uses
+    its whole per-layer allowance).  No fp32 rounding between layers: E allows for that separately."""
+    cur = x.astype(np.float64)
+    for li, L in enumerate(layers):
+        out, s = _torch_layer(L, cur)
+        cur = out + sign_of(li, out.shape) * tol * s
+    return cur
+
+
+def test_chain_error_bound_is_pinned_from_both_sides():
+    tol = 1e-5
+    # (a) nonnegative weights, biases and image: every ReLU is active and nothing cancels, so a chain that errs by
+    # +tol*S at every layer deviates by exactly the first-order bound; E must cover it and may not be much larger
+    x, layers = _small_network(seed=4)
+    pos = []
+    for L in layers:
+        L = dict(L)
+        for k in ("w", "bias"):
+            if k in L:
+                L[k] = np.abs(L[k])
+        pos.append(L)
+    outs = R.mobilenet_v1_forward(x, pos, tol=tol)
+    dev = _perturbed_chain(x, pos, tol, lambda li, shape: 1.0) - outs[-1]["ref"]
+    e = outs[-1]["E"]
+    assert np.all(dev > 0) and np.all(dev <= e)
+    assert np.all(e <= 1.02 * dev), float(np.max(e / dev))       # slack: E also allows for rounding activations to fp32
+    for rec in outs:                                             # and at every layer on the way
+        assert np.all(rec["E"] >= tol * rec["S"])
+    # (b) the network as generated (signed weights), errors of random sign and of one sign: inside E
+    x, layers = _small_network(seed=5)
+    outs = R.mobilenet_v1_forward(x, layers, tol=tol)
+    r = np.random.default_rng(77)
+    for sign_of in (lambda li, shape: 1.0, lambda li, shape: -1.0,
+                    lambda li, shape: r.choice([-1.0, 1.0], size=shape)):
+        dev = np.abs(_perturbed_chain(x, layers, tol, sign_of) - outs[-1]["ref"])
+        assert np.all(dev <= outs[-1]["E"])
+    # E scales with the per-layer tolerance (up to the fixed fp32-rounding allowance)
+    outs10 = R.mobilenet_v1_forward(x, layers, tol=10 * tol)
+    ratio = outs10[-1]["E"] / outs[-1]["E"]
+    assert np.all(ratio > 9.0) and np.all(ratio <= 10.0 + 1e-9)
