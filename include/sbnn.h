@@ -18,8 +18,15 @@
  *     memory of the current CUDA device, 16-byte aligned, owned by the caller.
  *     Input and output buffers must not overlap.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default
- *     stream).  Compute calls only enqueue kernels on it and return; they never
- *     synchronise.  Calls that create, pack or free objects may synchronise.
+ *     stream).  Calls that create, pack, prepare or free objects may allocate and
+ *     synchronise.  A compute call only enqueues kernels on the stream and returns,
+ *     provided sbnn_prepare has been called for the layer with a shape at least as
+ *     large (sbnn_mobilenet_v1_create does the same for the chain); without it, the
+ *     first call of a layer at a new shape or in a new mode may build a private
+ *     weight layout or grow the per-device scratch buffer, both synchronously.
+ *   - Packed layers and networks belong to the device that was current when they were
+ *     packed / created; a compute call made while another device is current returns
+ *     SBNN_ERR_CUDA.
  *   - Every function returns an sbnn_status; nothing throws, aborts or exits.
  *     On error no kernel is launched.  sbnn_last_error() gives a thread-local
  *     one-line explanation of the most recent failure.
@@ -118,6 +125,21 @@ SBNN_API sbnn_status sbnn_packed_get(const sbnn_packed* p, sbnn_packed_view* vie
 SBNN_API sbnn_status sbnn_unpack_weights(const sbnn_packed* p, float* W_host_out, uint8_t* mask_host_out);
 /* Frees host and device copies.  NULL is accepted. */
 SBNN_API sbnn_status sbnn_packed_free(sbnn_packed* p);
+
+/*
+ * Set-up step of the engine for one layer (Section 3.5: the model is converted once, ahead of inference):
+ * does now everything that sbnn_conv1x1_gs / sbnn_conv1x1_gs_cm (KH = 1) or sbnn_conv3x3_gs (KH = 3) would
+ * otherwise do on first use for activations of up to N x H x W pixels with these flags -- builds the kernels'
+ * private weight layouts (for the 1x1 case those of every tile shape the library may choose, whatever the
+ * pixel count), raises the kernels' shared-memory limits, and grows the per-device scratch buffer to what
+ * the NHWC entry points need for this shape (with SBNN_BF16_TC: what the bf16 mode needs).  Allocates and
+ * may synchronise; launches nothing; the activation buffers need not exist yet.  Afterwards compute calls of
+ * this layer with no more pixels (3x3: the same W) only enqueue.  Call it once per layer and mode, outside
+ * any stream capture.  The scratch buffer never shrinks and an outgrown one is kept until the process exits,
+ * so a CUDA graph recorded over an entry point stays valid when a later, larger call makes the buffer grow;
+ * growth during a capture is refused with SBNN_ERR_UNSUPPORTED.
+ */
+SBNN_API sbnn_status sbnn_prepare(const sbnn_packed* w, int N, int H, int W, int flags);
 
 /* ------------------------------------------------------------------------------------------------
  * Group-sparse convolutions (Algorithm 1 for the 1x1 case; Section 3.2's connectivity group
@@ -345,6 +367,23 @@ SBNN_API sbnn_status sbnn_get_async_status(void* cuda_stream);
  * SBNN_ERR_TIMEOUT once (the word is cleared by that call) and the context stays usable.
  */
 SBNN_API sbnn_status sbnn_selftest_wait_timeout(void* cuda_stream);
+
+/*
+ * Diagnostic for the roofline of the arithmetic-bound kernels (the paper gives no counterpart: it quotes
+ * latencies only, Tables 3 and 4): enqueues a kernel in which 4 CTAs of 512 threads per SM each run
+ * `iterations` rounds of 32 packed fp32 FMAs (fma.rn.f32x2, the instruction the convolution kernels use) on
+ * registers only, and writes to *flop_out (host, may be NULL) the floating-point operations it performs.
+ * Timing it with events on `cuda_stream` gives the FP32 rate this GPU sustains at its current clocks.
+ */
+SBNN_API sbnn_status sbnn_selftest_fma_rate(int iterations, double* flop_out, void* cuda_stream);
+
+/*
+ * Test hook: overwrite the device number recorded in a packed layer, so that the refusal of compute calls
+ * on weights that live on another device can be exercised on a machine with a single GPU.  Not for
+ * production use: the device copies themselves do not move.  *previous (may be NULL) receives the number that
+ * was recorded, so the test can put it back before freeing the layer.
+ */
+SBNN_API sbnn_status sbnn_debug_set_packed_device(sbnn_packed* w, int device, int* previous);
 
 #ifdef __cplusplus
 }

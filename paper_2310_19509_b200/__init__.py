@@ -28,6 +28,9 @@ from .binding import (  # noqa: F401
     mobilenet_v1_layer_shape,
     pack_dw_pattern,
     pack_weights,
+    prepare,
+    selftest_fma_rate,
+    debug_set_packed_device,
     selftest_wait_timeout,
     status_str,
     to_channel_major,

@@ -64,6 +64,9 @@ def lib():
         "sbnn_get_async_status": [P],
         "sbnn_head_noalloc": [P, P, P, I, I, P],
         "sbnn_selftest_wait_timeout": [P],
+        "sbnn_prepare": [P, I, I, I, I],
+        "sbnn_selftest_fma_rate": [I, P, P],
+        "sbnn_debug_set_packed_device": [P, I, P],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -222,6 +225,25 @@ def avgpool(x, y, n, hw, c, stream=None):
 def head_noalloc(fc: Packed, x, logits, n, hw, stream=None):
     """Average pool + classifier through the library's fixed scratch array; allocates nothing."""
     _check(lib().sbnn_head_noalloc(fc.handle, _ptr(x), _ptr(logits), n, hw, _stream(stream)))
+
+
+def prepare(w: Packed, n, h, wd, flags=0):
+    """Build ahead of time what compute calls of this layer would build on first use (see sbnn_prepare)."""
+    _check(lib().sbnn_prepare(w.handle, n, h, wd, flags))
+
+
+def selftest_fma_rate(iterations, stream=None) -> float:
+    """Enqueue the register-only packed-FMA kernel; returns the flop it performs (time it with events)."""
+    flop = C.c_double()
+    _check(lib().sbnn_selftest_fma_rate(int(iterations), C.byref(flop), _stream(stream)))
+    return flop.value
+
+
+def debug_set_packed_device(w: Packed, device) -> int:
+    """Test hook: overwrite the device recorded in a packed layer; returns the previous value."""
+    prev = C.c_int()
+    _check(lib().sbnn_debug_set_packed_device(w.handle, int(device), C.byref(prev)))
+    return prev.value
 
 
 def selftest_wait_timeout(stream=None):

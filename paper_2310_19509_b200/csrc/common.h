@@ -22,6 +22,17 @@ sbnn_status check_device();
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// True while the calling thread is inside sbnn_prepare: the entry points then run their whole host path (private
+// weight layouts, scratch sizing, kernel attributes) but enqueue nothing and touch neither x_dev nor y_dev.
+bool prepare_only();
+struct PrepareScope {
+    PrepareScope();
+    ~PrepareScope();
+};
+
+// Raises a kernel's dynamic shared-memory limit to `bytes` on the current device, once per (device, kernel) and size.
+sbnn_status set_max_dyn_smem(const void* func, int bytes);
+
 #define SBNN_CUDA_TRY(expr)                                                                         \
     do {                                                                                            \
         cudaError_t e__ = (expr);                                                                   \
@@ -85,6 +96,8 @@ struct sbnn_packed {
 };
 
 namespace sbnn {
+// SBNN_OK if `w` has device copies and they live on the current device (else SBNN_ERR_CUDA, nothing is launched).
+sbnn_status check_packed_device(const sbnn_packed* w);
 // conv1x1_gs.cu
 sbnn_status prepare_default_1x1(const sbnn_packed* p);
 void free_streams_1x1(sbnn_packed* p);
@@ -103,8 +116,10 @@ sbnn_status async_status_word(int** out);
 // copied per dimension.  Elements outside the tensor are delivered as zeros.
 sbnn_status encode_tiled_map(void* out, const void* base, int elem_bytes, int rank, const unsigned long long* dims,
                              const unsigned long long* strides_bytes, const unsigned* box);
-// Per-device scratch buffer for channel-major copies made on behalf of NHWC callers (grows on demand, synchronously).
-sbnn_status scratch_workspace(size_t bytes, float** out);
+// Per-device scratch buffer for channel-major copies made on behalf of NHWC callers.  Grows on demand with a
+// synchronous allocation (the outgrown buffer is kept until the process exits, so work already enqueued or recorded
+// on it stays valid); growth while `st` is being captured is refused with SBNN_ERR_UNSUPPORTED.
+sbnn_status scratch_workspace(size_t bytes, cudaStream_t st, float** out);
 // cm_layers.cu: dense layers on channel-major activations ([C][ld]); arguments validated by the callers
 sbnn_status launch_transpose(const float* in, int ld_in, float* out, int ld_out, int R, int Ccols, cudaStream_t st);
 sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, int ldx, float* y, int ldy, int N, int H,

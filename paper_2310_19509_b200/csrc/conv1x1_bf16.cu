@@ -383,12 +383,14 @@ sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, int ngroups, 
     // bf16 channel-major copy of X in the per-device scratch buffer; rows padded to whole pixel tiles
     const int ldb = (M + TM - 1) / TM * TM;
     float* scratch = nullptr;
-    sbnn_status r = scratch_workspace((size_t)p->Cin * ldb * sizeof(__nv_bfloat16), &scratch);
+    sbnn_status r = scratch_workspace((size_t)p->Cin * ldb * sizeof(__nv_bfloat16), st, &scratch);
     if (r != SBNN_OK) return r;
     __nv_bfloat16* xb = reinterpret_cast<__nv_bfloat16*>(scratch);
-    dim3 tg((ldb + 31) / 32, (p->Cin + 31) / 32);
-    to_channel_major_bf16_kernel<<<tg, 256, 0, st>>>(x, xb, M, p->Cin, ldb);
-    SBNN_CUDA_TRY(cudaGetLastError());
+    if (!prepare_only()) {
+        dim3 tg((ldb + 31) / 32, (p->Cin + 31) / 32);
+        to_channel_major_bf16_kernel<<<tg, 256, 0, st>>>(x, xb, M, p->Cin, ldb);
+        SBNN_CUDA_TRY(cudaGetLastError());
+    }
 
     const int stage_bytes = (STAGE_X + s.max_blk * 16 + 127) / 128 * 128;
     // Two stages: with about 38 KB per stage that leaves room for two or three CTAs per SM, which measured faster
@@ -396,6 +398,8 @@ sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, int ngroups, 
     const int S = 2;
     const size_t smem = (size_t)S * stage_bytes + 2 * S * 8 + 16;
     if (smem > 200 * 1024) return fail(SBNN_ERR_UNSUPPORTED, "internal: bf16 tile needs %zu bytes of shared memory", smem);
+    if ((r = set_max_dyn_smem(reinterpret_cast<const void*>(&conv1x1_bf16_kernel<G, GPW>), (int)smem)) != SBNN_OK) return r;
+    if (prepare_only()) return SBNN_OK;
     MapB xmap;
     const unsigned long long dims[2] = {(unsigned long long)ldb, (unsigned long long)p->Cin};
     const unsigned long long strides[1] = {(unsigned long long)ldb * sizeof(__nv_bfloat16)};
@@ -403,7 +407,6 @@ sbnn_status launch_bf16(const sbnn_packed* p, const StreamBf16& s, int ngroups, 
     if ((r = encode_tiled_map(&xmap, xb, 2, 2, dims, strides, box)) != SBNN_OK) return r;
     int* status = nullptr;
     if ((r = async_status_word(&status)) != SBNN_OK) return r;
-    SBNN_CUDA_TRY(cudaFuncSetAttribute(conv1x1_bf16_kernel<G, GPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const long long nblk = (long long)(ldb / TM) * s.ntiles;
     if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
     conv1x1_bf16_kernel<G, GPW><<<(unsigned)nblk, (NWARP + 1) * 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin,

@@ -651,22 +651,13 @@ sbnn_status encode_x_map(const float* x, int ldx, int M, int Cin, int box_px, in
 template <class C>
 sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, int ldx, float* y, int ldy, int M,
                       int relu, bool out_cm, cudaStream_t st) {
-    static std::mutex mu;
-    static std::map<int, bool> configured;
-    {
-        std::lock_guard<std::mutex> lk(mu);
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (!configured[dev]) {
-            SBNN_CUDA_TRY(cudaFuncSetAttribute(conv1x1_cm_kernel<C, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
-            SBNN_CUDA_TRY(cudaFuncSetAttribute(conv1x1_cm_kernel<C, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM));
-            configured[dev] = true;
-        }
-    }
+    sbnn_status r = set_max_dyn_smem(reinterpret_cast<const void*>(&conv1x1_cm_kernel<C, false>), (int)C::SMEM);
+    if (r == SBNN_OK) r = set_max_dyn_smem(reinterpret_cast<const void*>(&conv1x1_cm_kernel<C, true>), (int)C::SMEM);
+    if (r != SBNN_OK) return r;
     if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
     int* status = nullptr;
-    sbnn_status r = status_word(&status);
-    if (r != SBNN_OK) return r;
+    if ((r = status_word(&status)) != SBNN_OK) return r;
+    if (prepare_only()) return SBNN_OK;
     const long long nblk = (long long)((M + C::TM - 1) / C::TM) * s.ntiles;
     if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
     const int total_tiles = (int)nblk;
@@ -758,13 +749,16 @@ bool few_tiles(const sbnn_packed* p, long long M) {
     return 2 * tiles < sm_count();
 }
 
-// Per-device scratch for the channel-major copy of X made on behalf of NHWC callers.  Grows on demand
-// (synchronously) and is kept until the process exits.
+// Per-device scratch for the channel-major copy of X made on behalf of NHWC callers.  Grows on demand with a
+// synchronous cudaMalloc; the outgrown buffer is parked, not freed, until the process exits: launches already
+// enqueued on it, and CUDA graphs a caller recorded over an entry point that uses it, keep reading valid memory.
+// (sbnn_prepare sizes it ahead of time, after which compute calls of no larger shape never get here to grow it.)
 struct Workspace {
     float* ptr = nullptr;
     size_t bytes = 0;
+    std::vector<float*> parked;
 };
-sbnn_status workspace(size_t bytes, float** out) {
+sbnn_status workspace(size_t bytes, cudaStream_t st, float** out) {
     static std::mutex mu;
     static std::map<int, Workspace> ws;
     int dev = 0;
@@ -772,10 +766,15 @@ sbnn_status workspace(size_t bytes, float** out) {
     std::lock_guard<std::mutex> lk(mu);
     Workspace& w = ws[dev];
     if (w.bytes < bytes) {
-        if (w.ptr) SBNN_CUDA_TRY(cudaFree(w.ptr));   // cudaFree waits for the launches that still use it
-        w.ptr = nullptr;
-        w.bytes = 0;
-        SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&w.ptr), bytes));
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (!prepare_only() && cudaStreamIsCapturing(st, &cs) != cudaSuccess) cudaGetLastError();
+        if (cs != cudaStreamCaptureStatusNone)
+            return fail(SBNN_ERR_UNSUPPORTED, "the scratch buffer must grow to %zu bytes, which cannot happen while the stream is "
+                        "being captured: call sbnn_prepare (or this entry point once) for this shape before capturing", bytes);
+        float* fresh = nullptr;
+        SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&fresh), bytes));
+        if (w.ptr) w.parked.push_back(w.ptr);
+        w.ptr = fresh;
         w.bytes = bytes;
     }
     *out = w.ptr;
@@ -784,7 +783,7 @@ sbnn_status workspace(size_t bytes, float** out) {
 
 }  // namespace
 
-sbnn_status scratch_workspace(size_t bytes, float** out) { return workspace(bytes, out); }
+sbnn_status scratch_workspace(size_t bytes, cudaStream_t st, float** out) { return workspace(bytes, st, out); }
 
 sbnn_status async_status_word(int** out) { return status_word(out); }
 
@@ -796,6 +795,24 @@ sbnn_status encode_tiled_map(void* out, const void* base, int elem_bytes, int ra
 sbnn_status prepare_default_cm(const sbnn_packed* p, long long M) {
     Stream1x1 s;
     return get_stream_cm(p, default_cfg_cm(p, M), &s);
+}
+
+sbnn_status prepare_all_cm(const sbnn_packed* p) {
+    // every tile shape default_cfg_cm can return for this layer's G and density
+    std::vector<TileCfg> all;
+    switch (p->G) {
+        case 1: all = {{8, 4, 8, 32}}; break;
+        case 2: all = {{8, 2, 8, 32}}; break;
+        case 4: all = {{8, 1, 16, 32}, {8, 2, 8, 32}, {8, 2, 11, 32}, {8, 2, 12, 32}}; break;
+        case 8: all = {{8, 1, 8, 32}, {8, 1, 12, 32}}; break;
+        default: all = {{4, 1, 8, 32}}; break;
+    }
+    PrepareScope scope;   // dispatch_cm then builds the stream and sets the kernel's attributes, and launches nothing
+    for (const TileCfg& c : all) {
+        sbnn_status r = dispatch_cm(p, c, nullptr, 0, nullptr, 0, 1, 0, false, nullptr);
+        if (r != SBNN_OK) return r;
+    }
+    return SBNN_OK;
 }
 
 sbnn_status prepare_cm(const sbnn_packed* p, int P, int GPW, int NW, int KC) {
@@ -826,11 +843,13 @@ sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M
     if (w->Cin < 128 || w->Cout < 64 || M < 2048) return SBNN_OK;
     const int ld = (M + 3) / 4 * 4;
     float* xt = nullptr;
-    sbnn_status r = workspace((size_t)w->Cin * ld * sizeof(float), &xt);
+    sbnn_status r = workspace((size_t)w->Cin * ld * sizeof(float), st, &xt);
     if (r != SBNN_OK) return r;
-    dim3 grid((M + 31) / 32, (w->Cin + 31) / 32);
-    to_channel_major_kernel<<<grid, 256, 0, st>>>(x, xt, M, w->Cin, ld);
-    SBNN_CUDA_TRY(cudaGetLastError());
+    if (!prepare_only()) {
+        dim3 grid((M + 31) / 32, (w->Cin + 31) / 32);
+        to_channel_major_kernel<<<grid, 256, 0, st>>>(x, xt, M, w->Cin, ld);
+        SBNN_CUDA_TRY(cudaGetLastError());
+    }
     r = dispatch_cm(w, default_cfg_cm(w, M), xt, ld, y, w->Cout, M, relu, false, st);
     if (r == SBNN_OK) *done = true;
     return r;
@@ -876,10 +895,10 @@ extern "C" sbnn_status sbnn_conv1x1_gs_cm(const sbnn_packed* w, const float* xt_
     if (out_cm ? (ldy < M || ldy % 4) : (ldy < w->Cout || ldy % 4))
         return fail(SBNN_ERR_SHAPE, "ldy=%d does not fit the output layout", ldy);
     if (!aligned16(xt_dev) || !aligned16(y_dev)) return fail(SBNN_ERR_ALIGN, "xt_dev and y_dev must be 16-byte aligned");
-    if (w->device < 0) return fail(SBNN_ERR_CUDA, "packed weights have no device copy (packed without a CUDA device)");
     if (M == 0) return SBNN_OK;
-    sbnn_status st = check_device();
+    sbnn_status st = check_packed_device(w);
     if (st != SBNN_OK) return st;
+    if ((st = check_device()) != SBNN_OK) return st;
     if (!(P | GPW | NW | KC) && few_tiles(w, M))
         return conv1x1_small(w, xt_dev, ldx, y_dev, ldy, M, flags & SBNN_RELU, out_cm, static_cast<cudaStream_t>(cuda_stream));
     const TileCfg c = (P | GPW | NW | KC) ? TileCfg{P, GPW, NW, KC} : default_cfg_cm(w, M);

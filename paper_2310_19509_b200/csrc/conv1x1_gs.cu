@@ -334,6 +334,7 @@ sbnn_status launch(const sbnn_packed* p, const Stream1x1& s, const float* x, flo
         return fail(SBNN_ERR_UNSUPPORTED, "internal: weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
     const long long nblk = (long long)((M + C::TM - 1) / C::TM) * s.ntiles;
     if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
+    if (prepare_only()) return SBNN_OK;
     dim3 grid((unsigned)nblk);
     conv1x1_gs_kernel<C><<<grid, C::NT, C::SMEM, st>>>(x, y, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
                                                        p->ngroups, s.nchunks, s.ntiles, relu);
@@ -389,8 +390,8 @@ sbnn_status check_args(const sbnn_packed* w, const float* x, float* y, int N, in
     if (flags & ~(SBNN_RELU | SBNN_BF16_TC)) return fail(SBNN_ERR_UNSUPPORTED, "unknown flag bits 0x%x", flags);
     if (!aligned16(x) || !aligned16(y)) return fail(SBNN_ERR_ALIGN, "x_dev and y_dev must be 16-byte aligned");
     if (w->Cin % 4) return fail(SBNN_ERR_UNSUPPORTED, "Cin=%d is not a multiple of 4", w->Cin);
-    if (w->device < 0) return fail(SBNN_ERR_CUDA, "packed weights have no device copy (packed without a CUDA device)");
-    return SBNN_OK;
+    if ((int64_t)N * H * W == 0) return SBNN_OK;
+    return check_packed_device(w);
 }
 
 }  // namespace

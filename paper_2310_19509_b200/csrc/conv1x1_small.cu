@@ -142,6 +142,7 @@ sbnn_status launch_small(const sbnn_packed* p, const float* x, int ldx, float* y
 sbnn_status conv1x1_small(const sbnn_packed* p, const float* x, int ldx, float* y, int ldy, int M, int relu, bool out_cm,
                           cudaStream_t st) {
     if (p->ngroups > 65535) return fail(SBNN_ERR_SHAPE, "too many groups for the few-pixel kernel");
+    if (prepare_only()) return SBNN_OK;   // reads the canonical arrays: nothing to build
     switch (p->G) {
         case 1: return launch_small<1>(p, x, ldx, y, ldy, M, relu, out_cm, st);
         case 2: return launch_small<2>(p, x, ldx, y, ldy, M, relu, out_cm, st);

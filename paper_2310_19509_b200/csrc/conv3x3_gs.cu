@@ -644,7 +644,9 @@ sbnn_status launch3(const sbnn_packed* p, const float* x, float* y, int N, int H
         }
     }
     if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
-    SBNN_CUDA_TRY(cudaFuncSetAttribute(conv3x3_gs_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    sbnn_status ra = set_max_dyn_smem(reinterpret_cast<const void*>(&conv3x3_gs_kernel<C>), (int)smem);
+    if (ra != SBNN_OK) return ra;
+    if (prepare_only()) return SBNN_OK;
     const long long NH = (long long)N * H;
     dim3 grid((unsigned)((NH + g.R - 1) / g.R), s.ntiles);
     conv3x3_gs_kernel<C><<<grid, C::NT, smem, st>>>(x, y, p->d_bias, s.rec, s.blk_ptr, g, relu);
@@ -701,7 +703,12 @@ sbnn_status launch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y,
         }
     }
     if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
-    SBNN_CUDA_TRY(cudaFuncSetAttribute(conv3x3_gs_cm_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    sbnn_status ra = set_max_dyn_smem(reinterpret_cast<const void*>(&conv3x3_gs_cm_kernel<C>), (int)smem);
+    if (ra != SBNN_OK) return ra;
+    if (prepare_only()) {
+        *done = true;
+        return SBNN_OK;
+    }
     const long long NH = (long long)N * H;
     dim3 grid((unsigned)((NH + g.R - 1) / g.R), s.ntiles);
     conv3x3_gs_cm_kernel<C><<<grid, C::NT, smem, st>>>(xt, ldx, y, p->d_bias, s.rec, s.blk_ptr, g, relu);
@@ -745,16 +752,20 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
         }
     }
     if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
+    sbnn_status r = set_max_dyn_smem(reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C>), (int)smem);
+    if (r != SBNN_OK) return r;
+    int* status = nullptr;
+    if ((r = async_status_word(&status)) != SBNN_OK) return r;
+    if (prepare_only()) {
+        *done = true;
+        return SBNN_OK;
+    }
     const long long NH = (long long)N * H;
     Map3 xmap;
     const unsigned long long dims[3] = {(unsigned long long)W, (unsigned long long)NH, (unsigned long long)p->Cin};
     const unsigned long long strides[2] = {(unsigned long long)W * 4, (unsigned long long)ldx * 4};
     const unsigned box[3] = {(unsigned)g.pitch, (unsigned)(g.R + 2), (unsigned)C::KC};
-    sbnn_status r = encode_tiled_map(&xmap, xt, 4, 3, dims, strides, box);
-    if (r != SBNN_OK) return r;
-    int* status = nullptr;
-    if ((r = async_status_word(&status)) != SBNN_OK) return r;
-    SBNN_CUDA_TRY(cudaFuncSetAttribute(conv3x3_gs_tma_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if ((r = encode_tiled_map(&xmap, xt, 4, 3, dims, strides, box)) != SBNN_OK) return r;
     dim3 grid((unsigned)((NH + g.R - 1) / g.R), s.ntiles);
     conv3x3_gs_tma_kernel<C><<<grid, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status);
     SBNN_CUDA_TRY(cudaGetLastError());
@@ -831,19 +842,19 @@ extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev,
     if (flags & ~SBNN_RELU) return fail(SBNN_ERR_UNSUPPORTED, "flag bits 0x%x not accepted by the 3x3 kernel", flags);
     if (!aligned16(x_dev) || !aligned16(y_dev)) return fail(SBNN_ERR_ALIGN, "x_dev and y_dev must be 16-byte aligned");
     if (w->Cin % 4) return fail(SBNN_ERR_UNSUPPORTED, "Cin=%d is not a multiple of 4", w->Cin);
-    if (w->device < 0) return fail(SBNN_ERR_CUDA, "packed weights have no device copy (packed without a CUDA device)");
     if ((int64_t)N * H * W == 0) return SBNN_OK;
     const int cw = choose_cw(W);
     if (!cw) return fail(SBNN_ERR_UNSUPPORTED, "W=%d: the 3x3 kernel handles rows of at most 256 pixels", W);
-    sbnn_status st = check_device();
+    sbnn_status st = check_packed_device(w);
     if (st != SBNN_OK) return st;
+    if ((st = check_device()) != SBNN_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (W % 4 == 0) {
         // fast path: planes of the input ([Cin][ld]) in the per-device scratch buffer, then the cp.async kernel
         const int M = N * H * W, ld = (M + 3) / 4 * 4;
         float* xt = nullptr;
-        if ((st = scratch_workspace((size_t)w->Cin * ld * sizeof(float), &xt)) != SBNN_OK) return st;
-        if ((st = launch_transpose(x_dev, w->Cin, xt, ld, M, w->Cin, s)) != SBNN_OK) return st;
+        if ((st = scratch_workspace((size_t)w->Cin * ld * sizeof(float), s, &xt)) != SBNN_OK) return st;
+        if (!prepare_only() && (st = launch_transpose(x_dev, w->Cin, xt, ld, M, w->Cin, s)) != SBNN_OK) return st;
         bool done = false;
         st = cw == 7 ? dispatch3_tma<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
                      : dispatch3_tma<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);

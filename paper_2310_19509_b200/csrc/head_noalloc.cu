@@ -69,8 +69,10 @@ extern "C" sbnn_status sbnn_head_noalloc(const sbnn_packed* fc, const float* x_d
                     (long long)N * fc->Cin, kHeadScratchFloats);
     if (!aligned16(x_dev) || !aligned16(logits_dev)) return fail(SBNN_ERR_ALIGN, "x_dev and logits_dev must be 16-byte aligned");
     if (N == 0) return SBNN_OK;
-    sbnn_status st = check_device();
+    // everything that can fail is checked before the first launch: on error nothing has been enqueued
+    sbnn_status st = check_packed_device(fc);
     if (st != SBNN_OK) return st;
+    if ((st = check_device()) != SBNN_OK) return st;
     float* pooled = nullptr;
     if ((st = scratch_address(&pooled)) != SBNN_OK) return st;
     const int total = N * (fc->Cin / 4);

@@ -116,12 +116,12 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
     if (st != SBNN_OK) return st;
     // The kernel-private weight layouts of the channel-major 1x1 kernel are built here, not in forward.
     for (int i = 0; i < SBNN_MBV1_NUM_BLOCKS; ++i) {
-        if (pw[i]->device < 0) return fail(SBNN_ERR_CUDA, "pointwise layer %d was packed without a CUDA device", i + 1);
+        if ((st = check_packed_device(pw[i])) != SBNN_OK) return st;
         const int hw = layer_table()[2 + 2 * i].hin;                 // the block's pointwise layer is entry 2 + 2*i
         if ((st = prepare_default_cm(pw[i], (long long)max_batch * hw * hw)) != SBNN_OK) return st;
         if ((st = prepare_default_cm(pw[i], (long long)hw * hw)) != SBNN_OK) return st;   // and the batch-1 choice
     }
-    if (fc->device < 0) return fail(SBNN_ERR_CUDA, "the classifier was packed without a CUDA device");
+    if ((st = check_packed_device(fc)) != SBNN_OK) return st;
     if ((st = prepare_default_cm(fc, max_batch)) != SBNN_OK) return st;
     sbnn_mbv1* n = new (std::nothrow) sbnn_mbv1;
     if (!n) return fail(SBNN_ERR_ALLOC, "out of host memory");
@@ -153,6 +153,17 @@ extern "C" sbnn_status sbnn_mobilenet_v1_create(const sbnn_packed* const* pw, co
 
 namespace {
 
+// SBNN_OK if the network's weights and workspaces live on the current device.
+sbnn_status check_net_device(const sbnn_mbv1* net) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(SBNN_ERR_CUDA, "no usable CUDA device");
+    }
+    if (dev != net->device)
+        return fail(SBNN_ERR_CUDA, "the network was created on device %d, the current device is %d", net->device, dev);
+    return SBNN_OK;
+}
 
 // One layer on channel-major buffers.  in: channel-major [Cin][ld_in] (layer 0: the NHWC image);
 // out: channel-major [Cout][ld_out] (pool: [N][C]; classifier: [N][1000], reading the pooled [N][C]).
@@ -181,13 +192,14 @@ extern "C" sbnn_status sbnn_mobilenet_v1_run_layer(sbnn_mbv1* net, int layer, co
     if (layer < 0 || layer >= SBNN_MBV1_NUM_LAYERS) return fail(SBNN_ERR_SHAPE, "layer %d out of range", layer);
     if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
     if (N == 0) return SBNN_OK;
+    sbnn_status r = check_net_device(net);
+    if (r != SBNN_OK) return r;
     // The chain's kernels work on channel-major buffers; this entry point takes and returns NHWC, so
     // it converts on the way in and out through the network's own workspaces.
     const LayerShape& L = layer_table()[layer];
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int M_in = N * L.hin * L.hin, M_out = N * L.hout * L.hout;
     const int ld_in = round4(M_in), ld_out = round4(M_out);
-    sbnn_status r;
     const float* src = in;
     if (L.kind != 0) {                                                                   // NHWC [M][C] -> [C][ld]
         if ((r = launch_transpose(in, L.cin, net->ws[0], ld_in, M_in, L.cin, st)) != SBNN_OK) return r;
@@ -206,6 +218,8 @@ extern "C" sbnn_status sbnn_mobilenet_v1_run_layer_cm(sbnn_mbv1* net, int layer,
     if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
     if (!aligned16(in) || !aligned16(outp)) return fail(SBNN_ERR_ALIGN, "in_dev and out_dev must be 16-byte aligned");
     if (N == 0) return SBNN_OK;
+    sbnn_status r = check_net_device(net);
+    if (r != SBNN_OK) return r;
     return run_cm(net, layer, in, outp, N, stream);
 }
 
@@ -239,6 +253,8 @@ extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_
     if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
     if (!aligned16(logits_dev)) return fail(SBNN_ERR_ALIGN, "logits_dev must be 16-byte aligned");
     if (N == 0) return SBNN_OK;
+    sbnn_status dr = check_net_device(net);
+    if (dr != SBNN_OK) return dr;
     cudaStream_t user = static_cast<cudaStream_t>(stream);
     // A caller that is itself capturing gets the plain launches recorded into its own graph.
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;

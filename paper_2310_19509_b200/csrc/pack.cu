@@ -5,7 +5,9 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
+#include <utility>
 
 #include "common.h"
 
@@ -52,12 +54,47 @@ sbnn_status check_device() {
     return SBNN_OK;
 }
 
+sbnn_status check_packed_device(const sbnn_packed* w) {
+    if (w->device < 0) return fail(SBNN_ERR_CUDA, "packed weights have no device copy (packed without a CUDA device)");
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(SBNN_ERR_CUDA, "no usable CUDA device: %s", cudaGetErrorString(e));
+    }
+    if (dev != w->device)
+        return fail(SBNN_ERR_CUDA, "weights were packed on device %d, the current device is %d", w->device, dev);
+    return SBNN_OK;
+}
+
+static thread_local int g_prepare_depth = 0;
+bool prepare_only() { return g_prepare_depth > 0; }
+PrepareScope::PrepareScope() { ++g_prepare_depth; }
+PrepareScope::~PrepareScope() { --g_prepare_depth; }
+
+sbnn_status set_max_dyn_smem(const void* func, int bytes) {
+    static std::mutex mu;
+    static std::map<std::pair<int, const void*>, int> limit;
+    int dev = 0;
+    SBNN_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(mu);
+    int& cur = limit[{dev, func}];
+    if (bytes > cur) {
+        SBNN_CUDA_TRY(cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+        cur = bytes;
+    }
+    return SBNN_OK;
+}
+
 static bool supported_group(int G) { return G == 1 || G == 2 || G == 4 || G == 8 || G == 16; }
 
 template <typename T>
 static sbnn_status upload(T** dst, const std::vector<T>& src) {
-    size_t bytes = (src.size() ? src.size() : 1) * sizeof(T);
+    // At least one whole unit of the widest group (16 floats): kernels that fetch a unit ahead read unit 0 of an
+    // empty layer, which must be addressable (and is zero).
+    const size_t bytes = std::max<size_t>(src.size() * sizeof(T), 64);
     SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(dst), bytes));
+    if (src.size() * sizeof(T) < 64) SBNN_CUDA_TRY(cudaMemset(*dst, 0, bytes));
     if (!src.empty()) SBNN_CUDA_TRY(cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice));
     return SBNN_OK;
 }

@@ -215,3 +215,87 @@ def test_library_layer_table_matches_oracle_and_generator_tables():
         assert g["kind"] == kind and g["stride"] == s
         if kind not in ("pool", "fc"):
             assert h_out == hin // s
+
+
+def test_header_compiles_as_c99_and_the_binding_mirrors_the_view_struct(tmp_path):
+    """include/sbnn.h is a C header: a C99 program that includes it, packs a layer, borrows the view, unpacks and
+    frees through the C interface must compile with -Wall -Werror, link against libsbnn.so and run; the size and
+    field offsets it prints for sbnn_packed_view must be those of the ctypes mirror in the binding."""
+    import subprocess
+    from paper_2310_19509_b200 import binding
+    src = tmp_path / "use_sbnn.c"
+    src.write_text(r'''
+#include <stddef.h>
+#include <stdio.h>
+#include <string.h>
+#include "sbnn.h"
+int main(void) {
+    float w[8 * 8];
+    uint8_t m[8 * 8];
+    float bias[8] = {0.5f, -1.0f, 0.25f, 2.0f, 0.0f, 1.0f, -2.0f, 3.0f};
+    float w2[8 * 8];
+    uint8_t m2[8 * 8];
+    sbnn_packed* p = NULL;
+    sbnn_packed_view v;
+    sbnn_status st;
+    int o, c, bad = 0;
+    for (o = 0; o < 8; ++o)
+        for (c = 0; c < 8; ++c) {
+            w[o * 8 + c] = (float)(o * 8 + c + 1);
+            m[o * 8 + c] = (uint8_t)(((o / 4) + c) % 2);       /* rows 0-3 share a mask, rows 4-7 the other */
+        }
+    st = sbnn_pack_weights(w, m, bias, 8, 1, 1, 8, 4, &p);
+    if (st != SBNN_OK) { printf("pack: %s %s\n", sbnn_status_str(st), sbnn_last_error()); return 1; }
+    if (sbnn_packed_get(p, &v) != SBNN_OK) return 2;
+    if (v.Cout != 8 || v.Cin != 8 || v.G != 4 || v.ngroups != 2 || v.nnz_units != 8 || v.tap_mask != NULL) return 3;
+    if (v.group_ptr[0] != 0 || v.group_ptr[1] != 4 || v.group_ptr[2] != 8) return 4;
+    if (v.idx[0] != 1 || v.idx[3] != 7 || v.idx[4] != 0 || v.idx[7] != 6) return 5;
+    if (v.val[0] != w[0 * 8 + 1] || v.val[1] != w[1 * 8 + 1] || v.bias[3] != 2.0f) return 6;
+    if (sbnn_unpack_weights(p, w2, m2) != SBNN_OK) return 7;
+    for (o = 0; o < 64; ++o) bad += (m2[o] != m[o]) || (w2[o] != (m[o] ? w[o] : 0.0f));
+    if (bad) return 8;
+    if (sbnn_pack_weights(w, m, bias, 8, 1, 1, 8, 3, &p) != SBNN_ERR_GROUP) return 9;
+    if (strlen(sbnn_last_error()) == 0) return 10;
+    if (sbnn_packed_free(p) != SBNN_OK) return 11;
+    printf("%zu %zu %zu %zu %zu %zu %zu\n", sizeof(sbnn_packed_view), offsetof(sbnn_packed_view, nnz_units),
+           offsetof(sbnn_packed_view, group_ptr), offsetof(sbnn_packed_view, idx), offsetof(sbnn_packed_view, val),
+           offsetof(sbnn_packed_view, bias), offsetof(sbnn_packed_view, tap_mask));
+    return 0;
+}
+''')
+    exe = tmp_path / "use_sbnn"
+    libdir = os.path.dirname(sbnn.lib_path())
+    subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(ROOT, "include"),
+                    str(src), "-o", str(exe), "-L", libdir, "-l:libsbnn.so", f"-Wl,-rpath,{libdir}"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, (out.returncode, out.stdout, out.stderr)
+    got = [int(t) for t in out.stdout.split()]
+    V = binding._View
+    assert got == [C.sizeof(V), V.nnz_units.offset, V.group_ptr.offset, V.idx.offset, V.val.offset, V.bias.offset,
+                   V.tap_mask.offset]
+
+
+def test_weights_of_another_device_are_refused_without_a_launch():
+    """A packed layer records the device it was uploaded to.  With the recorded device overwritten by the test hook,
+    every compute entry point must return a status (never dereference the other device's pointers).  On a machine
+    without a GPU the calls fail one check earlier; with one GPU the message names both devices."""
+    L = sbnn.lib()
+    w = np.ones((8, 1, 1, 8), np.float32)
+    m = np.ones((8, 1, 1, 8), np.uint8)
+    p = sbnn.pack_weights(w, m, None, 4)
+    p3 = sbnn.pack_weights(np.ones((8, 3, 3, 8), np.float32), np.ones((8, 3, 3, 8), np.uint8), None, 4)
+    was = [sbnn.debug_set_packed_device(q, 7) for q in (p, p3)]
+    try:
+        calls = [lambda: L.sbnn_conv1x1_gs(p.handle, 256, 512, 1, 2, 2, 0, None),
+                 lambda: L.sbnn_conv1x1_gs_tuned(p.handle, 256, 512, 1, 2, 2, 0, 4, 1, 8, 64, None),
+                 lambda: L.sbnn_conv1x1_gs_cm(p.handle, 256, 4, 512, 8, 4, 0, 0, 0, 0, 0, None),
+                 lambda: L.sbnn_head_noalloc(p.handle, 256, 512, 1, 4, None),
+                 lambda: L.sbnn_prepare(p.handle, 1, 2, 2, 0),
+                 lambda: L.sbnn_conv3x3_gs(p3.handle, 256, 512, 1, 4, 4, 0, None),
+                 lambda: L.sbnn_prepare(p3.handle, 1, 4, 4, 0)]
+        for i, call in enumerate(calls):
+            assert call() == 9, f"call {i}"                                           # SBNN_ERR_CUDA
+            assert len(L.sbnn_last_error()) > 0
+    finally:
+        for q, d in zip((p, p3), was):
+            sbnn.debug_set_packed_device(q, d)                                        # so that free() releases the real copies

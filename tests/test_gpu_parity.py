@@ -30,19 +30,41 @@ def assert_within(y_gpu, ref, s, tol=TOL, what=""):
     return float(np.max(np.where(s > 0, np.abs(y - ref) / np.maximum(tol * s, 1e-300), 0.0)))
 
 
+GUARD = 256          # floats of NaN canary on either side of every output buffer
+
+
+class Guarded:
+    """An output buffer with GUARD floats of NaN before and after it: `t` is the tensor handed to the library
+    (16-byte aligned, NaN-filled so unwritten outputs show), check() asserts that the canaries are untouched."""
+
+    def __init__(self, shape):
+        n = int(np.prod(shape))
+        self.full = torch.full((n + 2 * GUARD,), float("nan"), device="cuda", dtype=torch.float32)
+        self.t = self.full[GUARD:GUARD + n].view(*shape)
+        self.n = n
+
+    def check(self, what=""):
+        assert bool(torch.isnan(self.full[:GUARD]).all()), f"{what}: wrote before the output buffer"
+        assert bool(torch.isnan(self.full[GUARD + self.n:]).all()), f"{what}: wrote past the output buffer"
+
+    def numpy(self, what=""):
+        self.check(what)
+        return self.t.cpu().numpy()
+
+
 def run_1x1(d, flags=sbnn.SBNN_RELU, cfg=None):
     x = d["x"]
     n, h, w, cin = x.shape
     cout = d["w"].shape[0]
     p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], d["g"])
     xd = dev(x)
-    yd = torch.full((n, h, w, cout), float("nan"), device="cuda", dtype=torch.float32)
+    out = Guarded((n, h, w, cout))
     if cfg is None:
-        sbnn.conv1x1_gs(p, xd, yd, n, h, w, flags)
+        sbnn.conv1x1_gs(p, xd, out.t, n, h, w, flags)
     else:
-        sbnn.conv1x1_gs_tuned(p, xd, yd, n, h, w, flags, *cfg)
+        sbnn.conv1x1_gs_tuned(p, xd, out.t, n, h, w, flags, *cfg)
     sbnn.get_async_status()
-    y = yd.cpu().numpy()
+    y = out.numpy("1x1")
     p.free()
     return y
 
@@ -211,15 +233,16 @@ def test_mobilenet_v1_batch1_layer_isolated_and_end_to_end(sparsity):
     # (i) every layer alone, fed the oracle's fp32 input of that layer
     for li, rec in enumerate(outs):
         ref, s = rec["ref"], rec["S"]
-        yd = torch.full(ref.shape, float("nan"), device="cuda", dtype=torch.float32)
-        net.run_layer(li, dev(rec["in"]), yd, 1)
+        out = Guarded(ref.shape)
+        net.run_layer(li, dev(rec["in"]), out.t, 1)
         sbnn.get_async_status()
-        assert_within(yd.cpu().numpy(), ref, s, what=f"layer {li} {rec['name']}")
+        assert_within(out.numpy(f"layer {li}"), ref, s, what=f"layer {li} {rec['name']}")
     # (ii) the chain, against the propagated first-order bound
-    logits = torch.full((1, 1000), float("nan"), device="cuda")
+    lg = Guarded((1, 1000))
+    logits = lg.t
     net.forward(dev(x), logits, 1)
     sbnn.get_async_status()
-    y = logits.cpu().numpy().astype(np.float64).reshape(outs[-1]["ref"].shape)
+    y = lg.numpy("forward").astype(np.float64).reshape(outs[-1]["ref"].shape)
     err = np.abs(y - outs[-1]["ref"])
     assert np.all(err <= outs[-1]["E"]), f"worst ratio {np.max(err / outs[-1]['E'])}"
     # two copies of the image in one call give the same logits twice, bit for bit, and the single-image result
@@ -271,18 +294,26 @@ def test_forward_graph_replay_matches_plain_launches():
 
 def test_forward_accepts_an_image_that_is_only_4_byte_aligned():
     """The first layer's fast kernel needs 16-byte aligned rows; an input at an odd float offset takes the generic
-    first-layer kernel and must give the same logits (same order of sums: compared closely, not bit for bit)."""
+    first-layer kernel.  Both routes are compared with the oracle's chain (propagated bound), and the generic
+    first-layer kernel alone with the oracle's first layer."""
     x, layers = mobilenet_v1_inputs(1, 50, 4, seed=6)
+    outs = R.mobilenet_v1_forward(x, layers)
+    ref, e = outs[-1]["ref"].reshape(1, 1000), outs[-1]["E"].reshape(1, 1000)
     net = build_net(layers, 1)
     flat = torch.zeros(x.size + 1, device="cuda")
     flat[1:] = dev(x).reshape(-1)
-    a = torch.full((1, 1000), float("nan"), device="cuda")
-    b = torch.full((1, 1000), float("nan"), device="cuda")
-    net.forward(dev(x), a, 1)
-    net.forward(flat[1:], b, 1)
+    for src in (dev(x), flat[1:]):                   # aligned (fast first-layer kernel), then at an odd float offset
+        lg = Guarded((1, 1000))
+        net.forward(src, lg.t, 1)
+        sbnn.get_async_status()
+        y = lg.numpy("forward").astype(np.float64)
+        assert np.all(np.isfinite(y))
+        assert np.all(np.abs(y - ref) <= e), f"worst ratio {np.max(np.abs(y - ref) / e)}"
+    # layer 0 alone on the unaligned image, against the oracle's first layer
+    out = Guarded(outs[0]["ref"].shape)
+    net.run_layer(0, flat[1:], out.t, 1)
     sbnn.get_async_status()
-    assert bool(torch.isfinite(b).all())
-    assert torch.allclose(a, b, rtol=1e-4, atol=1e-5)
+    assert_within(out.numpy("conv0"), outs[0]["ref"], outs[0]["S"], what="first layer, 4-byte aligned image")
     net.free()
 
 
@@ -291,10 +322,10 @@ def run_3x3(d, flags=sbnn.SBNN_RELU):
     n, h, w, cin = x.shape
     cout = d["w"].shape[0]
     p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], d["g"])
-    yd = torch.full((n, h, w, cout), float("nan"), device="cuda", dtype=torch.float32)
-    sbnn.conv3x3_gs(p, dev(x), yd, n, h, w, flags)
+    out = Guarded((n, h, w, cout))
+    sbnn.conv3x3_gs(p, dev(x), out.t, n, h, w, flags)
     sbnn.get_async_status()
-    y = yd.cpu().numpy()
+    y = out.numpy("3x3")
     p.free()
     return y
 
@@ -369,15 +400,17 @@ def run_cm(d, flags, tile, out_cm):
     xt = torch.full((cin, ld), float("nan"), device="cuda")
     sbnn.to_channel_major(dev(x), xt, m, cin, ld)
     if out_cm:
-        yd = torch.full((cout, ld), float("nan"), device="cuda")
-        sbnn.conv1x1_gs_cm(p, xt, ld, yd, ld, m, flags | sbnn.SBNN_OUT_CM, tile)
+        out = Guarded((cout, ld))
+        sbnn.conv1x1_gs_cm(p, xt, ld, out.t, ld, m, flags | sbnn.SBNN_OUT_CM, tile)
         sbnn.get_async_status()
-        y = yd.cpu().numpy()[:, :m].T.reshape(n, h, w, cout)
+        full = out.numpy("cm")
+        assert np.all(np.isnan(full[:, m:]))                 # the row padding past the last pixel stays untouched
+        y = full[:, :m].T.reshape(n, h, w, cout)
     else:
-        yd = torch.full((m, cout), float("nan"), device="cuda")
-        sbnn.conv1x1_gs_cm(p, xt, ld, yd, cout, m, flags, tile)
+        out = Guarded((m, cout))
+        sbnn.conv1x1_gs_cm(p, xt, ld, out.t, cout, m, flags, tile)
         sbnn.get_async_status()
-        y = yd.cpu().numpy().reshape(n, h, w, cout)
+        y = out.numpy("cm").reshape(n, h, w, cout)
     p.free()
     return y
 
@@ -495,3 +528,71 @@ def test_expired_wait_is_reported_and_the_context_stays_usable():
     y = run_1x1(d)
     ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
     assert_within(y, ref, s, what="after an expired wait")
+
+
+def test_weights_of_another_device_are_refused_and_the_context_stays_usable():
+    """With the recorded device of a packed layer overwritten (test hook), the compute calls return SBNN_ERR_CUDA
+    naming both devices and launch nothing; with the number restored the same call works."""
+    d = WL.single_conv_inputs(1, 4, 4, 16, 16, 1, 4, 50, seed=3)
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    x, out = dev(d["x"]), Guarded((1, 4, 4, 16))
+    was = sbnn.debug_set_packed_device(p, 5)
+    assert was == torch.cuda.current_device()
+    for call in (lambda: sbnn.conv1x1_gs(p, x, out.t, 1, 4, 4), lambda: sbnn.head_noalloc(p, x, out.t, 1, 16),
+                 lambda: sbnn.prepare(p, 1, 4, 4)):
+        with pytest.raises(sbnn.SbnnError) as e:
+            call()
+        assert e.value.name == "SBNN_ERR_CUDA" and "device 5" in e.value.detail
+    sbnn.get_async_status()
+    assert bool(torch.isnan(out.t).all())                     # nothing ran
+    sbnn.debug_set_packed_device(p, was)
+    sbnn.conv1x1_gs(p, x, out.t, 1, 4, 4)
+    sbnn.get_async_status()
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    assert_within(out.numpy(), ref, s)
+    p.free()
+
+
+def test_prepare_then_calls_only_enqueue_and_capture_refuses_to_grow_the_scratch():
+    """sbnn_prepare builds the private layouts and sizes the per-device scratch for a shape; a larger NHWC call made
+    while its stream is being captured is refused (the scratch cannot grow there) and leaves the capture intact; after
+    preparing for that shape the same call is captured, and replaying the graph gives the oracle's result."""
+    d = WL.single_conv_inputs(1, 1, 2600, 256, 64, 1, 4, 50, seed=17)           # Cin >= 128, M >= 2048: channel-major route
+    n, h, w, cin = d["x"].shape
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    big = WL.single_conv_inputs(1, 1, 180000, 256, 64, 1, 4, 50, seed=17)       # same layer, 184 MB of scratch
+    bx = dev(big["x"])
+    bout = Guarded((1, 1, 180000, 64))
+    side = torch.cuda.Stream()
+    refused = None
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        try:
+            sbnn.conv1x1_gs(p, bx, bout.t, 1, 1, 180000, stream=torch.cuda.current_stream())
+        except sbnn.SbnnError as e:
+            refused = e
+    if refused is not None:          # (not refused only if an earlier test already grew the scratch this far)
+        assert refused.name == "SBNN_ERR_UNSUPPORTED" and "sbnn_prepare" in refused.detail
+    sbnn.prepare(p, 1, 1, 180000)
+    g2 = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g2, stream=side):
+        sbnn.conv1x1_gs(p, bx, bout.t, 1, 1, 180000, stream=torch.cuda.current_stream())
+    g2.replay()
+    torch.cuda.synchronize()
+    sbnn.get_async_status()
+    y = bout.numpy("captured call")
+    pix = np.arange(0, 180000, 61)
+    xs = np.ascontiguousarray(big["x"].reshape(-1, cin)[pix]).reshape(1, 1, len(pix), cin)
+    ref, s = R.conv2d(xs, big["w"], big["mask"], big["bias"], relu=True)
+    assert_within(y.reshape(-1, 64)[pix].reshape(ref.shape), ref, s, what="graph replay after sbnn_prepare")
+    p.free()
+
+
+def test_few_pixel_kernel_on_a_layer_without_kept_units():
+    """Every unit pruned: the few-pixel kernel's look-ahead fetch has no unit to read; the output is act(bias)."""
+    d = WL.single_conv_inputs(1, 3, 5, 40, 24, 1, 4, 100, seed=10)
+    assert not d["mask"].any()
+    for relu in (True, False):
+        y = run_cm(d, sbnn.SBNN_RELU if relu else 0, (0, 0, 0, 0), True)
+        want = np.maximum(d["bias"], 0) if relu else d["bias"]
+        assert np.array_equal(y, np.broadcast_to(want, y.shape))

@@ -10,6 +10,7 @@ import pytest
 import torch
 
 import paper_2310_19509_b200 as sbnn
+from oracle import reference as R
 from sbnn_inputs import workloads as WL
 
 pytestmark = pytest.mark.gpu
@@ -43,6 +44,15 @@ def test_head_noalloc_matches_pool_then_classifier_twice_in_a_row():
         s = np.abs(pooled.astype(np.float64)) @ np.abs(w).T + np.abs(d["bias"].astype(np.float64))
         assert np.all(np.isfinite(got))
         assert np.all(np.abs(got.astype(np.float64) - want) <= TOL * s), f"call {call}"
+        # and against the CPU oracle: mean over the positions, then the classifier on the fp32-rounded means.  A head
+        # that is within TOL*S on each of its two steps deviates by at most |W| (TOL*S_pool) + TOL*S_fc.
+        pref, ps = R.avgpool(x.reshape(nn, 7, 7, c))
+        pooled_ref = pref.astype(np.float32)
+        ref, sfc = R.conv2d(pooled_ref.reshape(nn, 1, 1, c), d["w"], d["mask"], d["bias"], relu=False)
+        e_in = (TOL * ps + np.abs(pref) * 2.0 ** -24).astype(np.float32) * np.float32(1 + 2.0 ** -20)
+        e, _ = R.conv2d(e_in.reshape(nn, 1, 1, c), np.abs(d["w"]), d["mask"], None, relu=False)
+        bound = (e + TOL * sfc).reshape(nn, cout)
+        assert np.all(np.abs(got.astype(np.float64) - ref.reshape(nn, cout)) <= bound), f"call {call} vs oracle"
     fc.free()
 
 
