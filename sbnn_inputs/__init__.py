@@ -8,6 +8,7 @@ from .rng import uniform01, normal, u64_stream
 from .masks import removed_units, group_mask_balanced, group_mask_layer_global, group_mask_magnitude, expand_mask, tap_pattern_mask, dw_pattern_mask
 from .workloads import (
     single_conv_inputs,
+    config5_family,
     mobilenet_v1_shapes,
     mobilenet_v1_inputs,
 )
@@ -16,5 +17,5 @@ __all__ = [
     "uniform01", "normal", "u64_stream",
     "removed_units", "group_mask_balanced", "group_mask_layer_global",
     "group_mask_magnitude", "expand_mask", "tap_pattern_mask", "dw_pattern_mask",
-    "single_conv_inputs", "mobilenet_v1_shapes", "mobilenet_v1_inputs",
+    "single_conv_inputs", "config5_family", "mobilenet_v1_shapes", "mobilenet_v1_inputs",
 ]

@@ -53,6 +53,21 @@ def config5(g, sparsity_pct, seed=0, n=256):
     return single_conv_inputs(n, 14, 14, 1024, 1024, 1, g, sparsity_pct, seed, 0.02, 0.05)
 
 
+def config5_family(cases, seed=0, n=256):
+    """The layers of the sparsity sweep for several (g, sparsity_pct) pairs.  Activations, weights and bias do not
+    depend on g or the sparsity (same streams, same seed), so they are drawn once and shared; only the masks differ.
+    Yields the same dicts as config5(g, sparsity_pct, seed, n)."""
+    base = None
+    for g, sp in cases:
+        if base is None:
+            base = config5(g, sp, seed, n)
+            yield base
+            continue
+        um = _masks.group_mask_balanced(seed, STREAM_MASK, 1024 // g, 1024, sp, 1)
+        yield {"x": base["x"], "w": base["w"], "bias": base["bias"], "mask": _masks.expand_mask(um, g, 1, 1),
+               "unit_mask": um, "g": g, "sparsity_pct": sp}
+
+
 def mobilenet_v1_shapes():
     """Layer list of MobileNet-v1, width 1.0, 224x224x3 input (Howard et al. 2017, Table 1).
 
