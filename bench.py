@@ -27,18 +27,35 @@ import numpy as np  # noqa: E402
 
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FP32 lanes x 2 flop x max SM clock
 HBM_FALLBACK_GBS = 6650.0
+BF16_FALLBACK_TFLOPS = 1590.0
 METRIC = "mobilenet_v1_images_per_s"
-PW_DRAM_BYTES_PER_STEP = 746.5e6
+# DRAM bytes (read + write) of the 13 pointwise launches of one default step, from the ncu capture summarised in
+# profiles/bench_mobilenet_v1_b64_s50_launch_list.md, and the SHA-1 of the kernel source the capture was taken with:
+# the figure is reported only while the kernel source still has that hash.
+PW_DRAM_BYTES_PER_STEP = None
+PW_DRAM_KERNEL_SHA1 = None
+PW_KERNEL_SOURCES = ("paper_2310_19509_b200/csrc/conv1x1_cm.cu", "paper_2310_19509_b200/csrc/pipeline.cuh")
+
+
+def kernel_source_sha1():
+    import hashlib
+    h = hashlib.sha1()
+    for rel in PW_KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 def measured_peaks():
+    """(HBM GB/s, bf16 dense TFLOP/s burst, 'measured' | 'fallback')."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         try:
-            return float(json.load(open(p))["hbm_gbs"]), "measured"
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), float(d.get("bf16_tflops", BF16_FALLBACK_TFLOPS)), "measured"
         except Exception:
             pass
-    return HBM_FALLBACK_GBS, "fallback"
+    return HBM_FALLBACK_GBS, BF16_FALLBACK_TFLOPS, "fallback"
 
 
 # ------------------------------------------------------------------------------------------
@@ -234,6 +251,100 @@ def sweep_oracle_lines():
                           "sample": f"{n_timed} of {n_full} images, scaled", "us": dt * 1e6 * n_full / n_timed}), flush=True)
 
 
+def measure_fma_peak(sbnn, torch):
+    """FP32 rate of the register-only packed-FMA kernel of the library (TFLOP/s), best of 5 launches of about 1 ms."""
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    best = 0.0
+    for rep in range(7):
+        ev0.record()
+        flop = sbnn.selftest_fma_rate(4000)
+        ev1.record()
+        ev1.synchronize()
+        if rep >= 2:
+            best = max(best, flop / (ev0.elapsed_time(ev1) * 1e-3) / 1e12)
+    return best
+
+
+def _time_fn(torch, fn, reps, flush):
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        fn()
+    ts = []
+    for _ in range(reps):
+        flush.add_(1.0)
+        ev0.record()
+        fn()
+        ev1.record()
+        ev1.synchronize()
+        ts.append(ev0.elapsed_time(ev1) * 1e-3)
+    return float(np.median(ts))
+
+
+def dense_library_us(torch, m, cin, cout, k, shape4, reps, flush):
+    """Dense library times of one layer shape, microseconds: cuDNN conv2d on channels-last tensors and, for 1x1, cuBLAS
+    addmm on [M][Cin] x [Cin][Cout], each with TF32 off (like for like with the fp32 kernels) and on (context)."""
+    n, h, w = shape4
+    x = torch.rand((n, h, w, cin), device="cuda")
+    xt = x.permute(0, 3, 1, 2)
+    wt = torch.randn(cout, cin, k, k, device="cuda").contiguous(memory_format=torch.channels_last)
+    b = torch.randn(cout, device="cuda")
+    out = {}
+    for tag, tf32 in (("fp32", False), ("tf32", True)):
+        torch.backends.cudnn.allow_tf32 = tf32
+        torch.backends.cuda.matmul.allow_tf32 = tf32
+        out[f"cudnn_{tag}_us"] = round(_time_fn(torch, lambda: torch.relu_(torch.nn.functional.conv2d(xt, wt, b, padding=(k - 1) // 2)),
+                                                reps, flush) * 1e6, 1)
+        if k == 1:
+            x2, w2 = x.reshape(m, cin), wt.reshape(cout, cin).t().contiguous()
+            out[f"cublas_{tag}_us"] = round(_time_fn(torch, lambda: torch.relu_(torch.addmm(b, x2, w2)), reps, flush) * 1e6, 1)
+    torch.backends.cudnn.allow_tf32 = False
+    torch.backends.cuda.matmul.allow_tf32 = False
+    return out
+
+
+def single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, reps):
+    """The single-layer configurations (config 1, config 4, the ten config-5 cases in fp32 and in the bf16 tensor-core
+    mode) through the NHWC entry points, beside dense cuDNN / cuBLAS of the same shape.  fp32 fractions are against
+    max(nonzero flop / FP32 peak, bytes / HBM); bf16 fractions against max(nonzero flop / bf16 tensor peak, bytes / HBM)."""
+    from sbnn_inputs import workloads as WL
+    out, dense = [], {}
+
+    def one(name, d, k, flags, mode):
+        x = d["x"]
+        n, h, w, cin = x.shape
+        cout, g = d["w"].shape[0], d["g"]
+        m = n * h * w
+        p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], g)
+        xd = torch.from_numpy(x).cuda()
+        yd = torch.empty((n, h, w, cout), device="cuda")
+        fn = (lambda: sbnn.conv3x3_gs(p, xd, yd, n, h, w, flags)) if k == 3 else (lambda: sbnn.conv1x1_gs(p, xd, yd, n, h, w, flags))
+        t = _time_fn(torch, fn, reps, flush)
+        sbnn.get_async_status()
+        units = int(d["unit_mask"].sum())
+        flops = 2.0 * m * g * k * k * units
+        byts = 4.0 * (m * (cin + cout) + units * (1 + g * k * k) + cout + cout // g + 1)
+        peak = bf16_tflops if mode == "bf16_tc" else FP32_PEAK_TFLOPS
+        t_alu, t_hbm = flops / (peak * 1e12), byts / (hbm_gbs * 1e9)
+        rec = {"case": name, "mode": mode, "G": g, "sparsity_pct": d["sparsity_pct"], "us": round(t * 1e6, 1),
+               "tflops_nonzero": round(flops / t / 1e12, 2), "roofline_us": round(max(t_alu, t_hbm) * 1e6, 1),
+               "frac": round(max(t_alu, t_hbm) / t, 3), "bound": ("tensor" if mode == "bf16_tc" else "alu") if t_alu > t_hbm else "hbm"}
+        key = (m, cin, cout, k)
+        if key not in dense:
+            dense[key] = dense_library_us(torch, m, cin, cout, k, (n, h, w), max(3, reps // 2), flush)
+        rec.update(dense[key])
+        out.append(rec)
+        p.free()
+        del xd, yd
+
+    one("config1", WL.config1(), 1, sbnn.SBNN_RELU, "fp32")
+    one("config4", WL.config4(), 3, sbnn.SBNN_RELU, "fp32")
+    cases = [(g, sp) for g in (4, 8) for sp in (0, 30, 50, 70, 90)]
+    for (g, sp), d in zip(cases, WL.config5_family(cases)):
+        one(f"config5_G{g}_s{sp}", d, 1, sbnn.SBNN_RELU, "fp32")
+        one(f"config5_G{g}_s{sp}", d, 1, sbnn.SBNN_RELU | sbnn.SBNN_BF16_TC, "bf16_tc")
+    return out
+
+
 def max_over_ranks(values, world, device="cpu"):
     """Element-wise maximum of per-rank timings over the process group (the job is as slow as its slowest replica)."""
     if world <= 1:
@@ -333,7 +444,8 @@ def run_gpu(args, rank, world, local_rank):
     chain_t = time_layers_in_chain(sbnn, torch, net, layers, batch, xd, max(args.layer_reps, 5))
     for r, t in zip(per, chain_t):
         r["s_cold"], r["s"] = r["s"], t          # the roofline uses the in-step durations; the cold ones are reported beside
-    hbm_gbs, peak_kind = measured_peaks()
+    hbm_gbs, bf16_tflops, peak_kind = measured_peaks()
+    fma_measured = measure_fma_peak(sbnn, torch)
     pw = [r for r in per if r["kind"] == "pw"]
     pw_t, pw_fl, pw_by = sum(r["s"] for r in pw), sum(r["flops"] for r in pw), sum(r["bytes"] for r in pw)
     pw_t_cold = sum(r["s_cold"] for r in pw)
@@ -346,10 +458,11 @@ def run_gpu(args, rank, world, local_rank):
         "timing": "CUDA events between the consecutive launches of a step (forward's order and buffers, no flush)",
         "frac_cold": pw_fl / pw_t_cold / 1e12 / FP32_PEAK_TFLOPS,
         "frac_cold_note": "each layer launched alone after a 256 MB write has flushed L2",
-        "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz (no measured FP32 peak on file)",
-        # dram__bytes_read.sum + dram__bytes_write.sum of the 13 launches of one step from the ncu capture in
-        # profiles/bench_mobilenet_v1_b64_s50_launch_list.md; valid for the default workload and this kernel only
-        "traffic": PW_DRAM_BYTES_PER_STEP if (batch == 64 and args.sparsity == 50) else None,
+        "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
+        "peak_measured": fma_measured,
+        "peak_measured_note": "register-only fma.rn.f32x2 kernel of the library (sbnn_selftest_fma_rate) timed in this run",
+        "frac_of_measured_peak": pw_fl / pw_t / 1e12 / fma_measured if fma_measured > 0 else None,
+        "traffic": PW_DRAM_BYTES_PER_STEP if (batch == 64 and args.sparsity == 50 and PW_DRAM_KERNEL_SHA1 == kernel_source_sha1()) else None,
         "algorithmic_bytes": pw_by,
         "mixed_frac": sum(t_roof(r) for r in pw) / pw_t,
         "mixed_note": f"sum over layers of max(nonzero flops/FP32 peak, bytes/{hbm_gbs:.0f} GB/s {peak_kind}) / measured",
@@ -360,6 +473,22 @@ def run_gpu(args, rank, world, local_rank):
     layers_out = [{"name": r["name"], "us": round(r["s"] * 1e6, 2), "us_cold": round(r["s_cold"] * 1e6, 2), "tflops": round(r["flops"] / r["s"] / 1e12, 2),
                    "gbs": round(r["bytes"] / r["s"] / 1e9, 1), "frac": round(t_roof(r) / r["s"], 3)} for r in per]
 
+    if not args.no_dense:
+        seen = {}
+        for r, L in zip(per, layers):
+            if L["kind"] != "pw":
+                continue
+            hin, cin, hout, cout = sbnn.mobilenet_v1_layer_shape(layers.index(L))
+            key = (hout, cin, cout)
+            if key not in seen:
+                seen[key] = dense_library_us(torch, batch * hout * hout, cin, cout, 1, (batch, hout, hout), 5, flush)
+            for lo in layers_out:
+                if lo["name"] == r["name"]:
+                    lo.update(seen[key])
+        roofline["dense_library_us_per_step"] = {k: round(sum(lo.get(k, 0.0) for lo in layers_out if lo["name"].startswith("pw")), 1)
+                                                 for k in ("cublas_fp32_us", "cublas_tf32_us", "cudnn_fp32_us", "cudnn_tf32_us")}
+        roofline["pointwise_us_per_step"] = round(pw_t * 1e6, 1)
+    single = single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, 7) if (world == 1 and not args.no_single) else None
     cpu = cpu_baseline(x, layers) if world == 1 and not args.no_cpu else None
     imgs = batch * world * args.steps
     assert abs(job_throughput(batch, args.steps, world, elapsed) - imgs / elapsed) < 1e-6 * imgs / elapsed
@@ -379,6 +508,8 @@ def run_gpu(args, rank, world, local_rank):
         "gpu_launches": 29 * args.steps,
         "clocks": clocks, "roofline": roofline, "layers": layers_out,
     }
+    if single is not None:
+        line["single_layer"] = single
     if cpu is not None:
         line["cpu_baseline"] = cpu
     print(json.dumps(line), flush=True)
@@ -396,6 +527,8 @@ def main():
     ap.add_argument("--sparsity", type=int, default=50)
     ap.add_argument("--layer-reps", type=int, default=10)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense cuDNN / cuBLAS times of the pointwise shapes")
+    ap.add_argument("--no-single", action="store_true", help="skip the single-layer configurations (configs 1, 4, 5)")
     ap.add_argument("--sweep", action="store_true", help="print extra lines for the single-layer configurations")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

@@ -683,6 +683,12 @@ sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, 
     X(4, 8, 2, 8, 32, 4)   \
     X(4, 8, 2, 11, 32, 3)  \
     X(4, 8, 2, 12, 32, 3)  \
+    X(4, 8, 2, 8, 64, 2)   \
+    X(4, 8, 2, 11, 64, 2)  \
+    X(4, 8, 2, 12, 64, 2)  \
+    X(4, 8, 1, 16, 64, 2)  \
+    X(8, 8, 1, 8, 64, 2)   \
+    X(8, 8, 1, 12, 64, 2)  \
     X(4, 4, 1, 8, 32, 4)   \
     X(8, 8, 1, 8, 32, 4)   \
     X(8, 8, 1, 12, 32, 3)  \
@@ -728,16 +734,18 @@ TileCfg default_cfg_cm(const sbnn_packed* p, long long M) {
         }
         return best;
     };
+    // Channels per pipeline step: 64 (two stages) wherever the layer has that many.  A warp's lists are per step, and
+    // every list costs a pipeline fill and drain, so longer steps are cheaper (config 5, G = 4, 50 %: 0.63 -> 0.68 of
+    // the roofline; 70 %: 0.55 -> 0.62); thin layers (Cin < 64) keep 32 so that no stage is half zeros.
+    const int kc = p->Cin >= 64 ? 64 : 32;
     switch (p->G) {
         case 1: return {8, 4, 8, 32};
         case 2: return {8, 2, 8, 32};
         case 4:
-            // Sparse layers leave each warp little work per step, so twice as many warps with one group
-            // each hide the per-step latencies better than the shared activation fetch of two groups saves
-            // (measured cross-over between 50 % and 70 % removed units).
-            if ((double)p->nnz < 0.4 * (double)p->ngroups * p->Cin) return {8, 1, 16, 32};
-            return pick({8, 2, 8, 32}, {{8, 2, 11, 32}, {8, 2, 12, 32}});
-        case 8: return pick({8, 1, 8, 32}, {{8, 1, 12, 32}});
+            // Two groups per warp with union lists at every density: with 64-channel steps they also beat one group
+            // per warp on twice the warps for sparse layers (config 5 at 70 / 90 %: 0.63 / 0.45 against 0.61 / 0.42).
+            return pick({8, 2, 8, kc}, {{8, 2, 11, kc}, {8, 2, 12, kc}});
+        case 8: return pick({8, 1, 8, kc}, {{8, 1, 12, kc}});
         default: return {4, 1, 8, 32};
     }
 }
@@ -803,8 +811,8 @@ sbnn_status prepare_all_cm(const sbnn_packed* p) {
     switch (p->G) {
         case 1: all = {{8, 4, 8, 32}}; break;
         case 2: all = {{8, 2, 8, 32}}; break;
-        case 4: all = {{8, 1, 16, 32}, {8, 2, 8, 32}, {8, 2, 11, 32}, {8, 2, 12, 32}}; break;
-        case 8: all = {{8, 1, 8, 32}, {8, 1, 12, 32}}; break;
+        case 4: all = {{8, 2, 8, 32}, {8, 2, 11, 32}, {8, 2, 12, 32}, {8, 2, 8, 64}, {8, 2, 11, 64}, {8, 2, 12, 64}}; break;
+        case 8: all = {{8, 1, 8, 32}, {8, 1, 12, 32}, {8, 1, 8, 64}, {8, 1, 12, 64}}; break;
         default: all = {{4, 1, 8, 32}}; break;
     }
     PrepareScope scope;   // dispatch_cm then builds the stream and sets the kernel's attributes, and launches nothing

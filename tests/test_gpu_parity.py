@@ -386,8 +386,9 @@ def test_3x3_dense_and_empty_masks():
 
 
 CM_CFGS = {1: [(8, 4, 8, 32)], 2: [(8, 2, 8, 32)],
-           4: [(8, 1, 16, 32), (8, 2, 8, 32), (8, 2, 11, 32), (8, 2, 12, 32), (4, 1, 8, 32)],
-           8: [(8, 1, 8, 32), (8, 1, 12, 32), (4, 1, 16, 32)], 16: [(4, 1, 8, 32)]}
+           4: [(8, 1, 16, 32), (8, 2, 8, 32), (8, 2, 11, 32), (8, 2, 12, 32), (4, 1, 8, 32),
+               (8, 1, 16, 64), (8, 2, 8, 64), (8, 2, 11, 64), (8, 2, 12, 64)],
+           8: [(8, 1, 8, 32), (8, 1, 12, 32), (4, 1, 16, 32), (8, 1, 8, 64), (8, 1, 12, 64)], 16: [(4, 1, 8, 32)]}
 
 
 def run_cm(d, flags, tile, out_cm):
