@@ -212,26 +212,34 @@ def time_layers(sbnn, torch, net, layers, batch, reps, flush):
 
 
 def time_layers_in_chain(sbnn, torch, net, layers, batch, xd, reps):
-    """The 29 launches in forward's order on forward-sized ping-pong buffers, a CUDA event between consecutive
-    launches: what each kernel takes inside a step (its input just written by its predecessor, no L2 flush)."""
+    """Cost of every layer inside a step: T(layers 0..l) - T(layers 0..l-1), where each prefix of the chain is recorded
+    into a CUDA graph (the way forward runs) and replayed back to back, CUDA events around `reps` replays, median of 3.
+    The 29 figures add up to the time of the whole chain, so they include what a kernel costs its neighbours (launch
+    gap, cold pipeline) and nothing that a step does not pay."""
     r4 = lambda v: (v + 3) // 4 * 4  # noqa: E731
-    bufs = [torch.empty(64 * r4(batch * 112 * 112) + 4096, device="cuda") for _ in range(2)]
-    logits = torch.empty((batch, 1000), device="cuda")
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(layers) + 1)]
-    samples = [[] for _ in layers]
-    for rep in range(reps + 2):
-        src = xd
-        for li, L in enumerate(layers):
-            dst = logits if L["kind"] == "fc" else bufs[li & 1]
-            evs[li].record()
-            net.run_layer_cm(li, src, dst, batch)
-            src = dst
-        evs[len(layers)].record()
-        evs[len(layers)].synchronize()
-        if rep >= 2:
-            for li in range(len(layers)):
-                samples[li].append(evs[li].elapsed_time(evs[li + 1]) * 1e-3)
-    return [float(np.median(v)) for v in samples]
+    out = torch.empty(64 * r4(batch * 112 * 112) + 4096, device="cuda")
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    prefix = []
+    for l in range(len(layers)):
+        net.forward_prefix(xd, out, batch, l)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            net.forward_prefix(xd, out, batch, l)
+        for _ in range(3):
+            g.replay()
+        runs = []
+        for _ in range(3):
+            torch.cuda.synchronize()
+            ev0.record()
+            for _ in range(reps):
+                g.replay()
+            ev1.record()
+            ev1.synchronize()
+            runs.append(ev0.elapsed_time(ev1) * 1e-3 / reps)
+        prefix.append(float(np.median(runs)))
+        del g
+    return [max(prefix[0], 0.0)] + [max(prefix[l] - prefix[l - 1], 0.0) for l in range(1, len(layers))]
 
 
 def sweep_oracle_lines():
@@ -441,7 +449,7 @@ def run_gpu(args, rank, world, local_rank):
     # per-layer timings for the roofline of the dominant kernel (the group-sparse 1x1)
     flush = torch.zeros(64 * 1024 * 1024, device="cuda")     # 256 MB > L2
     per = time_layers(sbnn, torch, net, layers, batch, args.layer_reps, flush)
-    chain_t = time_layers_in_chain(sbnn, torch, net, layers, batch, xd, max(args.layer_reps, 5))
+    chain_t = time_layers_in_chain(sbnn, torch, net, layers, batch, xd, max(args.layer_reps, 10))
     for r, t in zip(per, chain_t):
         r["s_cold"], r["s"] = r["s"], t          # the roofline uses the in-step durations; the cold ones are reported beside
     hbm_gbs, bf16_tflops, peak_kind = measured_peaks()
@@ -455,7 +463,9 @@ def run_gpu(args, rank, world, local_rank):
         "bound": "alu", "kernel": "conv1x1_cm_kernel (13 pointwise launches per step)",
         "achieved": pw_fl / pw_t / 1e12, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s",
         "frac": pw_fl / pw_t / 1e12 / FP32_PEAK_TFLOPS,
-        "timing": "CUDA events between the consecutive launches of a step (forward's order and buffers, no flush)",
+        "timing": "per layer: time of the chain's prefix up to and including the layer minus the prefix before it, each prefix a "
+                  "CUDA graph replayed back to back under CUDA events (forward's launches and buffers, no flush); the 29 "
+                  "figures add up to one whole forward",
         "frac_cold": pw_fl / pw_t_cold / 1e12 / FP32_PEAK_TFLOPS,
         "frac_cold_note": "each layer launched alone after a 256 MB write has flushed L2",
         "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
@@ -500,8 +510,8 @@ def run_gpu(args, rank, world, local_rank):
                                f"group-sparse G=4 at {args.sparsity}% (balanced random masks), rest dense",
                    "global_batch": batch * world, "parallelism": f"batch-sharded replicas x{world}, no collective",
                    "l2": "one step streams about 2.6 GB of activations through two ping-pong buffers (far above the "
-                         "126 MB L2); per-layer timings: in step order without a flush (roofline), and alone after a 256 MB "
-                         "write has flushed L2 (us_cold)"},
+                         "126 MB L2); per-layer timings: differences of chain prefixes replayed as CUDA graphs, no flush (us, roofline), "
+                         "and each layer launched alone after a 256 MB write has flushed L2 (us_cold)"},
         "effective_gflops_nonzero": sum(r["flops"] for r in per) / (elapsed / args.steps) / 1e9,
         "e2e": {"value": imgs / e2e_elapsed, "unit": "images/s", "h2d_bytes_per_step": int(x.nbytes),
                 "d2h_bytes_per_step": int(batch * 1000 * 4)},

@@ -322,6 +322,17 @@ SBNN_API sbnn_status sbnn_mobilenet_v1_run_layer(sbnn_mbv1* net, int layer, cons
 SBNN_API sbnn_status sbnn_mobilenet_v1_run_layer_cm(sbnn_mbv1* net, int layer, const float* in_dev, float* out_dev,
                                                     int N, void* cuda_stream);
 
+/*
+ * The first last_layer + 1 layers of the forward pass (Section 3.5), launched exactly as sbnn_mobilenet_v1_forward
+ * launches them (same kernels, same workspaces, no CUDA graph of the library's own), with the output of layer
+ * last_layer written to out_dev in the chain's layout: channel-major [Cout][ld], ld = N*side*side rounded up to 4
+ * (the pool: [1024][N rounded up to 4]; layer 28: the logits [N][1000]).  Gives access to every intermediate
+ * activation of the chain, and, by timing consecutive prefixes, to the cost of each layer inside a step.  The call
+ * only enqueues; it may be captured into a caller's CUDA graph.  out_dev: 16-byte aligned device memory of the caller.
+ */
+SBNN_API sbnn_status sbnn_mobilenet_v1_forward_prefix(sbnn_mbv1* net, const float* x_dev, float* out_dev, int N,
+                                                      int last_layer, void* cuda_stream);
+
 /* Shape of a layer of the chain: input side, input channels, output side, output channels. */
 SBNN_API sbnn_status sbnn_mobilenet_v1_layer_shape(int layer, int* Hin, int* Cin, int* Hout, int* Cout);
 

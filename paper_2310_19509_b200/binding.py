@@ -57,6 +57,7 @@ def lib():
         "sbnn_avgpool": [P, P, I, I, I, P],
         "sbnn_mobilenet_v1_create": [P, P, P, P, P, P, I, P],
         "sbnn_mobilenet_v1_forward": [P, P, P, I, P],
+        "sbnn_mobilenet_v1_forward_prefix": [P, P, P, I, I, P],
         "sbnn_mobilenet_v1_run_layer": [P, I, P, P, I, P],
         "sbnn_mobilenet_v1_run_layer_cm": [P, I, P, P, I, P],
         "sbnn_mobilenet_v1_layer_shape": [I, P, P, P, P],
@@ -282,6 +283,10 @@ class MobileNetV1:
 
     def forward(self, x, logits, n, stream=None):
         _check(lib().sbnn_mobilenet_v1_forward(self._h, _ptr(x), _ptr(logits), n, _stream(stream)))
+
+    def forward_prefix(self, x, out, n, last_layer, stream=None):
+        """Layers 0..last_layer as forward launches them; the last one's output (chain layout) goes to `out`."""
+        _check(lib().sbnn_mobilenet_v1_forward_prefix(self._h, _ptr(x), _ptr(out), n, int(last_layer), _stream(stream)))
 
     def run_layer(self, layer, x, y, n, stream=None):
         _check(lib().sbnn_mobilenet_v1_run_layer(self._h, layer, _ptr(x), _ptr(y), n, _stream(stream)))

@@ -52,6 +52,8 @@ dwconv3x3_cm_vec_kernel(const float* __restrict__ w, const float* __restrict__ b
 #pragma unroll
     for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);      // weights are [3][3][C]
     const float bias = b ? __ldg(b + c) : 0.0f;
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     float acc[4] = {bias, bias, bias, bias};
     const float* xc = x + (size_t)c * ldx;
     const int ix0 = strip * 4 * S;                                 // first input column under the strip
@@ -110,6 +112,8 @@ dwconv3x3_cm_rows_kernel(const float* __restrict__ w, const float* __restrict__ 
     for (int o = 0; o < RR; ++o)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[o][i] = bias;
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     const float* xc = x + (size_t)c * ldx + (size_t)f0 * W + strip * 4;
     const bool first = strip == 0, last = strip == spr - 1;
     // all loads first (they are independent), so that a thread has RR + 2 rows in flight
@@ -174,6 +178,8 @@ dwconv3x3_cm_rows_s2_kernel(const float* __restrict__ w, const float* __restrict
     for (int o = 0; o < RR; ++o)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[o][i] = bias;
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     const float* xc = x + (size_t)c * ldx + (size_t)(2 * f0) * W + strip * 8;   // input row 2*f0, first column of the strip
     const bool first = strip == 0;
     float4 A[2 * RR + 1], B[2 * RR + 1];                           // all loads first: 2*RR + 1 rows in flight
@@ -247,6 +253,8 @@ dwconv3x3_cm_px_kernel(const float* __restrict__ w, const float* __restrict__ b,
             wk[kh * 3 + kw] = __ldg(w + (kh * 3 + kw) * C + c);
         }
     const float bias = b ? __ldg(b + c) : 0.0f;
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     const float* pc = x + (size_t)c * ldx + (size_t)n0 * HW + oy * S * W + ox * S;   // centre tap, first image
     float* yc = y + (size_t)c * ldy + (size_t)n0 * HoWo + q;
 #pragma unroll
@@ -289,6 +297,8 @@ dwconv3x3_cm_col7_kernel(const float* __restrict__ w, const float* __restrict__ 
 #pragma unroll
     for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);
     const float bias = b ? __ldg(b + c) : 0.0f;
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     const bool lok = ox > 0, rok = ox + 1 < W, top = oy0 > 0, bot = oy0 + 7 < H;
     const float* pc = x + (size_t)c * ldx + (size_t)n0 * H * W + (oy0 - 1) * W + ox;   // window origin (centre column)
     float* yc = y + (size_t)c * ldy + (size_t)n0 * H * W + oy0 * W + ox;
@@ -340,6 +350,8 @@ dwconv3x3_cm_w14_kernel(const float* __restrict__ w, const float* __restrict__ b
 #pragma unroll
     for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);
     const float bias = b ? __ldg(b + c) : 0.0f;
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     const float* pc = x + (size_t)c * ldx + (size_t)n0 * H * W + (oy0 - 1) * W + 2 * j;   // input row oy0 - 1, own pair
     float* yc = y + (size_t)c * ldy + (size_t)n0 * H * W + oy0 * W + 2 * j;
 #pragma unroll
@@ -398,6 +410,8 @@ conv3x3_thin_cm32_kernel(const float* __restrict__ w, const float* __restrict__ 
         ws[i] = w[(size_t)(cg * 32 + o) * 9 * Cin + tc];
     }
     __syncthreads();
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     constexpr int TW = 2, IW = S * (TW - 1) + 3;
     const int strips = (Wo + TW - 1) / TW;
     const long long total = (long long)N * Ho * strips;
@@ -481,6 +495,8 @@ conv3x3_first_s2c3_kernel(const float* __restrict__ w, const float* __restrict__
         ws[i] = w[(size_t)(cg * 32 + o) * 9 * Cin + tc];
     }
     __syncthreads();
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     const int strips = Wo >> 1;
     const long long total = (long long)N * Ho * strips;
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -550,6 +566,8 @@ conv3x3_first_s2c3_kernel(const float* __restrict__ w, const float* __restrict__
 // shuffle steps for 49 values.)
 __global__ void __launch_bounds__(256)
 avgpool_cm_kernel(const float* __restrict__ x, int ldx, float* __restrict__ y, int ldy, int N, int HW, int C) {
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int sub = threadIdx.x & 7;
     const long long pair0 = t >> 3, pairs = (long long)N * C;
@@ -604,33 +622,35 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
         const long long items = NHo / RR * (W / 4);
         if (stride == 1 && H % RR == 0 && items > 0 && items < 0x7fffffffLL / 2) {
             dim3 gr((unsigned)((items + 127) / 128), C);
-            dwconv3x3_cm_rows_kernel<RR><<<gr, 128, 0, st>>>(w, b, x, ldx, y, ldy, (int)items, H, W, relu);
+            SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_rows_kernel<RR>, gr, 128, 0, st, w, b, x, ldx, y, ldy, (int)items, H, W, relu));
         } else if (stride == 2 && Ho % 2 == 0 && NHo / 2 * (Wo / 4) > 0 && NHo / 2 * (Wo / 4) < 0x7fffffffLL / 2) {
             const long long items2 = NHo / 2 * (Wo / 4);
             dim3 gr((unsigned)((items2 + 127) / 128), C);
-            dwconv3x3_cm_rows_s2_kernel<2><<<gr, 128, 0, st>>>(w, b, x, ldx, y, ldy, (int)items2, Ho, W, relu);
-        } else if (stride == 1)
-            dwconv3x3_cm_vec_kernel<1><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu);
-        else
-            dwconv3x3_cm_vec_kernel<2><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu);
+            SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_rows_s2_kernel<2>, gr, 128, 0, st, w, b, x, ldx, y, ldy, (int)items2, Ho, W, relu));
+        } else if (stride == 1) {
+            SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_vec_kernel<1>, grid, 256, 0, st, w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu));
+        } else {
+            SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_vec_kernel<2>, grid, 256, 0, st, w, b, x, ldx, y, ldy, NHo, H, W, Ho, Wo, relu));
+        }
     } else {
         constexpr int NI = 4;
         const int QB = (Ho * Wo + 255) / 256;
         const int cpb = Ho * Wo < 256 ? 256 / (Ho * Wo) : 1;          // channels per CTA for small planes
         dim3 grid((unsigned)(QB * ((N + NI - 1) / NI)), (C + cpb - 1) / cpb);
-#define SBNN_DW_PX(S_, WT_) dwconv3x3_cm_px_kernel<S_, NI, WT_><<<grid, 256, 0, st>>>(w, b, x, ldx, y, ldy, N, H, W, C, QB, relu)
+#define SBNN_DW_PX(S_, WT_) \
+    SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_px_kernel<S_, NI, WT_>, grid, 256, 0, st, w, b, x, ldx, y, ldy, N, H, W, C, QB, relu))
 #define SBNN_DW_C7(WT_)                                                                                       \
     {                                                                                                         \
         const int items = (H / 7) * W, qb = (items + 127) / 128;                                              \
         const int cpb7 = items < 128 ? 128 / items : 1;                                                       \
         dim3 g7((unsigned)(qb * ((N + NI - 1) / NI)), (C + cpb7 - 1) / cpb7);                                 \
-        dwconv3x3_cm_col7_kernel<NI, WT_><<<g7, 128, 0, st>>>(w, b, x, ldx, y, ldy, N, H, C, relu);            \
+        SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_col7_kernel<NI, WT_>, g7, 128, 0, st, w, b, x, ldx, y, ldy, N, H, C, relu)); \
     }
         if (stride == 1) {
             if (W == 14 && H == 14 && ldx % 2 == 0 && ldy % 2 == 0) {
                 constexpr int NI2 = 2;
                 dim3 g14((unsigned)((N + NI2 - 1) / NI2), (C + 7) / 8);
-                dwconv3x3_cm_w14_kernel<NI2><<<g14, 128, 0, st>>>(w, b, x, ldx, y, ldy, N, C, relu);
+                SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_w14_kernel<NI2>, g14, 128, 0, st, w, b, x, ldx, y, ldy, N, C, relu));
             } else if (W == 14 && H % 7 == 0) SBNN_DW_C7(14)
             else if (W == 7 && H % 7 == 0) SBNN_DW_C7(7)
             else SBNN_DW_PX(1, 0);
@@ -655,13 +675,13 @@ sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* 
         if (blocks > 0x7fffffff) return fail(SBNN_ERR_SHAPE, "tensor too large");
         dim3 grid((unsigned)blocks, Cout / 32);
         const size_t smem = sizeof(float) * 9 * Cin * 32;
-        if (stride == 2 && Cin == 3 && W % 4 == 0 && H % 2 == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0)
-            conv3x3_first_s2c3_kernel<<<grid, 128, smem, st>>>(w, b, x, y, ldy, N, H, W, Cout, Ho, Wo, relu);
-        else if (stride == 1)
-            conv3x3_thin_cm32_kernel<1><<<grid, 128, smem, st>>>(w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu);
-        else
-            conv3x3_thin_cm32_kernel<2><<<grid, 128, smem, st>>>(w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu);
-        SBNN_CUDA_TRY(cudaGetLastError());
+        if (stride == 2 && Cin == 3 && W % 4 == 0 && H % 2 == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+            SBNN_CUDA_TRY(launch_kernel(conv3x3_first_s2c3_kernel, grid, 128, smem, st, w, b, x, y, ldy, N, H, W, Cout, Ho, Wo, relu));
+        } else if (stride == 1) {
+            SBNN_CUDA_TRY(launch_kernel(conv3x3_thin_cm32_kernel<1>, grid, 128, smem, st, w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu));
+        } else {
+            SBNN_CUDA_TRY(launch_kernel(conv3x3_thin_cm32_kernel<2>, grid, 128, smem, st, w, b, x, y, ldy, N, H, W, Cin, Cout, Ho, Wo, relu));
+        }
         return SBNN_OK;
     }
     return fail(SBNN_ERR_UNSUPPORTED, "channel-major first layer needs Cout %% 32 == 0 and an even leading dimension");
@@ -669,8 +689,7 @@ sbnn_status launch_conv3x3_thin_cm(const float* w, const float* b, const float* 
 
 sbnn_status launch_avgpool_cm(const float* x, int ldx, float* y, int ldy, int N, int HW, int C, cudaStream_t st) {
     const long long threads = (long long)N * C * 8;
-    avgpool_cm_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(x, ldx, y, ldy, N, HW, C);
-    SBNN_CUDA_TRY(cudaGetLastError());
+    SBNN_CUDA_TRY(launch_kernel(avgpool_cm_kernel, dim3((unsigned)((threads + 255) / 256)), 256, 0, st, x, ldx, y, ldy, N, HW, C));
     return SBNN_OK;
 }
 

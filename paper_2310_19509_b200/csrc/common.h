@@ -30,6 +30,34 @@ struct PrepareScope {
     ~PrepareScope();
 };
 
+// True while the calling thread is inside the MobileNet chain's forward pass: kernels are then launched with
+// programmatic stream serialization, i.e. a kernel may become resident and run its set-up while its predecessor in
+// the stream drains.  Every kernel launched this way executes grid_dependency_wait() (pipeline.cuh) before it reads or
+// writes anything another kernel of the stream touches.
+bool chained_launch();
+struct ChainedLaunchScope {
+    ChainedLaunchScope();
+    ~ChainedLaunchScope();
+};
+
+// Kernel launch that honours chained_launch().  Arguments are converted to the kernel's parameter types.
+template <class... Params, class... Args>
+cudaError_t launch_kernel(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (chained_launch()) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
+
 // Raises a kernel's dynamic shared-memory limit to `bytes` on the current device, once per (device, kernel) and size.
 sbnn_status set_max_dyn_smem(const void* func, int bytes);
 

@@ -271,12 +271,15 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
                 if (issued >= S) ok = mbar_wait(empty + s, ((issued / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
                 if (!ok) break;
                 if (lane == 0) {
-                    // one tiled copy brings the step's KC x TM box of X (pixels past M and channels past Cin
-                    // arrive as zeros and count towards the bytes), a linear one the step's weight block
+                    // a linear copy brings the step's weight block, one tiled copy the step's KC x TM box of X
+                    // (pixels past M and channels past Cin arrive as zeros and count towards the bytes).  The
+                    // weights do not depend on the previous kernel of the stream, the activations do: the very
+                    // first box is requested only once that kernel has finished.
                     const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
                     mbar_arrive_expect_tx(full + s, (uint32_t)C::XS_BYTES + (uint32_t)wn * 16u);
-                    tensor_g2s_2d(xs0 + (size_t)s * C::XS_BYTES, &xmap, m0, k * KC, full + s);
                     bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, full + s);
+                    if (issued == 0) grid_dependency_wait();
+                    tensor_g2s_2d(xs0 + (size_t)s * C::XS_BYTES, &xmap, m0, k * KC, full + s);
                 }
             }
         }
@@ -291,6 +294,8 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
     }
 
     // ---------------- compute warps ----------------
+    grid_dependency_wait();       // Y may still be read by the previous kernel of the stream
+    grid_dependency_release();
     const unsigned lane_off = lane * 16;
     int consumed = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
@@ -666,12 +671,11 @@ sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, 
     r = encode_x_map(x, ldx, M, p->Cin, C::TM, C::KC, &xmap);
     if (r != SBNN_OK) return r;
     if (out_cm)
-        conv1x1_cm_kernel<C, true><<<grid, C::NT, C::SMEM, st>>>(xmap, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
-                                                                 p->ngroups, s.nchunks, s.ntiles, total_tiles, relu, status);
+        SBNN_CUDA_TRY(launch_kernel(conv1x1_cm_kernel<C, true>, grid, C::NT, C::SMEM, st, xmap, y, ldy, p->d_bias, s.rec, s.blk_ptr, M,
+                                    p->Cin, p->Cout, p->ngroups, s.nchunks, s.ntiles, total_tiles, relu, status));
     else
-        conv1x1_cm_kernel<C, false><<<grid, C::NT, C::SMEM, st>>>(xmap, y, ldy, p->d_bias, s.rec, s.blk_ptr, M, p->Cin, p->Cout,
-                                                                  p->ngroups, s.nchunks, s.ntiles, total_tiles, relu, status);
-    SBNN_CUDA_TRY(cudaGetLastError());
+        SBNN_CUDA_TRY(launch_kernel(conv1x1_cm_kernel<C, false>, grid, C::NT, C::SMEM, st, xmap, y, ldy, p->d_bias, s.rec, s.blk_ptr, M,
+                                    p->Cin, p->Cout, p->ngroups, s.nchunks, s.ntiles, total_tiles, relu, status));
     return SBNN_OK;
 }
 

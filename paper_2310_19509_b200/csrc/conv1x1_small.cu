@@ -8,6 +8,7 @@
 // channel-major tensor (it stays in L1/L2 for the other groups' CTAs), and the unit's index and its G weights
 // are the same address for the whole warp.  No private weight layout: the canonical packed arrays are read.
 #include "common.h"
+#include "pipeline.cuh"
 
 namespace sbnn {
 namespace {
@@ -65,6 +66,8 @@ conv1x1_small_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y
     for (int r = 0; r < G; ++r) acc[r] = 0.0f;
     UnitRegs<G> cur, nxt;
     fetch_unit<G>(idx, val, u0 + lane, uend, cur);
+    grid_dependency_wait();      // X comes from the previous kernel of the stream; the weights above do not
+    grid_dependency_release();
     for (int ub = u0; ub < uend; ub += 32) {
         fetch_unit<G>(idx, val, ub + 32 + lane, uend, nxt);        // the next 32 units, while these are consumed
         const int cnt = min(32, uend - ub);                        // warp-uniform
@@ -119,9 +122,9 @@ sbnn_status launch_small_ks(const sbnn_packed* p, const float* x, int ldx, float
                             cudaStream_t st) {
     dim3 grid((unsigned)((M + 31) / 32), (unsigned)p->ngroups);
     if (out_cm)
-        conv1x1_small_kernel<G, KS, true><<<grid, 32 * KS, 0, st>>>(x, ldx, y, ldy, p->d_group_ptr, p->d_idx, p->d_val, p->d_bias, M, relu);
+        SBNN_CUDA_TRY(launch_kernel(conv1x1_small_kernel<G, KS, true>, grid, 32 * KS, 0, st, x, ldx, y, ldy, p->d_group_ptr, p->d_idx, p->d_val, p->d_bias, M, relu));
     else
-        conv1x1_small_kernel<G, KS, false><<<grid, 32 * KS, 0, st>>>(x, ldx, y, ldy, p->d_group_ptr, p->d_idx, p->d_val, p->d_bias, M, relu);
+        SBNN_CUDA_TRY(launch_kernel(conv1x1_small_kernel<G, KS, false>, grid, 32 * KS, 0, st, x, ldx, y, ldy, p->d_group_ptr, p->d_idx, p->d_val, p->d_bias, M, relu));
     SBNN_CUDA_TRY(cudaGetLastError());
     return SBNN_OK;
 }

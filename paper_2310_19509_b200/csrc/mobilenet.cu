@@ -225,10 +225,16 @@ extern "C" sbnn_status sbnn_mobilenet_v1_run_layer_cm(sbnn_mbv1* net, int layer,
 
 namespace {
 
-sbnn_status forward_plain(sbnn_mbv1* net, const float* x_dev, float* logits_dev, int N, void* stream) {
+// Layers 0 .. last on the ping-pong workspaces; the output of layer `last` goes to out_dev.
+sbnn_status forward_plain(sbnn_mbv1* net, const float* x_dev, float* out_dev, int N, void* stream,
+                          int last = SBNN_MBV1_NUM_LAYERS - 1) {
+    // The kernels are launched with programmatic stream serialization: each may become resident and run its
+    // set-up (barrier initialisation, weight fetches) while its predecessor drains, and waits for the
+    // predecessor's completion before it touches an activation buffer.
+    ChainedLaunchScope chained;
     const float* cur = x_dev;
-    for (int l = 0; l < SBNN_MBV1_NUM_LAYERS; ++l) {
-        float* dst = (l == SBNN_MBV1_NUM_LAYERS - 1) ? logits_dev : net->ws[l & 1];
+    for (int l = 0; l <= last; ++l) {
+        float* dst = (l == last) ? out_dev : net->ws[l & 1];
         sbnn_status st = run_cm(net, l, cur, dst, N, stream);
         if (st != SBNN_OK) return st;
         cur = dst;
@@ -289,6 +295,21 @@ extern "C" sbnn_status sbnn_mobilenet_v1_forward(sbnn_mbv1* net, const float* x_
     }
     SBNN_CUDA_TRY(cudaGraphLaunch(e.exec, user));
     return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_mobilenet_v1_forward_prefix(sbnn_mbv1* net, const float* x_dev, float* out_dev, int N,
+                                                        int last_layer, void* stream) {
+    clear_error();
+    if (!net || !x_dev || !out_dev) return fail(SBNN_ERR_NULL, "net, x_dev and out_dev must not be NULL");
+    if (last_layer < 0 || last_layer >= SBNN_MBV1_NUM_LAYERS) return fail(SBNN_ERR_SHAPE, "layer %d out of range", last_layer);
+    if (N < 0 || N > net->max_batch) return fail(SBNN_ERR_SHAPE, "N=%d outside [0, max_batch=%d]", N, net->max_batch);
+    if (!aligned16(out_dev)) return fail(SBNN_ERR_ALIGN, "out_dev must be 16-byte aligned");
+    if (out_dev == net->ws[0] || out_dev == net->ws[1]) return fail(SBNN_ERR_SHAPE, "out_dev must not be a workspace of the network");
+    if (N == 0) return SBNN_OK;
+    sbnn_status r = check_net_device(net);
+    if (r != SBNN_OK) return r;
+    std::lock_guard<std::mutex> lk(net->mu);
+    return forward_plain(net, x_dev, out_dev, N, stream, last_layer);
 }
 
 extern "C" sbnn_status sbnn_mobilenet_v1_free(sbnn_mbv1* net) {

@@ -72,6 +72,11 @@ bool prepare_only() { return g_prepare_depth > 0; }
 PrepareScope::PrepareScope() { ++g_prepare_depth; }
 PrepareScope::~PrepareScope() { --g_prepare_depth; }
 
+static thread_local int g_chained_depth = 0;
+bool chained_launch() { return g_chained_depth > 0; }
+ChainedLaunchScope::ChainedLaunchScope() { ++g_chained_depth; }
+ChainedLaunchScope::~ChainedLaunchScope() { --g_chained_depth; }
+
 sbnn_status set_max_dyn_smem(const void* func, int bytes) {
     static std::mutex mu;
     static std::map<std::pair<int, const void*>, int> limit;

@@ -26,6 +26,15 @@ __device__ __forceinline__ void fma2(f32x2& d, f32x2 a, f32x2 b) {
     asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// grid_dependency_wait: returns once every kernel this one depends on in its stream has completed and its writes are
+// visible (immediately if the kernel was launched without programmatic serialization).  Code before it may only
+// touch memory no other kernel of the stream writes (weights, its own shared memory).  grid_dependency_release lets
+// the next kernel of the stream become resident as SM resources free up; that kernel still waits, in its own
+// grid_dependency_wait, for this one to finish.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- mbarrier -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));

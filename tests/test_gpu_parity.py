@@ -257,6 +257,32 @@ def test_mobilenet_v1_batch1_layer_isolated_and_end_to_end(sparsity):
     net.free()
 
 
+def test_forward_prefix_gives_the_intermediate_activations():
+    """sbnn_mobilenet_v1_forward_prefix: the output of a middle pointwise layer, of the last depthwise layer and of the
+    pool, each in the chain's channel-major layout, against the oracle's chained result within its propagated bound;
+    the full prefix equals forward's logits bit for bit."""
+    x, layers = mobilenet_v1_inputs(1, 30, 4, seed=0)
+    outs = R.mobilenet_v1_forward(x, layers)
+    net = build_net(layers, 1)
+    xd = dev(x)
+    for li in (6, 25, 27):
+        ref, e = outs[li]["ref"], outs[li]["E"]
+        n_, h_, w_, c_ = ref.shape
+        ld = (n_ * h_ * w_ + 3) // 4 * 4
+        out = Guarded((c_, ld))
+        net.forward_prefix(xd, out.t, 1, li)
+        sbnn.get_async_status()
+        y = out.numpy(f"prefix {li}")[:, :n_ * h_ * w_].T.reshape(ref.shape).astype(np.float64)
+        err = np.abs(y - ref)
+        assert np.all(err <= e), f"layer {li}: worst ratio {np.max(err / np.maximum(e, 1e-300))}"
+    lg, lp = Guarded((1, 1000)), Guarded((1, 1000))
+    net.forward(xd, lg.t, 1)
+    net.forward_prefix(xd, lp.t, 1, 28)
+    sbnn.get_async_status()
+    assert np.array_equal(lg.numpy("forward"), lp.numpy("prefix 28"))
+    net.free()
+
+
 def test_forward_graph_replay_matches_plain_launches():
     """forward records a CUDA graph on its second call with the same buffers and replays it afterwards: replays
     must give, bit for bit, what the plain first call gave, follow the current contents of the input buffer, and a
