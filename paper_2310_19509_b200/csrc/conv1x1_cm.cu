@@ -716,21 +716,41 @@ sbnn_status dispatch_cm(const sbnn_packed* p, const TileCfg& c, const float* x, 
 
 // Tile shape for a layer run on M pixels.  M <= 0 stands for "many pixels" (the choice made before M is known).
 TileCfg default_cfg_cm(const sbnn_packed* p, long long M) {
-    // Whole tiles are dealt to the SMs, so a launch takes ceil(tiles / SMs) rounds of one tile each, and a tile's
-    // time grows with its compute warps.  Among the warp counts instantiated for the layer's G take the one with
-    // the cheapest rounds (CTAs of 11 or 12 compute warps run about 5 % more efficiently per warp than 8), and
-    // stay with 8 unless another is at least 3 % cheaper.
-    auto rounds_cost = [&](const TileCfg& c) {
+    // Whole tiles are dealt to the persistent CTAs (CTA b takes tiles b, b + SMs, ...), and inside a CTA warp w runs
+    // on scheduler w % 4, so a tile lasts as long as the scheduler with the most busy warps, and the launch as long as
+    // the CTA with the most work.  The cost of a tile shape is that maximum, computed exactly from the layer's group
+    // count (warps of a ragged last group tile are idle).  Measured on the 1024 -> 1024 layer with 64-channel steps:
+    // 8 warps (2 per scheduler) 1034 us, 12 warps (3 per scheduler) 1039 us, 11 warps 1109 us -- eleven warps cost as
+    // much per tile as twelve; three warps on a scheduler hide about 2 % more latency than two.
+    auto launch_cost = [&](const TileCfg& c) {
         const long long ptiles = (M + c.TM() - 1) / c.TM(), gtiles = (p->ngroups + c.GT() - 1) / c.GT();
-        const long long sms = std::max(1, sm_count());
-        return (double)((ptiles * gtiles + sms - 1) / sms) * c.NW / (c.NW > 8 ? 1.05 : 1.0);
+        const long long sms = std::max(1, sm_count()), total = ptiles * gtiles;
+        auto tile_cost = [&](long long gtile) {
+            int load[4] = {0, 0, 0, 0};
+            for (int w = 0; w < c.NW; ++w)
+                if ((gtile * c.NW + w) * c.GPW < p->ngroups) ++load[w & 3];
+            const int m = std::max(std::max(load[0], load[1]), std::max(load[2], load[3]));
+            // (with the producer a 12-warp CTA has 13 warps, which the register file serves like 16: 128 registers a
+            // thread instead of the 154 the loop wants, measured 4-6 % slower per tile than the 11-warp CTA)
+            return (m >= 3 ? 0.98 * m : (double)m) * (c.NW == 12 ? 1.04 : 1.0);
+        };
+        double full_tile = 0.0;                      // cost of one pass over the group tiles of a pixel tile
+        for (long long g = 0; g < gtiles; ++g) full_tile += tile_cost(g);
+        if (total > 64 * sms) return (double)total / sms * full_tile / gtiles;   // many rounds: the average is exact enough
+        double worst = 0.0;
+        for (long long b = 0; b < std::min(sms, total); ++b) {
+            double sum = 0.0;
+            for (long long t = b; t < total; t += sms) sum += tile_cost(t % gtiles);
+            worst = std::max(worst, sum);
+        }
+        return worst;
     };
     auto pick = [&](const TileCfg& base, std::initializer_list<TileCfg> others) {
         if (M <= 0) return base;
         TileCfg best = base;
-        double best_cost = 0.97 * rounds_cost(base);
+        double best_cost = 0.99 * launch_cost(base);
         for (const TileCfg& c : others) {
-            const double cost = rounds_cost(c);
+            const double cost = launch_cost(c);
             if (cost < best_cost) {
                 best = c;
                 best_cost = cost;
