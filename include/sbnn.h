@@ -149,7 +149,9 @@ SBNN_API sbnn_status sbnn_prepare(const sbnn_packed* w, int N, int H, int W, int
 enum {
     SBNN_RELU = 1,    /* apply max(.,0) after the bias */
     SBNN_BF16_TC = 2, /* 1x1 only: round activations and weights to bf16 and contract on tensor cores, fp32 accumulate */
-    SBNN_OUT_CM = 4   /* sbnn_conv1x1_gs_cm only: write the output channel-major, [Cout][ldy] */
+    SBNN_OUT_CM = 4,  /* sbnn_conv1x1_gs_cm only: write the output channel-major, [Cout][ldy] */
+    SBNN_BF16_GATHER = 8 /* with SBNN_BF16_TC: contract per group over its kept channels only (warp-level MMA on gathered
+                            rows) instead of densely over the masked weights */
 };
 
 /*
@@ -158,8 +160,13 @@ enum {
  *   x_dev  [N][H][W][Cin] fp32, y_dev [N][H][W][Cout] fp32
  * Cin must be a multiple of 4 (else SBNN_ERR_UNSUPPORTED).  N*H*W == 0 returns SBNN_OK without a launch.
  * With SBNN_BF16_TC the activations and the kept weights are rounded to bf16 (to nearest even) and the
- * products are summed in fp32 on the tensor cores; bias and ReLU stay fp32.  The first call of a layer in
- * that mode builds a private re-layout of its weights (allocates and copies synchronously).
+ * products are summed in fp32 on the tensor cores; bias and ReLU stay fp32.  By default the contraction then runs
+ * densely over the masked weights (pruned weights are stored as zeros and multiplied: on the tcgen05 tensor cores
+ * that is faster than skipping them, because a group of G <= 8 output channels is too narrow an MMA); this needs
+ * Cin % 8 == 0 and Cout % 4 == 0, other shapes -- and every shape when SBNN_BF16_GATHER is added -- run the
+ * gathered kernel, which visits kept units only.  Both give the same result up to the order of the fp32 sums.
+ * The first call of a layer in either form builds a private re-layout of its weights (allocates and copies
+ * synchronously), and both convert X to bf16 in the per-device scratch buffer first.
  */
 SBNN_API sbnn_status sbnn_conv1x1_gs(const sbnn_packed* w, const float* x_dev, float* y_dev,
                                      int N, int H, int W, int flags, void* cuda_stream);

@@ -8,6 +8,7 @@ functions raises.
 from .binding import (  # noqa: F401
     SBNN_BF16_TC,
     SBNN_OUT_CM,
+    SBNN_BF16_GATHER,
     SBNN_RELU,
     MobileNetV1,
     Packed,

@@ -7,7 +7,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-SBNN_RELU, SBNN_BF16_TC, SBNN_OUT_CM = 1, 2, 4
+SBNN_RELU, SBNN_BF16_TC, SBNN_OUT_CM, SBNN_BF16_GATHER = 1, 2, 4, 8
 _lib = None
 
 

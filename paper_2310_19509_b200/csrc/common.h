@@ -121,6 +121,7 @@ struct sbnn_packed {
     mutable std::map<sbnn::TileCfg, sbnn::Stream1x1> streams_cm;   // channel-major kernel, see conv1x1_cm.cu
     mutable std::map<int, sbnn::Stream3x3> streams3x3;
     mutable void* bf16_stream = nullptr;  // see conv1x1_bf16.cu
+    mutable void* umma_weights = nullptr; // dense bf16 copy of the masked weights, see conv1x1_umma.cu
 };
 
 namespace sbnn {
@@ -142,8 +143,10 @@ sbnn_status async_status_word(int** out);
 // Fills a 128-byte tensor-map descriptor (CUtensorMap) for tiled copies out of an fp32 (elem_bytes 4) or bf16 (2)
 // tensor: `rank` dimensions, innermost first, `strides_bytes` for dimensions 1.. (multiples of 16), `box` = elements
 // copied per dimension.  Elements outside the tensor are delivered as zeros.
+// With swizzle128 the box's rows (at most 128 bytes) are written to shared memory with the 128-byte swizzle that the
+// tcgen05 operand descriptors expect.
 sbnn_status encode_tiled_map(void* out, const void* base, int elem_bytes, int rank, const unsigned long long* dims,
-                             const unsigned long long* strides_bytes, const unsigned* box);
+                             const unsigned long long* strides_bytes, const unsigned* box, bool swizzle128 = false);
 // Per-device scratch buffer for channel-major copies made on behalf of NHWC callers.  Grows on demand with a
 // synchronous allocation (the outgrown buffer is kept until the process exits, so work already enqueued or recorded
 // on it stays valid); growth while `st` is being captured is refused with SBNN_ERR_UNSUPPORTED.
@@ -161,6 +164,9 @@ sbnn_status conv1x1_small(const sbnn_packed* p, const float* x, int ldx, float* 
 // conv1x1_bf16.cu
 sbnn_status conv1x1_bf16(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st);
 void free_stream_bf16(sbnn_packed* p);
+// conv1x1_umma.cu: bf16 mode as a dense contraction over the masked weights (tcgen05); *done = false if the shape is not taken
+sbnn_status conv1x1_umma(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st, bool* done);
+void free_umma_weights(sbnn_packed* p);
 // conv3x3_gs.cu
 sbnn_status prepare_default_3x3(const sbnn_packed* p);
 void free_streams_3x3(sbnn_packed* p);

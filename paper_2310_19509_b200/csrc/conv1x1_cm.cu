@@ -621,7 +621,7 @@ sbnn_status get_encode(EncodeTiledFn* out) {
 // fp32 (elem_bytes 4) or bf16 (2) tensor of `rank` dimensions (innermost first), tiled copies of `box` elements,
 // zeros outside the tensor.
 sbnn_status encode_generic(void* out, const void* base, int elem_bytes, int rank, const unsigned long long* dims,
-                           const unsigned long long* strides_bytes, const unsigned* box) {
+                           const unsigned long long* strides_bytes, const unsigned* box, bool swizzle128 = false) {
     EncodeTiledFn encode = nullptr;
     sbnn_status r = get_encode(&encode);
     if (r != SBNN_OK) return r;
@@ -639,7 +639,8 @@ sbnn_status encode_generic(void* out, const void* base, int elem_bytes, int rank
     }
     const CUresult cr = encode(static_cast<CUtensorMap*>(out),
                                elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
-                               (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                               (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return fail(SBNN_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)cr);
     return SBNN_OK;
@@ -820,8 +821,9 @@ sbnn_status scratch_workspace(size_t bytes, cudaStream_t st, float** out) { retu
 sbnn_status async_status_word(int** out) { return status_word(out); }
 
 sbnn_status encode_tiled_map(void* out, const void* base, int elem_bytes, int rank, const unsigned long long* dims,
-                             const unsigned long long* strides_bytes, const unsigned* box) {
-    return encode_generic(out, base, elem_bytes, rank, dims, strides_bytes, box);
+                             const unsigned long long* strides_bytes, const unsigned* box, bool swizzle128) {
+    if (swizzle128 && (size_t)box[0] * elem_bytes > 128) return fail(SBNN_ERR_SHAPE, "a swizzled box row is at most 128 bytes");
+    return encode_generic(out, base, elem_bytes, rank, dims, strides_bytes, box, swizzle128);
 }
 
 sbnn_status prepare_default_cm(const sbnn_packed* p, long long M) {

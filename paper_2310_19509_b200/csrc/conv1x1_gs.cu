@@ -387,7 +387,9 @@ sbnn_status check_args(const sbnn_packed* w, const float* x, float* y, int N, in
     if (w->KH != 1 || w->KW != 1) return fail(SBNN_ERR_SHAPE, "packed layer is %dx%d, expected 1x1", w->KH, w->KW);
     if (N < 0 || H < 0 || W < 0) return fail(SBNN_ERR_SHAPE, "negative activation shape %dx%dx%d", N, H, W);
     if ((int64_t)N * H * W > 0x7fffffff) return fail(SBNN_ERR_SHAPE, "N*H*W exceeds 2^31-1");
-    if (flags & ~(SBNN_RELU | SBNN_BF16_TC)) return fail(SBNN_ERR_UNSUPPORTED, "unknown flag bits 0x%x", flags);
+    if (flags & ~(SBNN_RELU | SBNN_BF16_TC | SBNN_BF16_GATHER)) return fail(SBNN_ERR_UNSUPPORTED, "unknown flag bits 0x%x", flags);
+    if ((flags & SBNN_BF16_GATHER) && !(flags & SBNN_BF16_TC))
+        return fail(SBNN_ERR_UNSUPPORTED, "SBNN_BF16_GATHER selects a variant of SBNN_BF16_TC and needs that flag too");
     if (!aligned16(x) || !aligned16(y)) return fail(SBNN_ERR_ALIGN, "x_dev and y_dev must be 16-byte aligned");
     if (w->Cin % 4) return fail(SBNN_ERR_UNSUPPORTED, "Cin=%d is not a multiple of 4", w->Cin);
     if ((int64_t)N * H * W == 0) return SBNN_OK;
@@ -427,8 +429,14 @@ extern "C" sbnn_status sbnn_conv1x1_gs(const sbnn_packed* w, const float* x_dev,
     if (M == 0) return SBNN_OK;
     if ((st = check_device()) != SBNN_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (flags & SBNN_BF16_TC) return conv1x1_bf16(w, x_dev, y_dev, (int)M, flags & SBNN_RELU, s);
     bool done = false;
+    if (flags & SBNN_BF16_TC) {
+        // dense over the masked weights on the tcgen05 tensor cores, unless the gathered warp-level kernel is asked
+        // for or the shape is outside what the dense kernel takes
+        if (!(flags & SBNN_BF16_GATHER) && ((st = conv1x1_umma(w, x_dev, y_dev, (int)M, flags & SBNN_RELU, s, &done)) != SBNN_OK || done))
+            return st;
+        return conv1x1_bf16(w, x_dev, y_dev, (int)M, flags & SBNN_RELU, s);
+    }
     if ((st = conv1x1_via_cm(w, x_dev, y_dev, (int)M, flags & SBNN_RELU, s, &done)) != SBNN_OK || done) return st;
     return dispatch(w, choose_cfg(w, M), x_dev, y_dev, (int)M, flags & SBNN_RELU, s);
 }

@@ -53,7 +53,7 @@ extern "C" sbnn_status sbnn_prepare(const sbnn_packed* w, int N, int H, int W, i
     const float* x = reinterpret_cast<const float*>(uintptr_t(256));
     float* y = reinterpret_cast<float*>(uintptr_t(512));
     if (w->KH == 3) return sbnn_conv3x3_gs(w, x, y, N, H, W, flags & SBNN_RELU, nullptr);
-    sbnn_status st = sbnn_conv1x1_gs(w, x, y, N, H, W, flags & (SBNN_RELU | SBNN_BF16_TC), nullptr);
+    sbnn_status st = sbnn_conv1x1_gs(w, x, y, N, H, W, flags & (SBNN_RELU | SBNN_BF16_TC | SBNN_BF16_GATHER), nullptr);
     if (st != SBNN_OK || (flags & SBNN_BF16_TC)) return st;
     return prepare_all_cm(w);
 }

@@ -283,6 +283,7 @@ extern "C" sbnn_status sbnn_packed_free(sbnn_packed* p) {
         free_streams_1x1(p);
         free_streams_cm(p);
         free_stream_bf16(p);
+        free_umma_weights(p);
         free_streams_3x3(p);
         cudaFree(p->d_group_ptr);
         cudaFree(p->d_idx);

@@ -107,4 +107,22 @@ __device__ __forceinline__ void tensor_g2s_3d(void* dst_smem, const void* tensor
                  : "memory");
 }
 
+// ---- tiled copy shared -> global through a 2-D tensor map, tracked by the issuing thread's bulk groups ----
+// Stores the [box rows][box width] block at src_smem (laid out as the map's swizzle mode says, 128-byte aligned, 1024
+// with the 128-byte swizzle) to the box whose first element is (x, y); the part of the box outside the tensor is not
+// written (along x in whole 16-byte pieces).  x * element size must be a multiple of 16 bytes and neither coordinate
+// negative.  Shared-memory writes made with ordinary stores must be followed by fence_async_smem() in the writing
+// threads, and a barrier, before the copy is issued.
+__device__ __forceinline__ void tensor_s2g_2d(const void* tensor_map, int x, int y, const void* src_smem) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(tensor_map), "r"(x), "r"(y), "r"(smem_u32(src_smem))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits until all but the most recent one of the calling thread's bulk groups have finished READING their shared-memory source.
+__device__ __forceinline__ void bulk_wait_read_pending1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// Waits until the calling thread's bulk groups have completed altogether (their global writes are performed).
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 }  // namespace sbnn

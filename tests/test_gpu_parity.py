@@ -509,6 +509,33 @@ def test_bf16_tensor_core_mode(g):
         assert_within(y, ref, s, tol=1e-2, what=f"bf16 G={g} relu={relu} vs fp32 oracle")
 
 
+@pytest.mark.parametrize("g,cin,cout,m", [(8, 136, 264, 300), (4, 64, 128, 1000), (4, 1024, 1024, 128 * 3 + 5),
+                                          (16, 72, 48, 77), (4, 8, 4, 5), (8, 64, 512, 128 * 330 + 3)])
+def test_bf16_dense_tensor_core_path(g, cin, cout, m):
+    """SBNN_BF16_TC on shapes the tcgen05 kernel takes (Cin % 8 == 0): dense contraction over the masked weights.
+    Ragged pixel, channel and output-channel tiles, all three output-tile widths (64, 128, 256), and a case with
+    more tiles than two per SM, so that both accumulators and every pipeline stage are reused.  Against the
+    oracle on bf16-rounded operands at 1e-5 * S, against the fp32 oracle at the stated 1e-2 * S; the gathered
+    kernel (SBNN_BF16_GATHER) must agree with the same oracle."""
+    d = WL.single_conv_inputs(1, 1, m, cin, cout, 1, g, 50, seed=21, mask_mode="layer_global")
+    ref16, s16 = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True, bf16=True)
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    y = run_1x1(d, sbnn.SBNN_BF16_TC | sbnn.SBNN_RELU)
+    assert_within(y, ref16, s16, tol=1e-5, what=f"bf16 dense G={g} {cin}->{cout} M={m} vs bf16 oracle")
+    assert_within(y, ref, s, tol=1e-2, what=f"bf16 dense G={g} {cin}->{cout} M={m} vs fp32 oracle")
+    if m < 2000:
+        yg = run_1x1(d, sbnn.SBNN_BF16_TC | sbnn.SBNN_BF16_GATHER | sbnn.SBNN_RELU)
+        assert_within(yg, ref16, s16, tol=1e-5, what=f"bf16 gathered G={g} {cin}->{cout} M={m} vs bf16 oracle")
+
+
+def test_bf16_dense_path_without_relu_and_fully_pruned_layer():
+    for sp, relu in ((50, False), (100, True)):
+        d = WL.single_conv_inputs(1, 3, 50, 96, 40, 1, 4, sp, seed=22)
+        y = run_1x1(d, sbnn.SBNN_BF16_TC | (sbnn.SBNN_RELU if relu else 0))
+        ref16, s16 = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu, bf16=True)
+        assert_within(y, ref16, s16, tol=1e-5, what=f"bf16 dense sp={sp} relu={relu}")
+
+
 @pytest.mark.parametrize("g,cout", [(4, 12), (2, 6), (1, 5), (1, 16), (2, 22)])
 def test_bf16_mode_merged_groups_ragged_channel_count(g, cout):
     """Groups of fewer than 8 channels are merged into 8-column groups for the tensor cores; the last merged group
