@@ -42,6 +42,9 @@ struct K3 {
     static constexpr int UNIT = 1 + (9 * G + 3) / 4;   // record of one kept unit, 16-byte units
     static constexpr int HDR = (GT * 2 + 3) / 4;
     static constexpr int WS_U4 = HDR + GT * KC * UNIT;
+    // Pattern layers use a list of kept taps instead (quads of 4 taps: 4 offsets, then 4 x G weights), see build_stream3_taps.
+    static constexpr int TQUAD = 1 + G;
+    static constexpr int WS_U4_TAPS = HDR + GT * ((KC * 9 + 3) / 4 + 1) * TQUAD;
     static_assert(KC % 4 == 0, "KC");
 };
 
@@ -365,7 +368,7 @@ conv3x3_gs_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y
 // images: rows of a neighbouring image are replaced by a row of zeros kept beside the stages.  Waits are bounded.
 struct Map3 { alignas(64) unsigned char bytes[128]; };
 
-template <class C>
+template <class C, bool PAT>
 __global__ void __launch_bounds__(C::NT + 32, 1)
 conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, const float* __restrict__ bias,
                       const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, Geo3 geo, int relu, int S,
@@ -436,6 +439,8 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
         rowok[kh] = (kh == 0) ? (y > 0) : (kh == 2 ? (y < geo.H - 1) : true);
     }
     const float* zr = zrow + lx + 3;
+    const int lanebase = lrow * geo.pitch + lx + 3;                // tap (kh, kw) of a plane: + kh * pitch + kw, then CW inputs
+    const unsigned rowmask = (rowok[0] ? 1u : 0u) | 2u | (rowok[2] ? 4u : 0u);
 
     f32x2 acc[GPW][CW][GP];
 #pragma unroll
@@ -459,6 +464,42 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
         for (int q = 0; q < GPW; ++q) {
             const int2 hd = reinterpret_cast<const int2*>(ws)[gw * GPW + q];
             const uint4* r = ws + hd.x;
+            if constexpr (PAT) {
+                // Layers packed with kernel patterns (Section 3.3): the stream lists the kept taps of the group's kept
+                // kernels one by one, four to a record (offset of the tap's first input inside the stage with the kernel
+                // row in the top two bits, then the G weights of each), so pruned taps cost nothing and the loop has no
+                // data-dependent branch.  A list is padded to a whole record with taps of weight zero.
+                for (int it = 0; it < hd.y; ++it, r += C::TQUAD) {
+                    const uint4 off4 = r[0];
+                    const unsigned offs[4] = {off4.x, off4.y, off4.z, off4.w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const unsigned kh = offs[u] >> 30;
+                        const float* arow = ((rowmask >> kh) & 1u) ? xs + (offs[u] & 0x3FFFFFFFu) + lanebase : zr;
+                        f32x2 a[CW];
+#pragma unroll
+                        for (int i = 0; i < CW; ++i) a[i] = dup2(arow[i]);
+                        const float* wq = reinterpret_cast<const float*>(r + 1) + u * G;
+                        f32x2 w[GP];
+                        if constexpr (G % 4 == 0) {
+#pragma unroll
+                            for (int v = 0; v < G / 4; ++v) {
+                                const ulonglong2 t = reinterpret_cast<const ulonglong2*>(wq)[v];
+                                w[2 * v] = t.x;
+                                w[2 * v + 1] = t.y;
+                            }
+                        } else if constexpr (G == 2) {
+                            w[0] = *reinterpret_cast<const unsigned long long*>(wq);
+                        } else {
+                            w[0] = pack2(wq[0], 0.0f);
+                        }
+#pragma unroll
+                        for (int p = 0; p < CW; ++p)
+#pragma unroll
+                            for (int rr = 0; rr < GP; ++rr) fma2(acc[q][p][rr], a[p], w[rr]);
+                    }
+                }
+            } else {
             for (int it = 0; it < hd.y; ++it, r += C::UNIT) {
                 const float* plane = xs + r[0].x;
                 const float* wq = reinterpret_cast<const float*>(r + 1);   // [9][G]
@@ -489,6 +530,7 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
                             for (int rr = 0; rr < GP; ++rr) fma2(acc[q][p][rr], a[p + kw], w[rr]);
                     }
                 }
+            }
             }
         }
         __syncwarp();
@@ -606,6 +648,70 @@ sbnn_status build_stream3(const sbnn_packed* p, int GT, int KC, int plane, Strea
         cudaFree(s.blk_ptr);
         cudaGetLastError();
         return fail(SBNN_ERR_CUDA, "uploading the 3x3 weight stream: %s", cudaGetErrorString(e));
+    }
+    *out = s;
+    return SBNN_OK;
+}
+
+// Stream of a layer packed with kernel patterns, for the tiled-copy kernel: per (group tile, channel step) a header of
+// (start, records) per group, then per group the kept taps of its kept kernels in records of four:
+// [4 x offset][4 x G weights], offset = plane offset of the input channel + kh * pitch + kw (floats), kernel row kh in
+// bits 30-31.  The last record of a list is padded with taps of offset 0 and weight 0.
+sbnn_status build_stream3_taps(const sbnn_packed* p, int GT, int KC, int plane, int pitch, Stream3x3* out) {
+    const int G = p->G;
+    const int ntiles = (p->ngroups + GT - 1) / GT, nchunks = (p->Cin + KC - 1) / KC;
+    const int HDR = (GT * 2 + 3) / 4, TQUAD = 1 + G;
+    std::vector<int32_t> blk((size_t)ntiles * (nchunks + 1));
+    std::vector<uint32_t> rec;
+    int max_blk = 0;
+    try {
+        for (int t = 0; t < ntiles; ++t) {
+            for (int k = 0; k < nchunks; ++k) {
+                const size_t blk_beg = rec.size() / 4;
+                blk[(size_t)t * (nchunks + 1) + k] = (int32_t)blk_beg;
+                rec.resize(rec.size() + (size_t)HDR * 4, 0u);
+                for (int s = 0; s < GT; ++s) {
+                    const int g = t * GT + s;
+                    int lo = 0, hi = 0;
+                    if (g < p->ngroups) {
+                        const int32_t* b = p->idx.data() + p->group_ptr[g];
+                        const int32_t* e = p->idx.data() + p->group_ptr[g + 1];
+                        lo = (int)(std::lower_bound(b, e, k * KC) - p->idx.data());
+                        hi = (int)(std::lower_bound(b, e, (k + 1) * KC) - p->idx.data());
+                    }
+                    const size_t list_beg = rec.size();
+                    int ntaps = 0;
+                    for (int j = lo; j < hi; ++j)
+                        for (int tap = 0; tap < 9; ++tap) {
+                            if (!((p->tap_mask[j] >> tap) & 1u)) continue;
+                            if (ntaps % 4 == 0) rec.resize(rec.size() + (size_t)TQUAD * 4, 0u);
+                            const size_t base = list_beg + (size_t)(ntaps / 4) * TQUAD * 4;
+                            const int kh = tap / 3, kw = tap % 3, u = ntaps % 4;
+                            rec[base + u] = (uint32_t)((p->idx[j] - k * KC) * plane + kh * pitch + kw) | ((uint32_t)kh << 30);
+                            memcpy(&rec[base + 4 + (size_t)u * G], &p->val[((size_t)j * 9 + tap) * G], sizeof(float) * G);
+                            ++ntaps;
+                        }
+                    rec[blk_beg * 4 + 2 * s + 0] = (uint32_t)(list_beg / 4 - blk_beg);
+                    rec[blk_beg * 4 + 2 * s + 1] = (uint32_t)((ntaps + 3) / 4);
+                }
+                max_blk = std::max(max_blk, (int)(rec.size() / 4 - blk_beg));
+            }
+            blk[(size_t)t * (nchunks + 1) + nchunks] = (int32_t)(rec.size() / 4);
+        }
+    } catch (const std::bad_alloc&) {
+        return fail(SBNN_ERR_ALLOC, "out of host memory building the 3x3 tap stream");
+    }
+    Stream3x3 s;
+    s.ntiles = ntiles; s.nchunks = nchunks; s.max_blk = max_blk;
+    SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&s.rec), std::max<size_t>(rec.size() * 4, 16)));
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s.blk_ptr), blk.size() * 4);
+    if (e == cudaSuccess && !rec.empty()) e = cudaMemcpy(s.rec, rec.data(), rec.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(s.blk_ptr, blk.data(), blk.size() * 4, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(s.rec);
+        cudaFree(s.blk_ptr);
+        cudaGetLastError();
+        return fail(SBNN_ERR_CUDA, "uploading the 3x3 tap stream: %s", cudaGetErrorString(e));
     }
     *out = s;
     return SBNN_OK;
@@ -732,7 +838,10 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     g.nchunks = (p->Cin + C::KC - 1) / C::KC;
     g.dpp_row = g.dpp_x = 0;
     if (g.pitch > 256 || g.R + 2 > 256 || W % 4 || ldx % 4) return SBNN_OK;
-    const int stage_bytes = (C::KC * g.plane * 4 + C::WS_U4 * 16 + 127) / 128 * 128;
+    const bool pat = !p->tap_mask.empty();   // packed with kernel patterns: the kernel walks a list of kept taps
+    if (pat && (long long)C::KC * g.plane + 2LL * g.pitch + 2 >= (1LL << 30)) return SBNN_OK;
+    const int ws_u4 = pat ? C::WS_U4_TAPS : C::WS_U4;
+    const int stage_bytes = (C::KC * g.plane * 4 + ws_u4 * 16 + 127) / 128 * 128;
     const size_t tail = (size_t)2 * 3 * 8 + 16 + (size_t)g.pitch * 4;
     int S = 3;
     if ((size_t)S * stage_bytes + tail > 227 * 1024) S = 2;
@@ -741,18 +850,19 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     Stream3x3 s;
     {
         std::lock_guard<std::mutex> lk(p->mu);
-        const int key = (g.plane << 8) | (C::GT << 4) | (C::KC / 4);
+        const int key = (g.plane << 8) | (C::GT << 4) | (C::KC / 4) | (pat ? (1 << 30) : 0);
         auto it = p->streams3x3.find(key);
         if (it == p->streams3x3.end()) {
-            sbnn_status r = build_stream3(p, C::GT, C::KC, g.plane, &s);
+            sbnn_status r = pat ? build_stream3_taps(p, C::GT, C::KC, g.plane, g.pitch, &s) : build_stream3(p, C::GT, C::KC, g.plane, &s);
             if (r != SBNN_OK) return r;
             p->streams3x3[key] = s;
         } else {
             s = it->second;
         }
     }
-    if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
-    sbnn_status r = set_max_dyn_smem(reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C>), (int)smem);
+    if (s.max_blk > ws_u4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, ws_u4);
+    sbnn_status r = set_max_dyn_smem(pat ? reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C, true>)
+                                         : reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C, false>), (int)smem);
     if (r != SBNN_OK) return r;
     int* status = nullptr;
     if ((r = async_status_word(&status)) != SBNN_OK) return r;
@@ -767,7 +877,10 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     const unsigned box[3] = {(unsigned)g.pitch, (unsigned)(g.R + 2), (unsigned)C::KC};
     if ((r = encode_tiled_map(&xmap, xt, 4, 3, dims, strides, box)) != SBNN_OK) return r;
     dim3 grid((unsigned)((NH + g.R - 1) / g.R), s.ntiles);
-    conv3x3_gs_tma_kernel<C><<<grid, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status);
+    if (pat)
+        conv3x3_gs_tma_kernel<C, true><<<grid, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status);
+    else
+        conv3x3_gs_tma_kernel<C, false><<<grid, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status);
     SBNN_CUDA_TRY(cudaGetLastError());
     *done = true;
     return SBNN_OK;

@@ -395,6 +395,23 @@ def test_3x3_kernel_patterns(g, kept_taps):
     p.free()
 
 
+def test_3x3_kernel_patterns_on_config4_shape():
+    """Config 4's layer (28 x 28, 256 -> 256, G = 4, half of the kernels removed) on 2 images with the 56 four-tap
+    patterns on top: the tiled-copy kernel skips the pruned taps of every unit (several channel steps, two images in
+    one CTA's rows) and must still match the oracle's masked dense convolution."""
+    from sbnn_inputs import tap_pattern_mask
+    d = WL.config4(n=2)
+    m = tap_pattern_mask(0, 19, d["unit_mask"], 4, 4)
+    p = sbnn.pack_weights(d["w"], m, d["bias"], 4, tap_patterns=True)
+    n, h, w, _ = d["x"].shape
+    out = Guarded((n, h, w, 256))
+    sbnn.conv3x3_gs(p, dev(d["x"]), out.t, n, h, w, sbnn.SBNN_RELU)
+    sbnn.get_async_status()
+    ref, s = R.conv2d(d["x"], d["w"], m, d["bias"], relu=True)
+    assert_within(out.numpy("3x3 patterns"), ref, s, what="3x3 four-tap patterns, config-4 shape")
+    p.free()
+
+
 def test_3x3_row_too_wide_for_the_tiled_copy():
     """A 252-pixel row needs a plane pitch above the copy engine's 256-element box limit: the cp.async variant runs."""
     d = WL.single_conv_inputs(1, 3, 252, 12, 16, 3, 4, 50, seed=15, w_sigma=0.1)
