@@ -60,7 +60,8 @@ typedef enum {
     SBNN_ERR_ARCH = 7,                   /* current device is not compute capability 10.x */
     SBNN_ERR_ALLOC = 8,                  /* host or device allocation failed */
     SBNN_ERR_CUDA = 9,                   /* a CUDA runtime call failed or no device is present */
-    SBNN_ERR_TIMEOUT = 10                /* a bounded device-side wait gave up (reported by sbnn_get_async_status) */
+    SBNN_ERR_TIMEOUT = 10,               /* a bounded device-side wait gave up (reported by sbnn_get_async_status) */
+    SBNN_ERR_IO = 11                     /* a packed-layer file could not be opened, read or written, or is corrupt */
 } sbnn_status;
 
 /* Static name of a status code ("SBNN_OK", ...). Never NULL. */
@@ -125,6 +126,27 @@ SBNN_API sbnn_status sbnn_packed_get(const sbnn_packed* p, sbnn_packed_view* vie
 SBNN_API sbnn_status sbnn_unpack_weights(const sbnn_packed* p, float* W_host_out, uint8_t* mask_host_out);
 /* Frees host and device copies.  NULL is accepted. */
 SBNN_API sbnn_status sbnn_packed_free(sbnn_packed* p);
+
+/*
+ * Packed layers as files (Section 3.5: the conversion tool writes the pruned model in the engine's own sparse
+ * format, which the engine loads at start-up).  sbnn_packed_save writes the canonical arrays of one layer,
+ * sbnn_packed_load reads them back into a new packed layer: host copy plus, if a device is present, device copies,
+ * exactly as after packing.  File layout, little-endian, no padding:
+ *   bytes 0-7    magic 'S' 'B' 'N' 'N' 'P' 'K' 0x01 0x00
+ *   int32[8]     format version (1), Cout, KH, KW, Cin, G, has_tap_mask (0 or 1), 0
+ *   int64        nnz_units
+ *   int32        group_ptr[Cout/G + 1]
+ *   int32        idx[nnz_units]
+ *   float32      val[nnz_units][KH*KW][G]
+ *   float32      bias[Cout]
+ *   uint16       tap_mask[nnz_units]            only if has_tap_mask
+ *   uint64       FNV-1a (64 bit) of all preceding bytes
+ * Loading checks the magic, the version, the checksum and the structure (prefix sums, ascending in-range indices,
+ * non-empty tap masks) and returns SBNN_ERR_IO for a file that cannot be read, is truncated or corrupt,
+ * SBNN_ERR_UNSUPPORTED for another version and SBNN_ERR_SHAPE for inconsistent contents; *out is NULL then.
+ */
+SBNN_API sbnn_status sbnn_packed_save(const sbnn_packed* p, const char* path);
+SBNN_API sbnn_status sbnn_packed_load(const char* path, sbnn_packed** out);
 
 /*
  * Set-up step of the engine for one layer (Section 3.5: the model is converted once, ahead of inference):

@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     head_noalloc,
     lib,
     lib_path,
+    load_packed,
     mobilenet_v1_layer_shape,
     pack_dw_pattern,
     pack_weights,

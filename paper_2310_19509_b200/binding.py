@@ -44,6 +44,8 @@ def lib():
         "sbnn_packed_get": [P, P],
         "sbnn_unpack_weights": [P, P, P],
         "sbnn_packed_free": [P],
+        "sbnn_packed_save": [P, C.c_char_p],
+        "sbnn_packed_load": [C.c_char_p, P],
         "sbnn_conv1x1_gs": [P, P, P, I, I, I, I, P],
         "sbnn_conv1x1_gs_tuned": [P, P, P, I, I, I, I, I, I, I, I, P],
         "sbnn_conv3x3_gs": [P, P, P, I, I, I, I, P],
@@ -142,6 +144,10 @@ class Packed:
         _check(lib().sbnn_unpack_weights(self._h, w.ctypes.data, m.ctypes.data))
         return w, m
 
+    def save(self, path):
+        """Write the layer to a packed-layer file (see sbnn_packed_save for the layout)."""
+        _check(lib().sbnn_packed_save(self._h, os.fsencode(path)))
+
     def free(self):
         if self._h:
             lib().sbnn_packed_free(self._h)
@@ -152,6 +158,13 @@ class Packed:
             self.free()
         except Exception:
             pass
+
+
+def load_packed(path) -> Packed:
+    """Read a packed-layer file written by Packed.save / sbnn_packed_save."""
+    h = C.c_void_p()
+    _check(lib().sbnn_packed_load(os.fsencode(path), C.byref(h)))
+    return Packed(h)
 
 
 def pack_weights(w, mask, bias, g, tap_patterns=False) -> Packed:

@@ -121,6 +121,7 @@ extern "C" const char* sbnn_status_str(sbnn_status s) {
         case SBNN_ERR_ALLOC: return "SBNN_ERR_ALLOC";
         case SBNN_ERR_CUDA: return "SBNN_ERR_CUDA";
         case SBNN_ERR_TIMEOUT: return "SBNN_ERR_TIMEOUT";
+        case SBNN_ERR_IO: return "SBNN_ERR_IO";
     }
     return "SBNN_ERR_UNKNOWN";
 }
@@ -128,6 +129,31 @@ extern "C" const char* sbnn_status_str(sbnn_status s) {
 extern "C" const char* sbnn_last_error(void) { return g_err; }
 
 namespace {
+// Last step of packing and of loading: device copies of the canonical arrays and the default private layouts, if
+// there is a device; *out owns p afterwards (on failure p is freed).
+sbnn_status finish_packed(sbnn_packed* p, sbnn_packed** out) {
+    int ndev = 0, dev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0 || cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        *out = p;
+        return SBNN_OK;
+    }
+    sbnn_status st = SBNN_OK;
+    p->device = dev;
+    if ((st = upload(&p->d_group_ptr, p->group_ptr)) != SBNN_OK || (st = upload(&p->d_idx, p->idx)) != SBNN_OK ||
+        (st = upload(&p->d_val, p->val)) != SBNN_OK || (st = upload(&p->d_bias, p->bias)) != SBNN_OK) {
+        sbnn_packed_free(p);
+        return st;
+    }
+    st = (p->KH == 1) ? prepare_default_1x1(p) : prepare_default_3x3(p);
+    if (st != SBNN_OK) {
+        sbnn_packed_free(p);
+        return st;
+    }
+    *out = p;
+    return SBNN_OK;
+}
+
 // tap_patterns = false: a unit's mask is one value for all taps (connectivity pruning only).
 // tap_patterns = true: the taps of a unit may differ (kernel patterns), but not between the G filters of the group;
 // a unit is kept if any of its taps is, pruned taps are stored as zeros and remembered in tap_mask.
@@ -206,27 +232,7 @@ sbnn_status pack_impl(const float* W, const uint8_t* mask, const float* bias, in
         return fail(SBNN_ERR_ALLOC, "out of host memory while packing");
     }
 
-    // Device copies, if there is a device.
-    int ndev = 0, dev = 0;
-    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0 || cudaGetDevice(&dev) != cudaSuccess) {
-        cudaGetLastError();
-        *out = p;
-        return SBNN_OK;
-    }
-    sbnn_status st = SBNN_OK;
-    p->device = dev;
-    if ((st = upload(&p->d_group_ptr, p->group_ptr)) != SBNN_OK || (st = upload(&p->d_idx, p->idx)) != SBNN_OK ||
-        (st = upload(&p->d_val, p->val)) != SBNN_OK || (st = upload(&p->d_bias, p->bias)) != SBNN_OK) {
-        sbnn_packed_free(p);
-        return st;
-    }
-    st = (KH == 1) ? prepare_default_1x1(p) : prepare_default_3x3(p);
-    if (st != SBNN_OK) {
-        sbnn_packed_free(p);
-        return st;
-    }
-    *out = p;
-    return SBNN_OK;
+    return finish_packed(p, out);
 }
 }  // namespace
 
@@ -272,6 +278,127 @@ extern "C" sbnn_status sbnn_unpack_weights(const sbnn_packed* p, float* W, uint8
                 }
         }
     return SBNN_OK;
+}
+
+// ---- packed-layer files ------------------------------------------------------------------------------------
+namespace {
+const unsigned char kFileMagic[8] = {'S', 'B', 'N', 'N', 'P', 'K', 1, 0};
+
+// FNV-1a, 64 bit, over the bytes of the file that precede the checksum.
+struct Fnv {
+    uint64_t h = 1469598103934665603ull;
+    void add(const void* data, size_t n) {
+        const unsigned char* b = static_cast<const unsigned char*>(data);
+        for (size_t i = 0; i < n; ++i) h = (h ^ b[i]) * 1099511628211ull;
+    }
+};
+
+struct FileCloser {
+    FILE* f;
+    ~FileCloser() { if (f) fclose(f); }
+};
+}  // namespace
+
+extern "C" sbnn_status sbnn_packed_save(const sbnn_packed* p, const char* path) {
+    clear_error();
+    if (!p || !path) return fail(SBNN_ERR_NULL, "packed and path must not be NULL");
+    FileCloser fc{fopen(path, "wb")};
+    if (!fc.f) return fail(SBNN_ERR_IO, "cannot open %s for writing", path);
+    Fnv sum;
+    bool ok = true;
+    auto put = [&](const void* d, size_t n) {
+        sum.add(d, n);
+        ok = ok && (n == 0 || fwrite(d, 1, n, fc.f) == n);
+    };
+    const int32_t hdr[8] = {1, p->Cout, p->KH, p->KW, p->Cin, p->G, p->tap_mask.empty() ? 0 : 1, 0};
+    const int64_t nnz = p->nnz;
+    put(kFileMagic, 8);
+    put(hdr, sizeof(hdr));
+    put(&nnz, 8);
+    put(p->group_ptr.data(), p->group_ptr.size() * 4);
+    put(p->idx.data(), p->idx.size() * 4);
+    put(p->val.data(), p->val.size() * 4);
+    put(p->bias.data(), p->bias.size() * 4);
+    put(p->tap_mask.data(), p->tap_mask.size() * 2);
+    const uint64_t h = sum.h;
+    ok = ok && fwrite(&h, 1, 8, fc.f) == 8;
+    ok = ok && fflush(fc.f) == 0;
+    if (!ok) return fail(SBNN_ERR_IO, "short write to %s", path);
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_packed_load(const char* path, sbnn_packed** out) {
+    clear_error();
+    if (!path || !out) return fail(SBNN_ERR_NULL, "path and out must not be NULL");
+    *out = nullptr;
+    FileCloser fc{fopen(path, "rb")};
+    if (!fc.f) return fail(SBNN_ERR_IO, "cannot open %s", path);
+    Fnv sum;
+    bool ok = true;
+    auto get = [&](void* d, size_t n) {
+        ok = ok && (n == 0 || fread(d, 1, n, fc.f) == n);
+        if (ok) sum.add(d, n);
+    };
+    unsigned char magic[8];
+    int32_t hdr[8];
+    int64_t nnz = 0;
+    get(magic, 8);
+    get(hdr, sizeof(hdr));
+    get(&nnz, 8);
+    if (!ok) return fail(SBNN_ERR_IO, "%s is too short to be a packed layer", path);
+    if (memcmp(magic, kFileMagic, 8) != 0) return fail(SBNN_ERR_IO, "%s is not a packed-layer file (bad magic)", path);
+    if (hdr[0] != 1) return fail(SBNN_ERR_UNSUPPORTED, "%s has format version %d, this library reads version 1", path, hdr[0]);
+    const int Cout = hdr[1], KH = hdr[2], KW = hdr[3], Cin = hdr[4], G = hdr[5], has_taps = hdr[6];
+    if (Cout <= 0 || Cin <= 0 || !((KH == 1 && KW == 1) || (KH == 3 && KW == 3)) || !supported_group(G) || Cout % G ||
+        (has_taps != 0 && has_taps != 1) || nnz < 0 || nnz > (int64_t)(Cout / G) * Cin)
+        return fail(SBNN_ERR_SHAPE, "%s: inconsistent header (Cout=%d KH=%d KW=%d Cin=%d G=%d units=%lld)", path, Cout, KH, KW, Cin,
+                    G, (long long)nnz);
+    sbnn_packed* p = new (std::nothrow) sbnn_packed;
+    if (!p) return fail(SBNN_ERR_ALLOC, "out of host memory");
+    p->Cout = Cout; p->KH = KH; p->KW = KW; p->Cin = Cin; p->G = G; p->ngroups = Cout / G; p->nnz = nnz;
+    const int taps = KH * KW;
+    try {
+        p->group_ptr.resize(p->ngroups + 1);
+        p->idx.resize(nnz);
+        p->val.resize((size_t)nnz * taps * G);
+        p->bias.resize(Cout);
+        if (has_taps) p->tap_mask.resize(nnz);
+    } catch (const std::bad_alloc&) {
+        delete p;
+        return fail(SBNN_ERR_ALLOC, "out of host memory while loading %s", path);
+    }
+    get(p->group_ptr.data(), p->group_ptr.size() * 4);
+    get(p->idx.data(), p->idx.size() * 4);
+    get(p->val.data(), p->val.size() * 4);
+    get(p->bias.data(), p->bias.size() * 4);
+    get(p->tap_mask.data(), p->tap_mask.size() * 2);
+    uint64_t stored = 0;
+    const uint64_t computed = sum.h;
+    const bool have_sum = ok && fread(&stored, 1, 8, fc.f) == 8;
+    unsigned char extra;
+    const bool trailing = have_sum && fread(&extra, 1, 1, fc.f) == 1;
+    sbnn_status st = SBNN_OK;
+    if (!ok || !have_sum) st = fail(SBNN_ERR_IO, "%s is truncated", path);
+    else if (trailing) st = fail(SBNN_ERR_IO, "%s has bytes after the checksum", path);
+    else if (stored != computed) st = fail(SBNN_ERR_IO, "%s: checksum mismatch (file is corrupt)", path);
+    // structure: prefix sums, ascending in-range indices, tap masks inside the kernel and not empty
+    if (st == SBNN_OK && (p->group_ptr[0] != 0 || p->group_ptr[p->ngroups] != nnz))
+        st = fail(SBNN_ERR_SHAPE, "%s: group_ptr does not span the kept units", path);
+    for (int g = 0; st == SBNN_OK && g < p->ngroups; ++g) {
+        const int64_t lo = p->group_ptr[g], hi = p->group_ptr[g + 1];
+        if (lo > hi || hi > nnz) st = fail(SBNN_ERR_SHAPE, "%s: group_ptr is not monotone at group %d", path, g);
+        for (int64_t u = lo; st == SBNN_OK && u < hi; ++u) {
+            if (p->idx[u] < 0 || p->idx[u] >= Cin || (u > lo && p->idx[u] <= p->idx[u - 1]))
+                st = fail(SBNN_ERR_SHAPE, "%s: indices of group %d are not ascending inside [0, Cin)", path, g);
+            else if (has_taps && (p->tap_mask[u] == 0 || (p->tap_mask[u] >> taps) != 0))
+                st = fail(SBNN_ERR_SHAPE, "%s: tap mask of unit %lld is empty or reaches outside the kernel", path, (long long)u);
+        }
+    }
+    if (st != SBNN_OK) {
+        delete p;
+        return st;
+    }
+    return finish_packed(p, out);
 }
 
 extern "C" sbnn_status sbnn_packed_free(sbnn_packed* p) {

@@ -299,3 +299,111 @@ def test_weights_of_another_device_are_refused_without_a_launch():
     finally:
         for q, d in zip((p, p3), was):
             sbnn.debug_set_packed_device(q, d)                                        # so that free() releases the real copies
+
+
+# ---- packed-layer files (Section 3.5: the engine loads the converted model from its own sparse format) ----------
+
+def _read_packed_file(path):
+    """Independent reader of the documented file layout (include/sbnn.h), written from that description alone."""
+    import struct
+    raw = open(path, "rb").read()
+    assert raw[:8] == b"SBNNPK\x01\x00"
+    ver, cout, kh, kw, cin, g, has_taps, zero = struct.unpack_from("<8i", raw, 8)
+    (nnz,) = struct.unpack_from("<q", raw, 40)
+    off = 48
+    ng = cout // g
+    gp = np.frombuffer(raw, "<i4", ng + 1, off); off += 4 * (ng + 1)
+    idx = np.frombuffer(raw, "<i4", nnz, off); off += 4 * nnz
+    val = np.frombuffer(raw, "<f4", nnz * kh * kw * g, off).reshape(nnz, kh * kw, g); off += 4 * nnz * kh * kw * g
+    bias = np.frombuffer(raw, "<f4", cout, off); off += 4 * cout
+    taps = None
+    if has_taps:
+        taps = np.frombuffer(raw, "<u2", nnz, off); off += 2 * nnz
+    (stored,) = struct.unpack_from("<Q", raw, off)
+    assert off + 8 == len(raw)
+    h = 1469598103934665603
+    for byte in raw[:off]:
+        h = ((h ^ byte) * 1099511628211) & 0xFFFFFFFFFFFFFFFF
+    assert h == stored, "FNV-1a checksum of the file"
+    return dict(ver=ver, cout=cout, kh=kh, kw=kw, cin=cin, g=g, zero=zero, gp=gp, idx=idx, val=val, bias=bias, taps=taps)
+
+
+@pytest.mark.parametrize("k,g,cin,cout,patterns", [(1, 4, 24, 16, False), (3, 4, 12, 8, False), (3, 2, 10, 6, True),
+                                                   (1, 8, 16, 8, False)])
+def test_packed_layer_file_round_trip_and_layout(tmp_path, k, g, cin, cout, patterns):
+    rng = np.random.default_rng(31)
+    w = rng.standard_normal((cout, k, k, cin)).astype(np.float32)
+    b = rng.standard_normal(cout).astype(np.float32)
+    um = group_mask_layer_global(2, 3, cout // g, cin, 55)
+    m = tap_pattern_mask(2, 19, um, g, 4) if patterns else expand_mask(um, g, k, k)
+    p = sbnn.pack_weights(w, m, b, g, tap_patterns=patterns)
+    path = str(tmp_path / "layer.sbnn")
+    p.save(path)
+    # (i) the bytes on disk, read by a reader of our own, are the oracle's packing of the same layer
+    f = _read_packed_file(path)
+    assert (f["ver"], f["cout"], f["kh"], f["kw"], f["cin"], f["g"], f["zero"]) == (1, cout, k, k, cin, g, 0)
+    if patterns:
+        gp, idx, val, taps = R.pack_pattern(w, m, g)
+        assert np.array_equal(f["taps"], taps)
+    else:
+        gp, idx, val = R.pack(w, m, g)
+        assert f["taps"] is None
+    assert np.array_equal(f["gp"], gp) and np.array_equal(f["idx"], idx)
+    assert f["val"].tobytes() == np.asarray(val, np.float32).tobytes() and f["bias"].tobytes() == b.tobytes()
+    # (ii) loading gives back an identical layer
+    q = sbnn.load_packed(path)
+    v0, v1 = p.view(), q.view()
+    for key in v0:
+        a0, a1 = v0[key], v1[key]
+        if isinstance(a0, np.ndarray):
+            assert a0.dtype == a1.dtype and a0.tobytes() == a1.tobytes(), key
+        else:
+            assert a0 == a1 or (a0 is None and a1 is None), key
+    w2, m2 = q.unpack()
+    assert np.array_equal(m2, m)
+    p.free(); q.free()
+
+
+def test_packed_layer_file_errors(tmp_path):
+    rng = np.random.default_rng(32)
+    w = rng.standard_normal((8, 1, 1, 12)).astype(np.float32)
+    m = expand_mask(group_mask_balanced(3, 3, 2, 12, 50), 4, 1, 1)
+    p = sbnn.pack_weights(w, m, None, 4)
+    good = str(tmp_path / "good.sbnn")
+    p.save(good)
+    raw = open(good, "rb").read()
+    p.free()
+
+    def load(data, name):
+        path = str(tmp_path / name)
+        open(path, "wb").write(data)
+        with pytest.raises(sbnn.SbnnError) as e:
+            sbnn.load_packed(path)
+        return e.value.name
+
+    assert load(raw[:-3], "truncated") == "SBNN_ERR_IO"
+    assert load(raw[:20], "short") == "SBNN_ERR_IO"
+    assert load(raw + b"\0", "trailing") == "SBNN_ERR_IO"
+    assert load(b"NOTSBNN!" + raw[8:], "magic") == "SBNN_ERR_IO"
+    flipped = bytearray(raw); flipped[60] ^= 0x40
+    assert load(bytes(flipped), "flipped") == "SBNN_ERR_IO"                     # checksum
+    v2 = bytearray(raw); v2[8] = 2
+    assert load(bytes(v2), "version") == "SBNN_ERR_UNSUPPORTED"
+    with pytest.raises(sbnn.SbnnError) as e:
+        sbnn.load_packed(str(tmp_path / "missing.sbnn"))
+    assert e.value.name == "SBNN_ERR_IO"
+    with pytest.raises(sbnn.SbnnError) as e:
+        sbnn.pack_weights(w, m, None, 4).save(str(tmp_path / "no_such_dir" / "x.sbnn"))
+    assert e.value.name == "SBNN_ERR_IO"
+
+    # a file whose checksum is right but whose indices are not ascending is refused as inconsistent
+    import struct
+    bad = bytearray(raw[:-8])
+    ng = 2
+    off_idx = 48 + 4 * (ng + 1)
+    i0, i1 = struct.unpack_from("<2i", bad, off_idx)
+    struct.pack_into("<2i", bad, off_idx, i1, i0)
+    h = 1469598103934665603
+    for byte in bad:
+        h = ((h ^ byte) * 1099511628211) & 0xFFFFFFFFFFFFFFFF
+    assert load(bytes(bad) + struct.pack("<Q", h), "unsorted") == "SBNN_ERR_SHAPE"

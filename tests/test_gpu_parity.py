@@ -501,6 +501,39 @@ def test_channel_major_kernel_edge_cases():
         assert_within(y, ref, s, what=f"cm sp={sp}")
 
 
+def test_layer_loaded_from_a_file_computes_bit_for_bit_what_the_packed_one_does(tmp_path):
+    """sbnn_packed_save / sbnn_packed_load: the loaded layer has its own device copies and private layouts and must give
+    the very bits the original gives (1x1 through the pipelined kernel, 3x3 with kernel patterns through the tap lists)."""
+    from sbnn_inputs import tap_pattern_mask
+    d = WL.single_conv_inputs(1, 40, 60, 160, 96, 1, 4, 50, seed=23)
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    p.save(str(tmp_path / "pw.sbnn"))
+    q = sbnn.load_packed(str(tmp_path / "pw.sbnn"))
+    xd = dev(d["x"])
+    ya, yb = Guarded((1, 40, 60, 96)), Guarded((1, 40, 60, 96))
+    sbnn.conv1x1_gs(p, xd, ya.t, 1, 40, 60, sbnn.SBNN_RELU)
+    sbnn.conv1x1_gs(q, xd, yb.t, 1, 40, 60, sbnn.SBNN_RELU)
+    sbnn.get_async_status()
+    assert np.array_equal(ya.numpy("packed"), yb.numpy("loaded"))
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    assert_within(yb.numpy("loaded"), ref, s, what="loaded 1x1 layer")
+    p.free(); q.free()
+    d3 = WL.single_conv_inputs(2, 12, 28, 24, 32, 3, 4, 50, seed=24, w_sigma=0.1)
+    m = tap_pattern_mask(24, 19, d3["unit_mask"], 4, 4)
+    p3 = sbnn.pack_weights(d3["w"], m, d3["bias"], 4, tap_patterns=True)
+    p3.save(str(tmp_path / "c3.sbnn"))
+    q3 = sbnn.load_packed(str(tmp_path / "c3.sbnn"))
+    x3 = dev(d3["x"])
+    za, zb = Guarded((2, 12, 28, 32)), Guarded((2, 12, 28, 32))
+    sbnn.conv3x3_gs(p3, x3, za.t, 2, 12, 28, sbnn.SBNN_RELU)
+    sbnn.conv3x3_gs(q3, x3, zb.t, 2, 12, 28, sbnn.SBNN_RELU)
+    sbnn.get_async_status()
+    assert np.array_equal(za.numpy("packed 3x3"), zb.numpy("loaded 3x3"))
+    ref3, s3 = R.conv2d(d3["x"], d3["w"], m, d3["bias"], relu=True)
+    assert_within(zb.numpy("loaded 3x3"), ref3, s3, what="loaded 3x3 pattern layer")
+    p3.free(); q3.free()
+
+
 def test_wide_layer_through_the_nhwc_entry_point():
     """Config 5's layer shape at a reduced batch: the NHWC entry point routes it through the channel-major kernel."""
     for g, sp in ((4, 50), (8, 70)):
