@@ -114,6 +114,8 @@ def main(argv=None):
     ap.add_argument("--cm-tile", default=None, help="P,GPW,NW,KC: transpose + channel-major kernel with this tile")
     ap.add_argument("--bf16", action="store_true", help="time the bf16 tensor-core mode instead of the fp32 kernel")
     ap.add_argument("--only", default=None)
+    ap.add_argument("--layer", default=None, help="N,H,W,Cin,Cout,G,sparsity_pct: time that 1x1 layer as the MobileNet chain "
+                                                  "runs it (channel-major in and out, tile shape chosen by the library)")
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--batch5", type=int, default=256)
@@ -121,6 +123,23 @@ def main(argv=None):
     tile = tuple(int(t) for t in args.tile.split(",")) if args.tile else None
     cm_tile = tuple(int(t) for t in args.cm_tile.split(",")) if args.cm_tile else None
     flush = torch.zeros(64 * 1024 * 1024, device="cuda")
+    if args.layer:
+        n, h, w, cin, cout, g, sp = (int(v) for v in args.layer.split(","))
+        d = WL.single_conv_inputs(1, 1, 64, cin, cout, 1, g, sp, 0, 0.05, 0.05)     # the weights; activations are random
+        p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], g)
+        m = n * h * w
+        ld = (m + 3) // 4 * 4
+        xt, yt = torch.rand((cin, ld), device="cuda"), torch.empty((cout, ld), device="cuda")
+        f = lambda: sbnn.conv1x1_gs_cm(p, xt, ld, yt, ld, m, sbnn.SBNN_RELU | sbnn.SBNN_OUT_CM, cm_tile or (0, 0, 0, 0))  # noqa: E731
+        med, mn = _time(torch, f, args.reps, flush)
+        sbnn.get_async_status()
+        units = int(d["unit_mask"].sum())
+        flops, byts = 2.0 * m * g * units, 4.0 * (m * (cin + cout) + units * (1 + g) + cout + cout // g + 1)
+        roof = max(flops / FP32_PEAK, byts / _hbm())
+        print(json.dumps({"case": f"layer {args.layer}", "M": m, "us": med * 1e6, "us_min": mn * 1e6, "roofline_us": roof * 1e6,
+                          "frac": roof / med, "tile": cm_tile}), flush=True)
+        p.free()
+        return
     cases = [("config1", lambda: WL.config1(), 1)]
     for g in (4, 8):
         for sp in (0, 30, 50, 70, 90):
