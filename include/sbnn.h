@@ -262,6 +262,22 @@ SBNN_API sbnn_status sbnn_dwconv3x3_cm(const float* w_dev, const float* b_dev, c
                                        int ldy, int N, int H, int W, int C, int stride, int flags, void* cuda_stream);
 
 /*
+ * Depthwise 3x3 (stride 1, pad 1, dense) followed by a group-sparse 1x1 convolution, as one kernel: the two principal
+ * layers of the network (Section 3.2), which follow each other in every block, without the depthwise output ever being
+ * written to memory.  Channel-major tensors as in sbnn_dwconv3x3_cm / sbnn_conv1x1_gs_cm:
+ *   xt_dev [Cin][ldx] input of the depthwise layer, yt_dev [Cout][ldy] output of the pointwise layer (always channel-major),
+ *   dw_w_dev [3][3][Cin], dw_b_dev [Cin] or NULL, pw a packed 1x1 layer with pw->Cin = Cin,
+ *   dw_flags / pw_flags: SBNN_RELU or 0 for the activation after each of the two layers.
+ * Result: what sbnn_dwconv3x3_cm followed by sbnn_conv1x1_gs_cm gives, up to the order of the fp32 sums (the depthwise
+ * result is rounded to fp32 once, as when it is stored).  Takes G = 4 layers and image widths that are multiples of 4
+ * up to 124; other shapes return SBNN_ERR_UNSUPPORTED (run the two layers one after the other then).  The first call
+ * of a layer builds a private re-layout of its weights (allocates and copies synchronously).
+ */
+SBNN_API sbnn_status sbnn_dwconv3x3_conv1x1_gs_cm(const sbnn_packed* pw, const float* dw_w_dev, const float* dw_b_dev,
+                                                  const float* xt_dev, int ldx, float* yt_dev, int ldy, int N, int H, int W,
+                                                  int dw_flags, int pw_flags, void* cuda_stream);
+
+/*
  * Depthwise 3x3 with 3:9 kernel patterns (Section 3.2, DwConv3x3; Algorithm 2): in every row of a kernel the
  * middle weight stays and either the first or the third column is pruned, one pattern per block of go
  * consecutive channels (the paper's PatternInfo; go = 16, or 8 or 4 for channel counts that need it).

@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     conv3x3_gs,
     dwconv3x3,
     dwconv3x3_cm,
+    dwconv3x3_conv1x1_gs_cm,
     dwconv3x3_pattern,
     get_async_status,
     head_noalloc,

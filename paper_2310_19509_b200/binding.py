@@ -53,6 +53,7 @@ def lib():
         "sbnn_to_channel_major": [P, P, I, I, I, P],
         "sbnn_dwconv3x3": [P, P, P, P, I, I, I, I, I, I, P],
         "sbnn_dwconv3x3_cm": [P, P, P, I, P, I, I, I, I, I, I, I, P],
+        "sbnn_dwconv3x3_conv1x1_gs_cm": [P, P, P, P, I, P, I, I, I, I, I, I, P],
         "sbnn_pack_dw_pattern": [P, P, I, I, P, P],
         "sbnn_dwconv3x3_pattern": [P, P, I, P, P, P, I, I, I, I, I, I, P],
         "sbnn_conv3x3_dense": [P, P, P, P, I, I, I, I, I, I, I, P],
@@ -207,6 +208,12 @@ def dwconv3x3(w, b, x, y, n, h, wd, c, stride, flags=SBNN_RELU, stream=None):
 
 def dwconv3x3_cm(w, b, xt, ldx, yt, ldy, n, h, wd, c, stride, flags=SBNN_RELU, stream=None):
     _check(lib().sbnn_dwconv3x3_cm(_ptr(w), _ptr(b), _ptr(xt), ldx, _ptr(yt), ldy, n, h, wd, c, stride, flags, _stream(stream)))
+
+
+def dwconv3x3_conv1x1_gs_cm(pw: Packed, dw_w, dw_b, xt, ldx, yt, ldy, n, h, wd, dw_flags=SBNN_RELU, pw_flags=SBNN_RELU, stream=None):
+    """Depthwise 3x3 (stride 1) + group-sparse 1x1 as one kernel on channel-major tensors."""
+    _check(lib().sbnn_dwconv3x3_conv1x1_gs_cm(pw.handle, _ptr(dw_w), _ptr(dw_b), _ptr(xt), ldx, _ptr(yt), ldy, n, h, wd,
+                                              dw_flags, pw_flags, _stream(stream)))
 
 
 def pack_dw_pattern(w, mask, go):

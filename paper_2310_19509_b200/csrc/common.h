@@ -137,6 +137,10 @@ sbnn_status prepare_cm(const sbnn_packed* p, int P, int GPW, int NW, int KC);   
 void free_streams_cm(sbnn_packed* p);
 // Runs the NHWC call through the channel-major kernel if the shape profits; *done tells whether it did.
 sbnn_status conv1x1_via_cm(const sbnn_packed* w, const float* x, float* y, int M, int relu, cudaStream_t st, bool* done);
+// Depthwise 3x3 (stride 1) + group-sparse 1x1 in one kernel on channel-major tensors; *done = false (and SBNN_OK) when the
+// shape is outside what the fused kernel takes (G = 4, W a multiple of 4, W <= 124).
+sbnn_status dwconv3x3_conv1x1_fused_cm(const sbnn_packed* pw, const float* dw_w, const float* dw_b, const float* x, int ldx, float* y,
+                                       int ldy, int N, int H, int W, int relu_dw, int relu, cudaStream_t st, bool* done);
 sbnn_status read_async_status(int* value);
 // Device address of the status word that bounded waits report into (per device).
 sbnn_status async_status_word(int** out);

@@ -228,72 +228,17 @@ __device__ __forceinline__ void run_list_v(uint32_t r, int n, uint32_t xs, f32x2
     }
 }
 
+// The compute warps of the pipelined kernels: wait for a stage ("full": activations [KC][TM] at xs0, weight block at
+// ws0), run the warp's lists out of it, release it ("empty"), and write the tile's outputs.  Shared by the plain
+// kernel (stages filled by the copy engine) and the fused depthwise + pointwise kernel (activations written by the
+// CTA's own depthwise warps).
 template <class C, bool OUT_CM>
-__global__ void __launch_bounds__(C::NT, 1)
-conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ Y, int ldy,
-                  const float* __restrict__ bias, const uint4* __restrict__ rec,
-                  const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout, int ngroups, int nchunks,
-                  int ntiles, int total_tiles, int relu, int* status) {
-    constexpr int G = C::G, P = C::P, GPW = C::GPW, NW = C::NW, KC = C::KC, S = C::STAGES;
-    extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* xs0 = smem;
-    unsigned char* ws0 = smem + (size_t)S * C::XS_BYTES;
-    uint64_t* full = reinterpret_cast<uint64_t*>(ws0 + (size_t)S * C::WS_BYTES);
-    uint64_t* empty = full + S;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + S);
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // Persistent CTAs: CTA b works on tiles b, b + gridDim.x, ...  A tile index t = ptile * ntiles + gtile
-    // keeps the group tiles of one pixel tile adjacent, so they run at about the same time and the pixel
-    // tile's activations come from DRAM once and from L2 afterwards.  Stage and phase counters run on
-    // across tiles: the producer is already filling stages for the next tile while the compute warps
-    // finish the current one and write its outputs.
-
-    if (tid == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(full + s, 1);
-            mbar_init(empty + s, NW);
-        }
-        *abort_flag = 0;
-        mbar_fence_init();
-    }
-    __syncthreads();
-
-    if (warp == NW) {
-        // ---------------- producer warp ----------------
-        int issued = 0;
-        bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const int tile = t % ntiles, m0 = (t / ntiles) * C::TM;
-            const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
-            for (int k = 0; k < nchunks; ++k, ++issued) {
-                const int s = issued % S;
-                if (issued >= S) ok = mbar_wait(empty + s, ((issued / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
-                if (!ok) break;
-                if (lane == 0) {
-                    // a linear copy brings the step's weight block, one tiled copy the step's KC x TM box of X
-                    // (pixels past M and channels past Cin arrive as zeros and count towards the bytes).  The
-                    // weights do not depend on the previous kernel of the stream, the activations do: the very
-                    // first box is requested only once that kernel has finished.
-                    const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
-                    mbar_arrive_expect_tx(full + s, (uint32_t)C::XS_BYTES + (uint32_t)wn * 16u);
-                    bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, full + s);
-                    if (issued == 0) grid_dependency_wait();
-                    tensor_g2s_2d(xs0 + (size_t)s * C::XS_BYTES, &xmap, m0, k * KC, full + s);
-                }
-            }
-        }
-        if (!ok) {
-            // gave up: let the copies already issued land before the CTA's shared memory is released
-            for (int k = max(0, issued - S); k < issued; ++k) {
-                bool landed = false;
-                for (uint32_t i = 0; i < kWaitLimit && !landed; ++i) landed = mbar_try_wait(full + k % S, (k / S) & 1);
-            }
-        }
-        return;
-    }
-
-    // ---------------- compute warps ----------------
+__device__ __forceinline__ void compute_warps(unsigned char* xs0, unsigned char* ws0, uint64_t* full, uint64_t* empty,
+                                              volatile int* abort_flag, float* __restrict__ Y, int ldy,
+                                              const float* __restrict__ bias, int M, int ngroups, int nchunks, int ntiles,
+                                              int total_tiles, int relu, int* status) {
+    constexpr int G = C::G, P = C::P, GPW = C::GPW, S = C::STAGES;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     grid_dependency_wait();       // Y may still be read by the previous kernel of the stream
     grid_dependency_release();
     const unsigned lane_off = lane * 16;
@@ -416,6 +361,232 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
         }
     }
     }   // tiles
+}
+
+template <class C, bool OUT_CM>
+__global__ void __launch_bounds__(C::NT, 1)
+conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ Y, int ldy,
+                  const float* __restrict__ bias, const uint4* __restrict__ rec,
+                  const int32_t* __restrict__ blk_ptr, int M, int Cin, int Cout, int ngroups, int nchunks,
+                  int ntiles, int total_tiles, int relu, int* status) {
+    constexpr int G = C::G, P = C::P, GPW = C::GPW, NW = C::NW, KC = C::KC, S = C::STAGES;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* xs0 = smem;
+    unsigned char* ws0 = smem + (size_t)S * C::XS_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(ws0 + (size_t)S * C::WS_BYTES);
+    uint64_t* empty = full + S;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + S);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // Persistent CTAs: CTA b works on tiles b, b + gridDim.x, ...  A tile index t = ptile * ntiles + gtile
+    // keeps the group tiles of one pixel tile adjacent, so they run at about the same time and the pixel
+    // tile's activations come from DRAM once and from L2 afterwards.  Stage and phase counters run on
+    // across tiles: the producer is already filling stages for the next tile while the compute warps
+    // finish the current one and write its outputs.
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, NW);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == NW) {
+        // ---------------- producer warp ----------------
+        int issued = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const int tile = t % ntiles, m0 = (t / ntiles) * C::TM;
+            const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
+            for (int k = 0; k < nchunks; ++k, ++issued) {
+                const int s = issued % S;
+                if (issued >= S) ok = mbar_wait(empty + s, ((issued / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+                if (!ok) break;
+                if (lane == 0) {
+                    // a linear copy brings the step's weight block, one tiled copy the step's KC x TM box of X
+                    // (pixels past M and channels past Cin arrive as zeros and count towards the bytes).  The
+                    // weights do not depend on the previous kernel of the stream, the activations do: the very
+                    // first box is requested only once that kernel has finished.
+                    const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
+                    mbar_arrive_expect_tx(full + s, (uint32_t)C::XS_BYTES + (uint32_t)wn * 16u);
+                    bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, full + s);
+                    if (issued == 0) grid_dependency_wait();
+                    tensor_g2s_2d(xs0 + (size_t)s * C::XS_BYTES, &xmap, m0, k * KC, full + s);
+                }
+            }
+        }
+        if (!ok) {
+            // gave up: let the copies already issued land before the CTA's shared memory is released
+            for (int k = max(0, issued - S); k < issued; ++k) {
+                bool landed = false;
+                for (uint32_t i = 0; i < kWaitLimit && !landed; ++i) landed = mbar_try_wait(full + k % S, (k / S) & 1);
+            }
+        }
+        return;
+    }
+
+    // ---------------- compute warps ----------------
+    compute_warps<C, OUT_CM>(xs0, ws0, full, empty, abort_flag, Y, ldy, bias, M, ngroups, nchunks, ntiles, total_tiles, relu, status);
+}
+
+// ---- depthwise 3x3 (stride 1, pad 1) fused into the pointwise kernel -----------------------------------------
+// Y = pw( act( dw(X) ) ) without the depthwise output ever going to global memory (Section 3.2 names Conv1x1 and
+// DwConv3x3 as the two principal layers; one follows the other in every block of the network).  The CTA is the
+// pipelined kernel above plus NDW depthwise warps between the copy engine and the compute warps:
+//   * the producer warp copies, per channel step, the RAW input the step's 256 output pixels need: the pixels of a
+//     channel are contiguous, so the 3x3 neighbourhood of the run [m0, m0 + TM) lies in the run [m0 - W - 4,
+//     m0 + TM + W + 4) of the same plane, fetched as two boxes of KC x bw pixels (a box is at most 256 wide), zeros
+//     outside the tensor;
+//   * depthwise warp d computes channels d, d + NDW, ... of the step: a lane owns the same 2 x 4 pixels as a compute
+//     lane (aligned 16-byte loads of the three rows, the pixels left and right of its four from the neighbouring
+//     lanes by shuffle), masks the taps that fall outside the image (a run of four never straddles an image row,
+//     because W is a multiple of 4), adds the bias, applies the ReLU and writes the [KC][TM] activation stage that the
+//     compute warps read; the step's weight block still arrives by bulk copy on the same "full" barrier.
+// Barriers: raw_full / raw_empty between the copy engine and the depthwise warps, x_full (depthwise warps + weight
+// bytes) / x_empty between those and the compute warps; all waits bounded as above.
+constexpr int NDW = 3;
+
+template <class C>
+__global__ void __launch_bounds__(C::NT + NDW * 32, 1)
+dwpw_fused_kernel(const __grid_constant__ CUtensorMap rawmap, float* __restrict__ Y, int ldy, const float* __restrict__ bias,
+                  const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, const float* __restrict__ dw_w,
+                  const float* __restrict__ dw_b, int M, int Cin, int ngroups, int nchunks, int ntiles, int total_tiles,
+                  int H, int W, int bw, int relu_dw, int relu, int* status) {
+    constexpr int NW = C::NW, KC = C::KC, S = C::STAGES, RS = 2;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* xs0 = smem;
+    unsigned char* ws0 = smem + (size_t)S * C::XS_BYTES;
+    unsigned char* raw0 = ws0 + (size_t)S * C::WS_BYTES;
+    const uint32_t box_bytes = (uint32_t)KC * bw * 4u, raw_bytes = 2u * box_bytes;
+    uint64_t* x_full = reinterpret_cast<uint64_t*>(raw0 + (size_t)RS * raw_bytes);
+    uint64_t* x_empty = x_full + S;
+    uint64_t* raw_full = x_empty + S;
+    uint64_t* raw_empty = raw_full + RS;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(raw_empty + RS);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(x_full + s, 1 + NDW);
+            mbar_init(x_empty + s, NW);
+        }
+        for (int r = 0; r < RS; ++r) {
+            mbar_init(raw_full + r, 1);
+            mbar_init(raw_empty + r, NDW);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == NW) {
+        // ---------------- producer warp ----------------
+        int n = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const int tile = t % ntiles, m0 = (t / ntiles) * C::TM;
+            const int32_t* bp = blk_ptr + (size_t)tile * (nchunks + 1);
+            for (int k = 0; k < nchunks; ++k, ++n) {
+                const int r = n % RS, s = n % S;
+                if (n >= RS) ok = mbar_wait(raw_empty + r, ((n / RS) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+                if (!ok) break;
+                if (lane == 0) {
+                    unsigned char* dst = raw0 + (size_t)r * raw_bytes;
+                    mbar_arrive_expect_tx(raw_full + r, raw_bytes);
+                    if (n == 0) grid_dependency_wait();          // X comes from the previous kernel of the stream
+                    tensor_g2s_2d(dst, &rawmap, m0 - W - 4, k * KC, raw_full + r);
+                    tensor_g2s_2d(dst + box_bytes, &rawmap, m0 - W - 4 + bw, k * KC, raw_full + r);
+                }
+                if (n >= S) ok = mbar_wait(x_empty + s, ((n / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+                if (!ok) { ++n; break; }                         // the raw copies of this step are in flight
+                if (lane == 0) {
+                    const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
+                    mbar_arrive_expect_tx(x_full + s, (uint32_t)wn * 16u);
+                    bulk_g2s(ws0 + (size_t)s * C::WS_BYTES, rec + wbeg, (uint32_t)wn * 16u, x_full + s);
+                }
+            }
+        }
+        if (!ok) {   // gave up: let the raw copies already issued land before the CTA's shared memory is released
+            for (int k = max(0, n - RS); k < n; ++k) {
+                bool landed = false;
+                for (uint32_t i = 0; i < kWaitLimit && !landed; ++i) landed = mbar_try_wait(raw_full + k % RS, (k / RS) & 1);
+            }
+        }
+        return;
+    }
+
+    if (warp > NW) {
+        // ---------------- depthwise warps ----------------
+        const int d = warp - NW - 1;
+        int n = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            const int m0 = (t / ntiles) * C::TM;
+            // the lane's two runs of four pixels: position in the image decides which taps exist
+            int j0[2];
+            bool lz[2], rz[2], up[2], dn[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int p0 = i * 128 + 4 * lane, m = m0 + p0;
+                const int x = m % W, y = (m / W) % H;
+                j0[i] = p0 + W + 4;                               // index of the run's first pixel inside the raw rows
+                lz[i] = x == 0; rz[i] = x == W - 4; up[i] = y > 0; dn[i] = y < H - 1;
+            }
+            for (int k = 0; k < nchunks; ++k, ++n) {
+                const int r = n % RS, s = n % S;
+                if (!mbar_wait(raw_full + r, (n / RS) & 1, abort_flag, status, SBNN_ERR_TIMEOUT)) return;
+                if (n >= S && !mbar_wait(x_empty + s, ((n / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT)) return;
+                const float* raw = reinterpret_cast<const float*>(raw0 + (size_t)r * raw_bytes);
+                float* xst = reinterpret_cast<float*>(xs0 + (size_t)s * C::XS_BYTES);
+                // element j of channel row cl: first box holds j < bw, second the rest (bw is a multiple of 4)
+                auto at = [&](int cl, int j) -> const float* {
+                    return j < bw ? raw + cl * bw + j : raw + (KC + cl) * bw + (j - bw);
+                };
+                for (int cl = d; cl < KC; cl += NDW) {
+                    const int c = k * KC + cl;
+                    if (c >= Cin) break;                          // rows past Cin are referenced by no list
+                    float wk[9];
+#pragma unroll
+                    for (int q = 0; q < 9; ++q) wk[q] = __ldg(dw_w + q * Cin + c);
+                    const float b = dw_b ? __ldg(dw_b + c) : 0.0f;
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        float acc[4] = {b, b, b, b};
+#pragma unroll
+                        for (int kh = 0; kh < 3; ++kh) {
+                            const int jj = j0[i] + (kh - 1) * W;
+                            const bool rowok = kh == 0 ? up[i] : (kh == 2 ? dn[i] : true);
+                            float4 A = *reinterpret_cast<const float4*>(at(cl, jj));
+                            float L = __shfl_up_sync(0xffffffffu, A.w, 1), R = __shfl_down_sync(0xffffffffu, A.x, 1);
+                            if (lane == 0) L = *at(cl, jj - 1);
+                            if (lane == 31) R = *at(cl, jj + 4);
+                            if (lz[i]) L = 0.0f;
+                            if (rz[i]) R = 0.0f;
+                            if (!rowok) { A = make_float4(0.f, 0.f, 0.f, 0.f); L = 0.0f; R = 0.0f; }
+                            const float in[6] = {L, A.x, A.y, A.z, A.w, R};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                acc[e] = fmaf(in[e + 2], wk[kh * 3 + 2], fmaf(in[e + 1], wk[kh * 3 + 1], fmaf(in[e], wk[kh * 3], acc[e])));
+                        }
+                        float4 o = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                        if (relu_dw) o = make_float4(fmaxf(o.x, 0.f), fmaxf(o.y, 0.f), fmaxf(o.z, 0.f), fmaxf(o.w, 0.f));
+                        *reinterpret_cast<float4*>(xst + cl * C::TM + i * 128 + 4 * lane) = o;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(x_full + s);                      // this warp's channels of the stage are written
+                    mbar_arrive(raw_empty + r);                   // and it is done with the raw rows
+                }
+            }
+        }
+        return;
+    }
+
+    // ---------------- compute warps ----------------
+    compute_warps<C, true>(xs0, ws0, x_full, x_empty, abort_flag, Y, ldy, bias, M, ngroups, nchunks, ntiles, total_tiles, relu, status);
 }
 
 // Diagnostic: one warp waits, with a short cap, on an mbarrier that nothing ever completes.  Exercises the
@@ -680,6 +851,38 @@ sbnn_status launch_cm(const sbnn_packed* p, const Stream1x1& s, const float* x, 
     return SBNN_OK;
 }
 
+// Fused depthwise + pointwise launch (G = 4 layers, union lists, 8 warps, 32-channel steps, two stages).
+using FusedCfg = K2<4, 8, 2, 8, 32, 2>;
+
+sbnn_status launch_dwpw(const sbnn_packed* p, const float* dw_w, const float* dw_b, const float* x, int ldx, float* y, int ldy,
+                        int N, int H, int W, int relu_dw, int relu, cudaStream_t st, bool* done) {
+    using C = FusedCfg;
+    *done = false;
+    const long long M = (long long)N * H * W;
+    // the raw rows of a step: TM + 2W + 5 pixels, rounded up to two boxes of bw (a multiple of 4, at most 256)
+    const int bw = ((C::TM + 2 * W + 5 + 1) / 2 + 3) / 4 * 4;
+    const size_t smem = (size_t)C::STAGES * (C::XS_BYTES + C::WS_BYTES) + (size_t)2 * 2 * C::KC * bw * 4 + 128;
+    if (p->G != 4 || W % 4 || bw > 256 || smem > 227 * 1024 || M > 0x7fffffffLL - 1024) return SBNN_OK;
+    const TileCfg cfg{C::P, C::GPW, C::NW, C::KC};
+    Stream1x1 s;
+    sbnn_status r = get_stream_cm(p, cfg, &s);
+    if (r != SBNN_OK) return r;
+    if ((r = set_max_dyn_smem(reinterpret_cast<const void*>(&dwpw_fused_kernel<C>), 227 * 1024)) != SBNN_OK) return r;
+    if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
+    int* status = nullptr;
+    if ((r = status_word(&status)) != SBNN_OK) return r;
+    *done = true;
+    if (prepare_only()) return SBNN_OK;
+    const long long nblk = ((M + C::TM - 1) / C::TM) * s.ntiles;
+    if (nblk > 0x7fffffffLL) return fail(SBNN_ERR_SHAPE, "too many tiles");
+    CUtensorMap rawmap;
+    if ((r = encode_x_map(x, ldx, (int)M, p->Cin, bw, C::KC, &rawmap)) != SBNN_OK) return r;
+    dim3 grid((unsigned)std::min<long long>(nblk, sm_count()));
+    SBNN_CUDA_TRY(launch_kernel(dwpw_fused_kernel<C>, grid, C::NT + NDW * 32, smem, st, rawmap, y, ldy, p->d_bias, s.rec, s.blk_ptr, dw_w,
+                                dw_b, (int)M, p->Cin, p->ngroups, s.nchunks, s.ntiles, (int)nblk, H, W, bw, relu_dw, relu, status));
+    return SBNN_OK;
+}
+
 // Instantiated shapes: (G, P, GPW, NW, KC, STAGES).
 #define SBNN_K2_CONFIGS(X) \
     X(1, 8, 4, 8, 32, 4)   \
@@ -820,6 +1023,11 @@ sbnn_status scratch_workspace(size_t bytes, cudaStream_t st, float** out) { retu
 
 sbnn_status async_status_word(int** out) { return status_word(out); }
 
+sbnn_status dwconv3x3_conv1x1_fused_cm(const sbnn_packed* pw, const float* dw_w, const float* dw_b, const float* x, int ldx, float* y,
+                                       int ldy, int N, int H, int W, int relu_dw, int relu, cudaStream_t st, bool* done) {
+    return launch_dwpw(pw, dw_w, dw_b, x, ldx, y, ldy, N, H, W, relu_dw, relu, st, done);
+}
+
 sbnn_status encode_tiled_map(void* out, const void* base, int elem_bytes, int rank, const unsigned long long* dims,
                              const unsigned long long* strides_bytes, const unsigned* box, bool swizzle128) {
     if (swizzle128 && (size_t)box[0] * elem_bytes > 128) return fail(SBNN_ERR_SHAPE, "a swizzled box row is at most 128 bytes");
@@ -937,4 +1145,28 @@ extern "C" sbnn_status sbnn_conv1x1_gs_cm(const sbnn_packed* w, const float* xt_
         return conv1x1_small(w, xt_dev, ldx, y_dev, ldy, M, flags & SBNN_RELU, out_cm, static_cast<cudaStream_t>(cuda_stream));
     const TileCfg c = (P | GPW | NW | KC) ? TileCfg{P, GPW, NW, KC} : default_cfg_cm(w, M);
     return dispatch_cm(w, c, xt_dev, ldx, y_dev, ldy, M, flags & SBNN_RELU, out_cm, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" sbnn_status sbnn_dwconv3x3_conv1x1_gs_cm(const sbnn_packed* pw, const float* dw_w_dev, const float* dw_b_dev,
+                                                    const float* xt_dev, int ldx, float* yt_dev, int ldy, int N, int H, int W,
+                                                    int dw_flags, int pw_flags, void* cuda_stream) {
+    clear_error();
+    if (!pw || !dw_w_dev || !xt_dev || !yt_dev) return fail(SBNN_ERR_NULL, "pw, dw_w_dev, xt_dev and yt_dev must not be NULL");
+    if (pw->KH != 1 || pw->KW != 1) return fail(SBNN_ERR_SHAPE, "packed layer is %dx%d, expected 1x1", pw->KH, pw->KW);
+    if ((dw_flags & ~SBNN_RELU) || (pw_flags & ~SBNN_RELU)) return fail(SBNN_ERR_UNSUPPORTED, "only SBNN_RELU is accepted here");
+    if (N < 0 || H < 0 || W < 0) return fail(SBNN_ERR_SHAPE, "negative shape %dx%dx%d", N, H, W);
+    const long long M = (long long)N * H * W;
+    if (M > 0x7fffffffLL / 2) return fail(SBNN_ERR_SHAPE, "N*H*W too large");
+    if (ldx < M || ldy < M || ldx % 4 || ldy % 4) return fail(SBNN_ERR_SHAPE, "ldx=%d / ldy=%d must cover the %lld pixels and be multiples of 4", ldx, ldy, M);
+    if (!aligned16(xt_dev) || !aligned16(yt_dev)) return fail(SBNN_ERR_ALIGN, "xt_dev and yt_dev must be 16-byte aligned");
+    if (M == 0) return SBNN_OK;
+    sbnn_status st = check_packed_device(pw);
+    if (st != SBNN_OK) return st;
+    if ((st = check_device()) != SBNN_OK) return st;
+    bool done = false;
+    st = launch_dwpw(pw, dw_w_dev, dw_b_dev, xt_dev, ldx, yt_dev, ldy, N, H, W, dw_flags & SBNN_RELU, pw_flags & SBNN_RELU,
+                     static_cast<cudaStream_t>(cuda_stream), &done);
+    if (st != SBNN_OK) return st;
+    if (!done) return fail(SBNN_ERR_UNSUPPORTED, "the fused kernel takes G = 4 layers and image widths that are multiples of 4 up to 124");
+    return SBNN_OK;
 }

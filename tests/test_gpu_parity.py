@@ -170,6 +170,70 @@ def test_depthwise_channel_major_variants(stride, hw, n, c):
     assert bool(torch.isnan(yt[:, n * ho * wo:]).all())          # nothing written past the last pixel
 
 
+@pytest.mark.parametrize("n,h,w,cin,cout,relu_dw", [(3, 20, 28, 32, 64, True), (2, 9, 112, 32, 64, True), (5, 8, 12, 72, 40, False),
+                                                    (1, 56, 56, 128, 128, True), (2, 3, 4, 8, 8, True)])
+def test_fused_depthwise_pointwise(n, h, w, cin, cout, relu_dw):
+    """sbnn_dwconv3x3_conv1x1_gs_cm: depthwise 3x3 (stride 1) and group-sparse 1x1 in one kernel.  Several images (runs of
+    256 pixels cross image borders, so every padding mask is exercised), the widest supported map, a ragged last pixel
+    tile, several channel steps and group tiles, a channel count that is not a multiple of the step.  Oracle: depthwise
+    in fp64, rounded to fp32 as a stored activation would be, then the masked dense 1x1; the bound adds what the
+    depthwise layer's own tolerance and that rounding can contribute through |W~|."""
+    rng = np.random.default_rng(51)
+    x = rng.random((n, h, w, cin), dtype=np.float32)
+    dw_w = (rng.standard_normal((3, 3, cin)) * 0.4).astype(np.float32)
+    dw_b = (rng.standard_normal(cin) * 0.1).astype(np.float32)
+    d = WL.single_conv_inputs(1, 1, 4, cin, cout, 1, 4, 50, seed=52, mask_mode="layer_global")
+    m = n * h * w
+    ldx, ldy = (m + 3) // 4 * 4 + 4, (m + 3) // 4 * 4
+    xt = torch.full((cin, ldx), float("nan"), device="cuda")
+    xt[:, :m] = dev(x).reshape(m, cin).t()
+    out = Guarded((cout, ldy))
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    sbnn.dwconv3x3_conv1x1_gs_cm(p, dev(dw_w), dev(dw_b), xt, ldx, out.t, ldy, n, h, w,
+                                 sbnn.SBNN_RELU if relu_dw else 0, sbnn.SBNN_RELU)
+    sbnn.get_async_status()
+    full = out.numpy("fused")
+    assert np.all(np.isnan(full[:, m:]))
+    y = full[:, :m].T.reshape(n, h, w, cout).astype(np.float64)
+    mid, s_dw = R.dwconv3x3(x, dw_w, dw_b, stride=1, relu=relu_dw)
+    mid32 = mid.astype(np.float32)
+    ref, s_pw = R.conv2d(mid32, d["w"], d["mask"], d["bias"], relu=True)
+    e_mid = (1e-5 * s_dw + np.abs(mid) * 2.0 ** -23).astype(np.float32)          # depthwise tolerance + one fp32 rounding
+    prop, _ = R.conv2d(e_mid, np.abs(d["w"]), d["mask"], None, relu=False)
+    bound = 1e-5 * s_pw + prop * (1 + 1e-6)
+    err = np.abs(y - ref)
+    assert np.all(np.isfinite(y))
+    assert np.all(err <= bound), f"worst ratio {np.max(err / np.maximum(bound, 1e-300))}"
+    # and the two-kernel route agrees within the same bound
+    yt2 = torch.full((cin, ldy), float("nan"), device="cuda")
+    sbnn.dwconv3x3_cm(dev(dw_w), dev(dw_b), xt, ldx, yt2, ldy, n, h, w, cin, 1, sbnn.SBNN_RELU if relu_dw else 0)
+    out2 = Guarded((cout, ldy))
+    sbnn.conv1x1_gs_cm(p, yt2, ldy, out2.t, ldy, m, sbnn.SBNN_RELU | sbnn.SBNN_OUT_CM)
+    sbnn.get_async_status()
+    y2 = out2.numpy("two kernels")[:, :m].T.reshape(n, h, w, cout).astype(np.float64)
+    assert np.all(np.abs(y2 - ref) <= bound)
+    p.free()
+
+
+def test_fused_depthwise_pointwise_refuses_what_it_does_not_take():
+    d = WL.single_conv_inputs(1, 1, 4, 16, 16, 1, 8, 50, seed=53)
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 8)
+    xt = torch.zeros((16, 64), device="cuda")
+    yt = torch.zeros((16, 64), device="cuda")
+    w9, b = torch.zeros((3, 3, 16), device="cuda"), torch.zeros(16, device="cuda")
+    with pytest.raises(sbnn.SbnnError) as e:
+        sbnn.dwconv3x3_conv1x1_gs_cm(p, w9, b, xt, 64, yt, 64, 1, 8, 8)           # G = 8
+    assert e.value.name == "SBNN_ERR_UNSUPPORTED"
+    p.free()
+    d = WL.single_conv_inputs(1, 1, 4, 16, 16, 1, 4, 50, seed=53)
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    with pytest.raises(sbnn.SbnnError) as e:
+        sbnn.dwconv3x3_conv1x1_gs_cm(p, w9, b, xt, 64, yt, 64, 1, 9, 7)           # width not a multiple of 4
+    assert e.value.name in ("SBNN_ERR_UNSUPPORTED", "SBNN_ERR_SHAPE")
+    sbnn.get_async_status()
+    p.free()
+
+
 @pytest.mark.parametrize("stride", [1, 2])
 @pytest.mark.parametrize("shape,go", [((2, 9, 11, 32), 16), ((1, 14, 14, 48), 8), ((1, 1, 1, 4), 4), ((3, 7, 7, 64), 16)])
 def test_depthwise_3of9_patterns(stride, shape, go):
