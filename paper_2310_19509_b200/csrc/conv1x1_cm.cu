@@ -447,7 +447,7 @@ conv1x1_cm_kernel(const __grid_constant__ CUtensorMap xmap, float* __restrict__ 
 //     compute warps read; the step's weight block still arrives by bulk copy on the same "full" barrier.
 // Barriers: raw_full / raw_empty between the copy engine and the depthwise warps, x_full (depthwise warps + weight
 // bytes) / x_empty between those and the compute warps; all waits bounded as above.
-constexpr int NDW = 3;
+constexpr int NDW = 7;
 
 template <class C>
 __global__ void __launch_bounds__(C::NT + NDW * 32, 1)
@@ -466,8 +466,10 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap rawmap, float* __restrict_
     uint64_t* raw_full = x_empty + S;
     uint64_t* raw_empty = raw_full + RS;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(raw_empty + RS);
+    float* dwsm = reinterpret_cast<float*>(raw_empty + RS) + 4;      // depthwise weights [9][Cin], then the bias [Cin]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < 10 * Cin; i += blockDim.x) dwsm[i] = i < 9 * Cin ? __ldg(dw_w + i) : (dw_b ? __ldg(dw_b + i - 9 * Cin) : 0.0f);
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(x_full + s, 1 + NDW);
@@ -525,14 +527,23 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap rawmap, float* __restrict_
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             const int m0 = (t / ntiles) * C::TM;
             // the lane's two runs of four pixels: position in the image decides which taps exist
-            int j0[2];
-            bool lz[2], rz[2], up[2], dn[2];
+            // offA[i][kh]: where the run's row kh starts inside a channel's raw data (element j of a channel row sits in
+            // the first box for j < bw, in the second otherwise; bw is a multiple of 4, so a run never straddles them);
+            // offL / offR: the pixel left and right of the run (only lanes 0 and 31 fetch those, the others shuffle)
+            int offA[2][3], offL[2][3], offR[2][3];
+            bool lz[2], rz[2], rowok[2][3];
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
                 const int p0 = i * 128 + 4 * lane, m = m0 + p0;
                 const int x = m % W, y = (m / W) % H;
-                j0[i] = p0 + W + 4;                               // index of the run's first pixel inside the raw rows
-                lz[i] = x == 0; rz[i] = x == W - 4; up[i] = y > 0; dn[i] = y < H - 1;
+                lz[i] = x == 0; rz[i] = x == W - 4;
+                rowok[i][0] = y > 0; rowok[i][1] = true; rowok[i][2] = y < H - 1;
+#pragma unroll
+                for (int kh = 0; kh < 3; ++kh) {
+                    const int jj = p0 + W + 4 + (kh - 1) * W;     // index of the run's first pixel inside the raw row
+                    auto off = [&](int j) { return j < bw ? j : KC * bw + j - bw; };
+                    offA[i][kh] = off(jj); offL[i][kh] = off(jj - 1); offR[i][kh] = off(jj + 4);
+                }
             }
             for (int k = 0; k < nchunks; ++k, ++n) {
                 const int r = n % RS, s = n % S;
@@ -540,32 +551,40 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap rawmap, float* __restrict_
                 if (n >= S && !mbar_wait(x_empty + s, ((n / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT)) return;
                 const float* raw = reinterpret_cast<const float*>(raw0 + (size_t)r * raw_bytes);
                 float* xst = reinterpret_cast<float*>(xs0 + (size_t)s * C::XS_BYTES);
-                // element j of channel row cl: first box holds j < bw, second the rest (bw is a multiple of 4)
-                auto at = [&](int cl, int j) -> const float* {
-                    return j < bw ? raw + cl * bw + j : raw + (KC + cl) * bw + (j - bw);
-                };
-                for (int cl = d; cl < KC; cl += NDW) {
-                    const int c = k * KC + cl;
-                    if (c >= Cin) break;                          // rows past Cin are referenced by no list
+                // this warp's channels of the step: d, d + NDW, ... below min(KC, Cin - k*KC); rows past Cin are referenced
+                // by no list.  All loads of a channel are issued before its first FMA, two channels are in flight.
+                const int nch = min(KC, Cin - k * KC);
+                const int mine = nch > d ? (nch - d + NDW - 1) / NDW : 0;
+#pragma unroll 2
+                for (int u = 0; u < mine; ++u) {
+                    const int cl = d + u * NDW, c = k * KC + cl;
+                    const float* rc = raw + cl * bw;
+                    float4 A[2][3];
+                    float Le[2][3], Re[2][3];
+#pragma unroll
+                    for (int i = 0; i < 2; ++i)
+#pragma unroll
+                        for (int kh = 0; kh < 3; ++kh) {
+                            const bool ok = rowok[i][kh];
+                            A[i][kh] = ok ? *reinterpret_cast<const float4*>(rc + offA[i][kh]) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            Le[i][kh] = (lane == 0 && ok && !lz[i]) ? rc[offL[i][kh]] : 0.0f;
+                            Re[i][kh] = (lane == 31 && ok && !rz[i]) ? rc[offR[i][kh]] : 0.0f;
+                        }
                     float wk[9];
 #pragma unroll
-                    for (int q = 0; q < 9; ++q) wk[q] = __ldg(dw_w + q * Cin + c);
-                    const float b = dw_b ? __ldg(dw_b + c) : 0.0f;
+                    for (int q = 0; q < 9; ++q) wk[q] = dwsm[q * Cin + c];
+                    const float b = dwsm[9 * Cin + c];
 #pragma unroll
                     for (int i = 0; i < 2; ++i) {
                         float acc[4] = {b, b, b, b};
 #pragma unroll
                         for (int kh = 0; kh < 3; ++kh) {
-                            const int jj = j0[i] + (kh - 1) * W;
-                            const bool rowok = kh == 0 ? up[i] : (kh == 2 ? dn[i] : true);
-                            float4 A = *reinterpret_cast<const float4*>(at(cl, jj));
-                            float L = __shfl_up_sync(0xffffffffu, A.w, 1), R = __shfl_down_sync(0xffffffffu, A.x, 1);
-                            if (lane == 0) L = *at(cl, jj - 1);
-                            if (lane == 31) R = *at(cl, jj + 4);
-                            if (lz[i]) L = 0.0f;
+                            float L = __shfl_up_sync(0xffffffffu, A[i][kh].w, 1), R = __shfl_down_sync(0xffffffffu, A[i][kh].x, 1);
+                            if (lane == 0) L = Le[i][kh];
+                            if (lane == 31) R = Re[i][kh];
+                            if (lz[i]) L = 0.0f;                  // (a row that does not exist was loaded as zeros)
                             if (rz[i]) R = 0.0f;
-                            if (!rowok) { A = make_float4(0.f, 0.f, 0.f, 0.f); L = 0.0f; R = 0.0f; }
-                            const float in[6] = {L, A.x, A.y, A.z, A.w, R};
+                            const float in[6] = {L, A[i][kh].x, A[i][kh].y, A[i][kh].z, A[i][kh].w, R};
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
                                 acc[e] = fmaf(in[e + 2], wk[kh * 3 + 2], fmaf(in[e + 1], wk[kh * 3 + 1], fmaf(in[e], wk[kh * 3], acc[e])));
@@ -861,7 +880,7 @@ sbnn_status launch_dwpw(const sbnn_packed* p, const float* dw_w, const float* dw
     const long long M = (long long)N * H * W;
     // the raw rows of a step: TM + 2W + 5 pixels, rounded up to two boxes of bw (a multiple of 4, at most 256)
     const int bw = ((C::TM + 2 * W + 5 + 1) / 2 + 3) / 4 * 4;
-    const size_t smem = (size_t)C::STAGES * (C::XS_BYTES + C::WS_BYTES) + (size_t)2 * 2 * C::KC * bw * 4 + 128;
+    const size_t smem = (size_t)C::STAGES * (C::XS_BYTES + C::WS_BYTES) + (size_t)2 * 2 * C::KC * bw * 4 + 128 + (size_t)10 * p->Cin * 4;
     if (p->G != 4 || W % 4 || bw > 256 || smem > 227 * 1024 || M > 0x7fffffffLL - 1024) return SBNN_OK;
     const TileCfg cfg{C::P, C::GPW, C::NW, C::KC};
     Stream1x1 s;
