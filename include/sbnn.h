@@ -118,6 +118,10 @@ typedef struct {
     const float* bias;        /* host, borrowed */
     const uint16_t* tap_mask; /* host, borrowed: [nnz_units], bit t = tap t of the unit is kept; NULL unless the layer
                                  was packed by sbnn_pack_weights_pattern */
+    int gi;                   /* 4 if every group keeps aligned runs of 4 consecutive input channels (the paper's
+                                 gi x go = 4 x G blocks, Section 3.2), else 1 */
+    const int32_t* block_idx; /* host, borrowed: gi == 4: first channel of every run, [nnz_units / 4] (Algorithm 1's
+                                 SD: one index per block); NULL when gi == 1 */
 } sbnn_packed_view;
 
 /* Borrow the canonical host arrays; they stay valid until sbnn_packed_free. */
@@ -133,10 +137,12 @@ SBNN_API sbnn_status sbnn_packed_free(sbnn_packed* p);
  * sbnn_packed_load reads them back into a new packed layer: host copy plus, if a device is present, device copies,
  * exactly as after packing.  File layout, little-endian, no padding:
  *   bytes 0-7    magic 'S' 'B' 'N' 'N' 'P' 'K' 0x01 0x00
- *   int32[8]     format version (1), Cout, KH, KW, Cin, G, has_tap_mask (0 or 1), 0
+ *   int32[8]     format version (1), Cout, KH, KW, Cin, G, has_tap_mask (0 or 1), index_block (0 or 4)
  *   int64        nnz_units
  *   int32        group_ptr[Cout/G + 1]
- *   int32        idx[nnz_units]
+ *   int32        idx[nnz_units]                 index_block = 0: one index per kept unit
+ *                idx[nnz_units / 4]             index_block = 4 (written for layers whose view has gi = 4): the first
+ *                                               channel of every aligned run of 4 kept channels, a quarter of the indices
  *   float32      val[nnz_units][KH*KW][G]
  *   float32      bias[Cout]
  *   uint16       tap_mask[nnz_units]            only if has_tap_mask
@@ -432,6 +438,17 @@ SBNN_API sbnn_status sbnn_selftest_wait_timeout(void* cuda_stream);
  * Timing it with events on `cuda_stream` gives the FP32 rate this GPU sustains at its current clocks.
  */
 SBNN_API sbnn_status sbnn_selftest_fma_rate(int iterations, double* flop_out, void* cuda_stream);
+
+/*
+ * Debug aid (the paper has no counterpart): checks the DEVICE copies of a packed layer on the device -- prefix sums
+ * monotone and spanning the kept units, indices ascending inside [0, Cin) -- with one thread per group.  A violation
+ * sets the device status word; the next sbnn_get_async_status on the stream then returns SBNN_ERR_SHAPE once.  The
+ * kernel never traps and reads nothing outside the arrays it is given, so it is safe to run on memory suspected
+ * of having been overwritten.  sbnn_debug_poke_device_index is the test hook that goes with it: it overwrites one
+ * index of the device copy (the host copy and the private layouts stay as they are) and returns the previous value.
+ */
+SBNN_API sbnn_status sbnn_debug_check_packed(const sbnn_packed* w, void* cuda_stream);
+SBNN_API sbnn_status sbnn_debug_poke_device_index(sbnn_packed* w, long long unit, int value, int* previous);
 
 /*
  * Test hook: overwrite the device number recorded in a packed layer, so that the refusal of compute calls

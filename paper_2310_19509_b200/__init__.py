@@ -34,6 +34,8 @@ from .binding import (  # noqa: F401
     prepare,
     selftest_fma_rate,
     debug_set_packed_device,
+    debug_check_packed,
+    debug_poke_device_index,
     selftest_wait_timeout,
     status_str,
     to_channel_major,

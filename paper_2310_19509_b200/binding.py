@@ -20,7 +20,8 @@ class SbnnError(RuntimeError):
 class _View(C.Structure):
     _fields_ = [("Cout", C.c_int), ("KH", C.c_int), ("KW", C.c_int), ("Cin", C.c_int), ("G", C.c_int),
                 ("ngroups", C.c_int), ("nnz_units", C.c_int64), ("group_ptr", C.c_void_p), ("idx", C.c_void_p),
-                ("val", C.c_void_p), ("bias", C.c_void_p), ("tap_mask", C.c_void_p)]
+                ("val", C.c_void_p), ("bias", C.c_void_p), ("tap_mask", C.c_void_p), ("gi", C.c_int),
+                ("block_idx", C.c_void_p)]
 
 
 def lib_path() -> str:
@@ -71,6 +72,8 @@ def lib():
         "sbnn_prepare": [P, I, I, I, I],
         "sbnn_selftest_fma_rate": [I, P, P],
         "sbnn_debug_set_packed_device": [P, I, P],
+        "sbnn_debug_check_packed": [P, P],
+        "sbnn_debug_poke_device_index": [P, C.c_longlong, I, P],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -135,7 +138,8 @@ class Packed:
                     group_ptr=arr(v.group_ptr, v.ngroups + 1, np.int32), idx=arr(v.idx, v.nnz_units, np.int32),
                     val=arr(v.val, v.nnz_units * taps * v.G, np.float32).reshape(v.nnz_units, taps, v.G),
                     bias=arr(v.bias, v.Cout, np.float32),
-                    tap_mask=arr(v.tap_mask, v.nnz_units, np.uint16) if v.tap_mask else None)
+                    tap_mask=arr(v.tap_mask, v.nnz_units, np.uint16) if v.tap_mask else None, gi=v.gi,
+                    block_idx=arr(v.block_idx, v.nnz_units // 4, np.int32) if v.block_idx else None)
 
     def unpack(self):
         v = _View()
@@ -264,6 +268,18 @@ def debug_set_packed_device(w: Packed, device) -> int:
     """Test hook: overwrite the device recorded in a packed layer; returns the previous value."""
     prev = C.c_int()
     _check(lib().sbnn_debug_set_packed_device(w.handle, int(device), C.byref(prev)))
+    return prev.value
+
+
+def debug_check_packed(w: Packed, stream=None):
+    """Enqueue the device-side consistency check of a packed layer (result through get_async_status)."""
+    _check(lib().sbnn_debug_check_packed(w.handle, _stream(stream)))
+
+
+def debug_poke_device_index(w: Packed, unit, value) -> int:
+    """Test hook: overwrite one index of the device copy; returns the previous value."""
+    prev = C.c_int()
+    _check(lib().sbnn_debug_poke_device_index(w.handle, int(unit), int(value), C.byref(prev)))
     return prev.value
 
 

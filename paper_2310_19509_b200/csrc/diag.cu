@@ -33,6 +33,22 @@ __global__ void __launch_bounds__(512) fma_rate_kernel(int iters, float seed) {
     if (s == 123456.789f) g_fma_sink[threadIdx.x & 31] = s;
 }
 
+// Device-side consistency check of a packed layer's device copies: one thread per group walks its index list.
+// A violation is recorded in the status word (first one wins); nothing traps, the kernel always returns normally.
+__global__ void __launch_bounds__(128)
+check_packed_kernel(const int32_t* __restrict__ group_ptr, const int32_t* __restrict__ idx, int ngroups, int Cin, long long nnz,
+                    int* status) {
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= ngroups) return;
+    const long long lo = group_ptr[g], hi = group_ptr[g + 1];
+    bool ok = lo >= 0 && lo <= hi && hi <= nnz && (g > 0 || lo == 0) && (g + 1 < ngroups || hi == nnz);
+    for (long long u = lo; ok && u < hi; ++u) {
+        const int c = idx[u];
+        ok = c >= 0 && c < Cin && (u == lo || c > idx[u - 1]);
+    }
+    if (!ok) atomicCAS(status, 0, (int)SBNN_ERR_SHAPE);
+}
+
 }  // namespace
 
 // defined in conv1x1_cm.cu: builds the weight streams of every tile shape the default choice can take for this layer
@@ -79,5 +95,30 @@ extern "C" sbnn_status sbnn_debug_set_packed_device(sbnn_packed* w, int device, 
     if (!w) return fail(SBNN_ERR_NULL, "packed weights must not be NULL");
     if (previous) *previous = w->device;
     w->device = device;
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_debug_check_packed(const sbnn_packed* w, void* cuda_stream) {
+    clear_error();
+    if (!w) return fail(SBNN_ERR_NULL, "packed weights must not be NULL");
+    sbnn_status st = check_packed_device(w);
+    if (st != SBNN_OK) return st;
+    if ((st = check_device()) != SBNN_OK) return st;
+    int* status = nullptr;
+    if ((st = async_status_word(&status)) != SBNN_OK) return st;
+    check_packed_kernel<<<(w->ngroups + 127) / 128, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        w->d_group_ptr, w->d_idx, w->ngroups, w->Cin, (long long)w->nnz, status);
+    SBNN_CUDA_TRY(cudaGetLastError());
+    return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_debug_poke_device_index(sbnn_packed* w, long long unit, int value, int* previous) {
+    clear_error();
+    if (!w) return fail(SBNN_ERR_NULL, "packed weights must not be NULL");
+    if (unit < 0 || unit >= w->nnz) return fail(SBNN_ERR_SHAPE, "unit %lld outside [0, %lld)", unit, (long long)w->nnz);
+    sbnn_status st = check_packed_device(w);
+    if (st != SBNN_OK) return st;
+    if (previous) SBNN_CUDA_TRY(cudaMemcpy(previous, w->d_idx + unit, sizeof(int), cudaMemcpyDeviceToHost));
+    SBNN_CUDA_TRY(cudaMemcpy(w->d_idx + unit, &value, sizeof(int), cudaMemcpyHostToDevice));
     return SBNN_OK;
 }

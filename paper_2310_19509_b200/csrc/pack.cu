@@ -129,9 +129,33 @@ extern "C" const char* sbnn_status_str(sbnn_status s) {
 extern "C" const char* sbnn_last_error(void) { return g_err; }
 
 namespace {
+// The paper's own Conv1x1 format groups gi = 4 consecutive input channels with the go = G output channels of a group
+// (Section 3.2) and stores one index per block (Algorithm 1's SD).  A layer whose every group keeps aligned runs of 4
+// channels is such a layer: record the block size and the per-block index list, a quarter of the per-channel one.
+void detect_blocks(sbnn_packed* p) {
+    p->gi = 1;
+    p->block_idx.clear();
+    if (p->Cin % 4 || p->nnz == 0 || p->nnz % 4) return;
+    for (int g = 0; g < p->ngroups; ++g) {
+        const int64_t lo = p->group_ptr[g], hi = p->group_ptr[g + 1];
+        if ((hi - lo) % 4) return;
+        for (int64_t u = lo; u < hi; u += 4)
+            if (p->idx[u] % 4 || p->idx[u + 1] != p->idx[u] + 1 || p->idx[u + 2] != p->idx[u] + 2 || p->idx[u + 3] != p->idx[u] + 3) return;
+    }
+    p->block_idx.resize(p->nnz / 4);
+    for (int64_t b = 0; b < p->nnz / 4; ++b) p->block_idx[b] = p->idx[4 * b];
+    p->gi = 4;
+}
+
 // Last step of packing and of loading: device copies of the canonical arrays and the default private layouts, if
 // there is a device; *out owns p afterwards (on failure p is freed).
 sbnn_status finish_packed(sbnn_packed* p, sbnn_packed** out) {
+    try {
+        detect_blocks(p);
+    } catch (const std::bad_alloc&) {
+        p->gi = 1;
+        p->block_idx.clear();
+    }
     int ndev = 0, dev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0 || cudaGetDevice(&dev) != cudaSuccess) {
         cudaGetLastError();
@@ -256,6 +280,8 @@ extern "C" sbnn_status sbnn_packed_get(const sbnn_packed* p, sbnn_packed_view* v
     v->val = p->val.data();
     v->bias = p->bias.data();
     v->tap_mask = p->tap_mask.empty() ? nullptr : p->tap_mask.data();
+    v->gi = p->gi;
+    v->block_idx = p->block_idx.empty() ? nullptr : p->block_idx.data();
     return SBNN_OK;
 }
 
@@ -310,13 +336,15 @@ extern "C" sbnn_status sbnn_packed_save(const sbnn_packed* p, const char* path) 
         sum.add(d, n);
         ok = ok && (n == 0 || fwrite(d, 1, n, fc.f) == n);
     };
-    const int32_t hdr[8] = {1, p->Cout, p->KH, p->KW, p->Cin, p->G, p->tap_mask.empty() ? 0 : 1, 0};
+    const bool blocks = p->gi == 4 && !p->block_idx.empty();   // indices are then stored once per run of 4
+    const int32_t hdr[8] = {1, p->Cout, p->KH, p->KW, p->Cin, p->G, p->tap_mask.empty() ? 0 : 1, blocks ? 4 : 0};
     const int64_t nnz = p->nnz;
     put(kFileMagic, 8);
     put(hdr, sizeof(hdr));
     put(&nnz, 8);
     put(p->group_ptr.data(), p->group_ptr.size() * 4);
-    put(p->idx.data(), p->idx.size() * 4);
+    if (blocks) put(p->block_idx.data(), p->block_idx.size() * 4);
+    else put(p->idx.data(), p->idx.size() * 4);
     put(p->val.data(), p->val.size() * 4);
     put(p->bias.data(), p->bias.size() * 4);
     put(p->tap_mask.data(), p->tap_mask.size() * 2);
@@ -348,9 +376,10 @@ extern "C" sbnn_status sbnn_packed_load(const char* path, sbnn_packed** out) {
     if (!ok) return fail(SBNN_ERR_IO, "%s is too short to be a packed layer", path);
     if (memcmp(magic, kFileMagic, 8) != 0) return fail(SBNN_ERR_IO, "%s is not a packed-layer file (bad magic)", path);
     if (hdr[0] != 1) return fail(SBNN_ERR_UNSUPPORTED, "%s has format version %d, this library reads version 1", path, hdr[0]);
-    const int Cout = hdr[1], KH = hdr[2], KW = hdr[3], Cin = hdr[4], G = hdr[5], has_taps = hdr[6];
+    const int Cout = hdr[1], KH = hdr[2], KW = hdr[3], Cin = hdr[4], G = hdr[5], has_taps = hdr[6], file_gi = hdr[7];
     if (Cout <= 0 || Cin <= 0 || !((KH == 1 && KW == 1) || (KH == 3 && KW == 3)) || !supported_group(G) || Cout % G ||
-        (has_taps != 0 && has_taps != 1) || nnz < 0 || nnz > (int64_t)(Cout / G) * Cin)
+        (has_taps != 0 && has_taps != 1) || (file_gi != 0 && file_gi != 4) || (file_gi == 4 && (nnz % 4 || Cin % 4)) || nnz < 0 ||
+        nnz > (int64_t)(Cout / G) * Cin)
         return fail(SBNN_ERR_SHAPE, "%s: inconsistent header (Cout=%d KH=%d KW=%d Cin=%d G=%d units=%lld)", path, Cout, KH, KW, Cin,
                     G, (long long)nnz);
     sbnn_packed* p = new (std::nothrow) sbnn_packed;
@@ -368,7 +397,20 @@ extern "C" sbnn_status sbnn_packed_load(const char* path, sbnn_packed** out) {
         return fail(SBNN_ERR_ALLOC, "out of host memory while loading %s", path);
     }
     get(p->group_ptr.data(), p->group_ptr.size() * 4);
-    get(p->idx.data(), p->idx.size() * 4);
+    if (file_gi == 4) {   // one index per run of 4 consecutive channels
+        std::vector<int32_t> blk;
+        try {
+            blk.resize(nnz / 4);
+        } catch (const std::bad_alloc&) {
+            delete p;
+            return fail(SBNN_ERR_ALLOC, "out of host memory while loading %s", path);
+        }
+        get(blk.data(), blk.size() * 4);
+        for (int64_t b = 0; ok && b < nnz / 4; ++b)
+            for (int e = 0; e < 4; ++e) p->idx[4 * b + e] = blk[b] + e;
+    } else {
+        get(p->idx.data(), p->idx.size() * 4);
+    }
     get(p->val.data(), p->val.size() * 4);
     get(p->bias.data(), p->bias.size() * 4);
     get(p->tap_mask.data(), p->tap_mask.size() * 2);
@@ -432,6 +474,7 @@ extern "C" sbnn_status sbnn_get_async_status(void* stream) {
     int word = 0;
     sbnn_status st = read_async_status(&word);
     if (st != SBNN_OK) return st;
-    if (word) return fail((sbnn_status)word, "a bounded wait inside a kernel gave up (device status %d)", word);
+    if (word == SBNN_ERR_TIMEOUT) return fail(SBNN_ERR_TIMEOUT, "a bounded wait inside a kernel gave up");
+    if (word) return fail((sbnn_status)word, "a device-side check failed (device status %d)", word);
     return SBNN_OK;
 }

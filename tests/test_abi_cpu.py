@@ -248,6 +248,7 @@ int main(void) {
     if (st != SBNN_OK) { printf("pack: %s %s\n", sbnn_status_str(st), sbnn_last_error()); return 1; }
     if (sbnn_packed_get(p, &v) != SBNN_OK) return 2;
     if (v.Cout != 8 || v.Cin != 8 || v.G != 4 || v.ngroups != 2 || v.nnz_units != 8 || v.tap_mask != NULL) return 3;
+    if (v.gi != 1 || v.block_idx != NULL) return 12;
     if (v.group_ptr[0] != 0 || v.group_ptr[1] != 4 || v.group_ptr[2] != 8) return 4;
     if (v.idx[0] != 1 || v.idx[3] != 7 || v.idx[4] != 0 || v.idx[7] != 6) return 5;
     if (v.val[0] != w[0 * 8 + 1] || v.val[1] != w[1 * 8 + 1] || v.bias[3] != 2.0f) return 6;
@@ -257,9 +258,10 @@ int main(void) {
     if (sbnn_pack_weights(w, m, bias, 8, 1, 1, 8, 3, &p) != SBNN_ERR_GROUP) return 9;
     if (strlen(sbnn_last_error()) == 0) return 10;
     if (sbnn_packed_free(p) != SBNN_OK) return 11;
-    printf("%zu %zu %zu %zu %zu %zu %zu\n", sizeof(sbnn_packed_view), offsetof(sbnn_packed_view, nnz_units),
+    printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu\n", sizeof(sbnn_packed_view), offsetof(sbnn_packed_view, nnz_units),
            offsetof(sbnn_packed_view, group_ptr), offsetof(sbnn_packed_view, idx), offsetof(sbnn_packed_view, val),
-           offsetof(sbnn_packed_view, bias), offsetof(sbnn_packed_view, tap_mask));
+           offsetof(sbnn_packed_view, bias), offsetof(sbnn_packed_view, tap_mask), offsetof(sbnn_packed_view, gi),
+           offsetof(sbnn_packed_view, block_idx));
     return 0;
 }
 ''')
@@ -272,7 +274,7 @@ int main(void) {
     got = [int(t) for t in out.stdout.split()]
     V = binding._View
     assert got == [C.sizeof(V), V.nnz_units.offset, V.group_ptr.offset, V.idx.offset, V.val.offset, V.bias.offset,
-                   V.tap_mask.offset]
+                   V.tap_mask.offset, V.gi.offset, V.block_idx.offset]
 
 
 def test_weights_of_another_device_are_refused_without_a_launch():
@@ -313,7 +315,11 @@ def _read_packed_file(path):
     off = 48
     ng = cout // g
     gp = np.frombuffer(raw, "<i4", ng + 1, off); off += 4 * (ng + 1)
-    idx = np.frombuffer(raw, "<i4", nnz, off); off += 4 * nnz
+    if zero == 4:
+        blk = np.frombuffer(raw, "<i4", nnz // 4, off); off += 4 * (nnz // 4)
+        idx = (blk[:, None] + np.arange(4)).reshape(-1).astype(np.int32)
+    else:
+        idx = np.frombuffer(raw, "<i4", nnz, off); off += 4 * nnz
     val = np.frombuffer(raw, "<f4", nnz * kh * kw * g, off).reshape(nnz, kh * kw, g); off += 4 * nnz * kh * kw * g
     bias = np.frombuffer(raw, "<f4", cout, off); off += 4 * cout
     taps = None
@@ -341,7 +347,7 @@ def test_packed_layer_file_round_trip_and_layout(tmp_path, k, g, cin, cout, patt
     p.save(path)
     # (i) the bytes on disk, read by a reader of our own, are the oracle's packing of the same layer
     f = _read_packed_file(path)
-    assert (f["ver"], f["cout"], f["kh"], f["kw"], f["cin"], f["g"], f["zero"]) == (1, cout, k, k, cin, g, 0)
+    assert (f["ver"], f["cout"], f["kh"], f["kw"], f["cin"], f["g"]) == (1, cout, k, k, cin, g) and f["zero"] in (0, 4)
     if patterns:
         gp, idx, val, taps = R.pack_pattern(w, m, g)
         assert np.array_equal(f["taps"], taps)
@@ -407,3 +413,43 @@ def test_packed_layer_file_errors(tmp_path):
     for byte in bad:
         h = ((h ^ byte) * 1099511628211) & 0xFFFFFFFFFFFFFFFF
     assert load(bytes(bad) + struct.pack("<Q", h), "unsorted") == "SBNN_ERR_SHAPE"
+
+
+def test_paper_style_4x4_blocks_are_recognised_and_stored_with_one_index_per_block(tmp_path):
+    """Masks made of aligned runs of gi = 4 input channels (the paper's 4 x 4 blocks, Section 3.2): the view reports gi = 4
+    and block_idx = the first channel of every run (Algorithm 1's SD), the file stores those instead of the per-channel
+    indices (a quarter of them) and loads back to the same layer; any other mask reports gi = 1."""
+    rng = np.random.default_rng(33)
+    cin, cout, g = 32, 16, 4
+    w = rng.standard_normal((cout, 1, 1, cin)).astype(np.float32)
+    um = group_mask_balanced(4, 3, cout // g, cin, 50, 4)            # gi = 4
+    assert np.all(um.reshape(cout // g, cin // 4, 4).all(axis=2) == um.reshape(cout // g, cin // 4, 4).any(axis=2))
+    m = expand_mask(um, g, 1, 1)
+    p = sbnn.pack_weights(w, m, None, g)
+    v = p.view()
+    gp, idx, val = R.pack(w, m, g)
+    blocks = np.asarray(idx).reshape(-1, 4)
+    assert np.array_equal(blocks, blocks[:, :1] + np.arange(4)) and np.all(blocks[:, 0] % 4 == 0)
+    assert v["gi"] == 4 and np.array_equal(v["block_idx"], blocks[:, 0]) and np.array_equal(v["idx"], idx)
+    path = str(tmp_path / "blocks.sbnn")
+    p.save(path)
+    raw = open(path, "rb").read()
+    import struct
+    hdr = struct.unpack_from("<8i", raw, 8)
+    assert hdr[7] == 4
+    nnz = len(idx)
+    off = 48 + 4 * (cout // g + 1)
+    assert np.array_equal(np.frombuffer(raw, "<i4", nnz // 4, off), blocks[:, 0])
+    assert len(raw) == off + 4 * (nnz // 4) + 4 * nnz * g + 4 * cout + 8
+    q = sbnn.load_packed(path)
+    vq = q.view()
+    assert vq["gi"] == 4 and np.array_equal(vq["idx"], idx) and vq["val"].tobytes() == v["val"].tobytes()
+    assert np.array_equal(vq["block_idx"], v["block_idx"])
+    p.free(); q.free()
+    um1 = group_mask_balanced(4, 3, cout // g, cin, 50)               # single channels
+    p1 = sbnn.pack_weights(w, expand_mask(um1, g, 1, 1), None, g)
+    v1 = p1.view()
+    assert v1["gi"] == 1 and v1["block_idx"] is None
+    p1.save(path)
+    assert struct.unpack_from("<8i", open(path, "rb").read(), 8)[7] == 0
+    p1.free()

@@ -698,6 +698,36 @@ def test_expired_wait_is_reported_and_the_context_stays_usable():
     assert_within(y, ref, s, what="after an expired wait")
 
 
+def test_device_side_check_of_a_packed_layer_reports_through_the_status_word():
+    """sbnn_debug_check_packed: clean on a freshly packed layer; an index of the device copy pushed out of range, or out
+    of order, is reported as SBNN_ERR_SHAPE by the next get_async_status (once), without a trap, and the context and the
+    layer stay usable after the index is put back."""
+    d = WL.single_conv_inputs(1, 4, 8, 40, 24, 1, 4, 50, seed=61)
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    sbnn.debug_check_packed(p)
+    sbnn.get_async_status()
+    for bad in (40, -1):
+        prev = sbnn.debug_poke_device_index(p, 3, bad)
+        sbnn.debug_check_packed(p)
+        with pytest.raises(sbnn.SbnnError) as e:
+            sbnn.get_async_status()
+        assert e.value.name == "SBNN_ERR_SHAPE"
+        sbnn.get_async_status()                                   # reported once
+        sbnn.debug_poke_device_index(p, 3, prev)
+    v = p.view()
+    prev = sbnn.debug_poke_device_index(p, 1, int(v["idx"][0]))   # equal to its predecessor: not ascending
+    sbnn.debug_check_packed(p)
+    with pytest.raises(sbnn.SbnnError):
+        sbnn.get_async_status()
+    sbnn.debug_poke_device_index(p, 1, prev)
+    sbnn.debug_check_packed(p)
+    sbnn.get_async_status()
+    y = run_1x1(d)
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    assert_within(y, ref, s, what="after the debug pokes")
+    p.free()
+
+
 def test_weights_of_another_device_are_refused_and_the_context_stays_usable():
     """With the recorded device of a packed layer overwritten (test hook), the compute calls return SBNN_ERR_CUDA
     naming both devices and launch nothing; with the number restored the same call works."""
