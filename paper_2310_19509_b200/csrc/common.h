@@ -121,6 +121,7 @@ struct sbnn_packed {
     mutable std::mutex mu;
     mutable std::map<sbnn::TileCfg, sbnn::Stream1x1> streams1x1;
     mutable std::map<sbnn::TileCfg, sbnn::Stream1x1> streams_cm;   // channel-major kernel, see conv1x1_cm.cu
+    mutable std::map<long long, sbnn::TileCfg> cfg_cm;             // tile shape chosen for a pixel count (the choice costs a loop over the tiles)
     mutable std::map<int, sbnn::Stream3x3> streams3x3;
     mutable void* bf16_stream = nullptr;  // see conv1x1_bf16.cu
     mutable void* umma_weights = nullptr; // dense bf16 copy of the masked weights, see conv1x1_umma.cu

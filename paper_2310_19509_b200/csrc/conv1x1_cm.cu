@@ -938,7 +938,21 @@ sbnn_status dispatch_cm(const sbnn_packed* p, const TileCfg& c, const float* x, 
 }
 
 // Tile shape for a layer run on M pixels.  M <= 0 stands for "many pixels" (the choice made before M is known).
+TileCfg choose_cfg_cm(const sbnn_packed* p, long long M);
+
+// The choice is made once per (layer, pixel count) and remembered: computing it walks the layer's tiles.
 TileCfg default_cfg_cm(const sbnn_packed* p, long long M) {
+    if (M <= 0) return choose_cfg_cm(p, M);
+    std::lock_guard<std::mutex> lk(p->mu);
+    auto it = p->cfg_cm.find(M);
+    if (it != p->cfg_cm.end()) return it->second;
+    if (p->cfg_cm.size() > 64) p->cfg_cm.clear();
+    const TileCfg c = choose_cfg_cm(p, M);
+    p->cfg_cm[M] = c;
+    return c;
+}
+
+TileCfg choose_cfg_cm(const sbnn_packed* p, long long M) {
     // Whole tiles are dealt to the persistent CTAs (CTA b takes tiles b, b + SMs, ...), and inside a CTA warp w runs
     // on scheduler w % 4, so a tile lasts as long as the scheduler with the most busy warps, and the launch as long as
     // the CTA with the most work.  The cost of a tile shape is that maximum, computed exactly from the layer's group
