@@ -336,6 +336,17 @@ def single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, reps):
         rec = {"case": name, "mode": mode, "G": g, "sparsity_pct": d["sparsity_pct"], "us": round(t * 1e6, 1),
                "tflops_nonzero": round(flops / t / 1e12, 2), "roofline_us": round(max(t_alu, t_hbm) * 1e6, 1),
                "frac": round(max(t_alu, t_hbm) / t, 3), "bound": ("tensor" if mode == "bf16_tc" else "alu") if t_alu > t_hbm else "hbm"}
+        if k == 1 and mode == "fp32" and cin >= 128:
+            # the same layer in the kernel's own layout (channel-major in and out, as the MobileNet chain calls it): no
+            # conversion pass, row-contiguous output
+            ld = (m + 3) // 4 * 4
+            xt, yt = torch.empty((cin, ld), device="cuda"), torch.empty((cout, ld), device="cuda")
+            sbnn.to_channel_major(xd, xt, m, cin, ld)
+            tc = _time_fn(torch, lambda: sbnn.conv1x1_gs_cm(p, xt, ld, yt, ld, m, flags | sbnn.SBNN_OUT_CM), reps, flush)
+            sbnn.get_async_status()
+            rec["us_channel_major"] = round(tc * 1e6, 1)
+            rec["frac_channel_major"] = round(max(t_alu, t_hbm) / tc, 3)
+            del xt, yt
         key = (m, cin, cout, k)
         if key not in dense:
             dense[key] = dense_library_us(torch, m, cin, cout, k, (n, h, w), max(3, reps // 2), flush)
