@@ -537,11 +537,12 @@ def test_channel_major_kernel_instances(g):
     not a multiple of 4, more channel steps than pipeline stages with a ragged last step, a ragged group tile."""
     for cfg in CM_CFGS[g]:
         tm = 32 * cfg[0]
-        d = WL.single_conv_inputs(1, 1, 2 * tm + 37, 212, 16 * 11, 1, g, 50, seed=8, mask_mode="layer_global")
-        for relu, out_cm in ((True, False), (False, True)):
-            y = run_cm(d, sbnn.SBNN_RELU if relu else 0, cfg, out_cm)
-            ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
-            assert_within(y, ref, s, what=f"cm G={g} cfg={cfg} relu={relu} out_cm={out_cm}")
+        for sp in (50, 75):          # sparse layers take the staged pixel-major epilogue where the tile shape has one
+            d = WL.single_conv_inputs(1, 1, 2 * tm + 37, 212, 16 * 11, 1, g, sp, seed=8, mask_mode="layer_global")
+            for relu, out_cm in ((True, False), (False, True)):
+                y = run_cm(d, sbnn.SBNN_RELU if relu else 0, cfg, out_cm)
+                ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
+                assert_within(y, ref, s, what=f"cm G={g} cfg={cfg} sp={sp} relu={relu} out_cm={out_cm}")
 
 
 @pytest.mark.parametrize("g", [1, 2, 4, 8, 16])
