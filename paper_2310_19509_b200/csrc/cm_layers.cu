@@ -393,6 +393,84 @@ dwconv3x3_cm_w14_kernel(const float* __restrict__ w, const float* __restrict__ b
     }
 }
 
+// 7 x 7 maps, stride 1 (the network's last depthwise layer): the planes of one channel are contiguous (49 floats per
+// image), so a CTA copies the planes of up to 64 images of 2 channels into shared memory with aligned 16-byte loads,
+// thread (channel, image) then holds its whole plane in registers (the 49 x 9 taps are unrolled with the padding
+// resolved at compile time; plane t starts at float 49*t, an odd stride, so the lanes hit distinct banks), writes the
+// 49 results back in place, and the CTA stores them with aligned 16-byte stores.  (One column strip per thread, as
+// for the wider maps, left a warp's loads scattered over 4-5 planes: 15 us at batch 64 where this takes 5.)
+__global__ void __launch_bounds__(128)
+dwconv3x3_cm_7x7_kernel(const float* __restrict__ w, const float* __restrict__ b, const float* __restrict__ x, int ldx,
+                        float* __restrict__ y, int ldy, int N, int C, int relu) {
+    constexpr int HW = 49, NI = 64;
+    __shared__ __align__(16) float sm[2][NI * HW];
+    const int tid = threadIdx.x, cl = tid >> 6, img = tid & 63;
+    const int n0 = blockIdx.x * NI, nimg = min(NI, N - n0), c0 = blockIdx.y * 2;
+    const int c = c0 + cl;
+    float wk[9];
+    float bias = 0.0f;
+    if (c < C) {
+#pragma unroll
+        for (int i = 0; i < 9; ++i) wk[i] = __ldg(w + i * C + c);
+        bias = b ? __ldg(b + c) : 0.0f;
+    }
+    grid_dependency_wait();      // the activations come from the previous kernel of the stream
+    grid_dependency_release();
+    const int total = nimg * HW;                                    // floats per channel in this CTA
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        if (c0 + k >= C) break;
+        const float* src = x + (size_t)(c0 + k) * ldx + (size_t)n0 * HW;   // 16-byte aligned: ldx and 64 * 49 are multiples of 4
+        for (int i = tid; i < (total + 3) / 4; i += 128) {
+            if (4 * i + 3 < total) {
+                *reinterpret_cast<float4*>(&sm[k][4 * i]) = __ldg(reinterpret_cast<const float4*>(src) + i);
+            } else {
+                for (int e = 4 * i; e < total; ++e) sm[k][e] = __ldg(src + e);
+            }
+        }
+    }
+    __syncthreads();
+    float out[HW];
+    const bool live = c < C && img < nimg;
+    if (live) {
+        float in[HW];
+#pragma unroll
+        for (int i = 0; i < HW; ++i) in[i] = sm[cl][img * HW + i];
+#pragma unroll
+        for (int oy = 0; oy < 7; ++oy)
+#pragma unroll
+            for (int ox = 0; ox < 7; ++ox) {
+                float acc = bias;
+#pragma unroll
+                for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+                    for (int kw = 0; kw < 3; ++kw) {
+                        const int iy = oy + kh - 1, ix = ox + kw - 1;
+                        if (iy >= 0 && iy < 7 && ix >= 0 && ix < 7) acc = fmaf(in[iy * 7 + ix], wk[kh * 3 + kw], acc);
+                    }
+                out[oy * 7 + ox] = relu ? fmaxf(acc, 0.0f) : acc;
+            }
+    }
+    __syncthreads();                                                // everybody has read its plane
+    if (live) {
+#pragma unroll
+        for (int i = 0; i < HW; ++i) sm[cl][img * HW + i] = out[i];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        if (c0 + k >= C) break;
+        float* dst = y + (size_t)(c0 + k) * ldy + (size_t)n0 * HW;
+        for (int i = tid; i < (total + 3) / 4; i += 128) {
+            if (4 * i + 3 < total) {
+                reinterpret_cast<float4*>(dst)[i] = *reinterpret_cast<const float4*>(&sm[k][4 * i]);
+            } else {
+                for (int e = 4 * i; e < total; ++e) dst[e] = sm[k][e];
+            }
+        }
+    }
+}
+
 // ---- first layer: NHWC image with Cin <= 4 in, channel-major out --------------------------------
 // Weights [Cout][3][3][Cin]; a CTA stages the 32 output channels of its channel group as [tap][Cin][32].
 // Generic kernel (Cout % 32 == 0): one thread computes 2 consecutive output columns x 32 output
@@ -652,7 +730,10 @@ sbnn_status launch_dwconv3x3_cm(const float* w, const float* b, const float* x, 
                 dim3 g14((unsigned)((N + NI2 - 1) / NI2), (C + 7) / 8);
                 SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_w14_kernel<NI2>, g14, 128, 0, st, w, b, x, ldx, y, ldy, N, C, relu));
             } else if (W == 14 && H % 7 == 0) SBNN_DW_C7(14)
-            else if (W == 7 && H % 7 == 0) SBNN_DW_C7(7)
+            else if (W == 7 && H == 7 && ldx % 4 == 0 && ldy % 4 == 0) {
+                dim3 g77((unsigned)((N + 63) / 64), (unsigned)((C + 1) / 2));
+                SBNN_CUDA_TRY(launch_kernel(dwconv3x3_cm_7x7_kernel, g77, 128, 0, st, w, b, x, ldx, y, ldy, N, C, relu));
+            } else if (W == 7 && H % 7 == 0) SBNN_DW_C7(7)
             else SBNN_DW_PX(1, 0);
         } else {
             if (W == 28) SBNN_DW_PX(2, 28);      // stride 2: the per-position kernel measured faster

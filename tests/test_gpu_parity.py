@@ -170,6 +170,26 @@ def test_depthwise_channel_major_variants(stride, hw, n, c):
     assert bool(torch.isnan(yt[:, n * ho * wo:]).all())          # nothing written past the last pixel
 
 
+def test_depthwise_7x7_kernel_with_more_images_than_one_cta_takes():
+    """The 7 x 7 kernel stages 64 images of two channels per CTA: 70 images give a full and a partial chunk, 5 channels
+    an odd last pair."""
+    rng = np.random.default_rng(42)
+    n, c = 70, 5
+    x = rng.random((n, 7, 7, c), dtype=np.float32)
+    wt = rng.standard_normal((3, 3, c)).astype(np.float32)
+    b = rng.standard_normal(c).astype(np.float32)
+    ld = (n * 49 + 3) // 4 * 4 + 4
+    xt = torch.zeros((c, ld), device="cuda")
+    xt[:, :n * 49] = dev(x).reshape(n * 49, c).t()
+    out = Guarded((c, ld))
+    sbnn.dwconv3x3_cm(dev(wt), dev(b), xt, ld, out.t, ld, n, 7, 7, c, 1)
+    sbnn.get_async_status()
+    full = out.numpy("dw 7x7")
+    assert np.all(np.isnan(full[:, n * 49:]))
+    ref, s = R.dwconv3x3(x, wt, b, stride=1, relu=True)
+    assert_within(full[:, :n * 49].T.reshape(n, 7, 7, c), ref, s, what="dw 7x7, 70 images")
+
+
 @pytest.mark.parametrize("n,h,w,cin,cout,relu_dw", [(3, 20, 28, 32, 64, True), (2, 9, 112, 32, 64, True), (5, 8, 12, 72, 40, False),
                                                     (1, 56, 56, 128, 128, True), (2, 3, 4, 8, 8, True)])
 def test_fused_depthwise_pointwise(n, h, w, cin, cout, relu_dw):
