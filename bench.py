@@ -364,6 +364,35 @@ def single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, reps):
     return out
 
 
+def other_chain_configs(sbnn, torch, default_batch, default_sparsity):
+    """The chain's other configurations (batch 64 at 70 %, batch 1 at 30 %): forward time by graph replay, inputs resident."""
+    from sbnn_inputs import mobilenet_v1_inputs
+    out = []
+    for batch, sp in ((64, 70), (1, 30)):
+        if (batch, sp) == (default_batch, default_sparsity):
+            continue
+        x, layers = mobilenet_v1_inputs(batch, sp, 4, seed=0)
+        net = build_network(sbnn, torch, layers, batch)
+        xd = torch.from_numpy(x).cuda()
+        logits = torch.empty((batch, 1000), device="cuda")
+        for _ in range(5):
+            net.forward(xd, logits, batch)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        reps = 100
+        ev0.record()
+        for _ in range(reps):
+            net.forward(xd, logits, batch)
+        ev1.record()
+        ev1.synchronize()
+        sbnn.get_async_status()
+        ms = ev0.elapsed_time(ev1) / reps
+        out.append({"batch": batch, "pointwise_sparsity_pct": sp, "ms_per_forward": round(ms, 4), "images_per_s": round(batch / ms * 1e3, 1)})
+        net.free()
+        del xd, logits
+    return out
+
+
 def max_over_ranks(values, world, device="cpu"):
     """Element-wise maximum of per-rank timings over the process group (the job is as slow as its slowest replica)."""
     if world <= 1:
@@ -510,6 +539,7 @@ def run_gpu(args, rank, world, local_rank):
                                                  for k in ("cublas_fp32_us", "cublas_tf32_us", "cudnn_fp32_us", "cudnn_tf32_us")}
         roofline["pointwise_us_per_step"] = round(pw_t * 1e6, 1)
     single = single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, 7) if (world == 1 and not args.no_single) else None
+    others = other_chain_configs(sbnn, torch, batch, args.sparsity) if (world == 1 and not args.no_single) else None
     cpu = cpu_baseline(x, layers) if world == 1 and not args.no_cpu else None
     imgs = batch * world * args.steps
     assert abs(job_throughput(batch, args.steps, world, elapsed) - imgs / elapsed) < 1e-6 * imgs / elapsed
@@ -531,6 +561,8 @@ def run_gpu(args, rank, world, local_rank):
     }
     if single is not None:
         line["single_layer"] = single
+    if others is not None:
+        line["other_chain_configs"] = others
     if cpu is not None:
         line["cpu_baseline"] = cpu
     print(json.dumps(line), flush=True)
