@@ -99,6 +99,17 @@ struct Stream3x3 {
     int32_t* blk_ptr = nullptr;
     int ntiles = 0, nchunks = 0;
     int max_blk = 0;
+    std::vector<int32_t> blk_host;   // host copy of blk_ptr: the block sizes weigh the shares of the persistent CTAs
+};
+
+// How one launch of the 3x3 copy-engine kernel deals the channel steps of its tiles to the persistent CTAs
+// (device memory; see conv3x3_gs.cu).
+struct Plan3x3 {
+    int32_t* cta_ptr = nullptr;  // [ncta + 1] offsets into segs
+    void* segs = nullptr;
+    int ncta = 0;
+    int nslots = 0;              // partial-sum slots the split tiles need
+    int ncounters = 0;           // split tiles
 };
 
 }  // namespace sbnn
@@ -123,6 +134,7 @@ struct sbnn_packed {
     mutable std::map<sbnn::TileCfg, sbnn::Stream1x1> streams_cm;   // channel-major kernel, see conv1x1_cm.cu
     mutable std::map<long long, sbnn::TileCfg> cfg_cm;             // tile shape chosen for a pixel count (the choice costs a loop over the tiles)
     mutable std::map<int, sbnn::Stream3x3> streams3x3;
+    mutable std::map<long long, sbnn::Plan3x3> plans3x3;           // per (stream, row tiles of the launch, CTAs)
     mutable void* bf16_stream = nullptr;  // see conv1x1_bf16.cu
     mutable void* umma_weights = nullptr; // dense bf16 copy of the masked weights, see conv1x1_umma.cu
 };

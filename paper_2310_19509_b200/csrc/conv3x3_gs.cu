@@ -35,9 +35,11 @@ struct Geo3 {
     int dpp_row, dpp_x;     // how (row, x) advance when a thread's staged pixel index grows by its stride
 };
 
-template <int G_, int CW_, int GPW_, int NPW_, int NGW_, int KC_>
+// RPL = output rows per lane (copy-engine kernel only): with two, a lane's CW x 2 outputs share the four input rows
+// and the nine weight vectors of a kept kernel, so 36 activation loads and 9 weight loads feed 2 * 63 * G FMAs.
+template <int G_, int CW_, int GPW_, int NPW_, int NGW_, int KC_, int RPL_ = 1>
 struct K3 {
-    static constexpr int G = G_, CW = CW_, GPW = GPW_, NPW = NPW_, NGW = NGW_, KC = KC_;
+    static constexpr int G = G_, CW = CW_, GPW = GPW_, NPW = NPW_, NGW = NGW_, KC = KC_, RPL = RPL_;
     static constexpr int NW = NPW * NGW, NT = NW * 32, GT = NGW * GPW;
     static constexpr int UNIT = 1 + (9 * G + 3) / 4;   // record of one kept unit, 16-byte units
     static constexpr int HDR = (GT * 2 + 3) / 4;
@@ -368,25 +370,44 @@ conv3x3_gs_cm_kernel(const float* __restrict__ X, int ldx, float* __restrict__ Y
 // images: rows of a neighbouring image are replaced by a row of zeros kept beside the stages.  Waits are bounded.
 struct Map3 { alignas(64) unsigned char bytes[128]; };
 
+// The launch is a fixed number of persistent CTAs (one per SM), and the channel steps of all tiles, laid end to end,
+// are dealt to them in equal shares of weight-stream volume, so a launch whose tile count is not a multiple of the SM
+// count (config 4 of the paper's Table-3-style shapes: 256 equal tiles on 148 SMs) leaves no SM idle in a last round.
+// A share is a list of segments; a tile that falls into several shares has nparts > 1: each part writes its partial
+// sums to its slot, counts itself in on the tile's counter, and the part that arrives last adds the slots in part
+// order (so the result does not depend on which part that was), adds the bias and stores the tile.  Nobody waits.
+struct Seg3 {
+    int bx, by;            // row tile, group tile
+    int k0, k1;            // channel steps [k0, k1)
+    int part, nparts;      // this segment's position among the tile's parts
+    int slot, counter;     // first partial-sum slot and arrival counter of the tile (nparts > 1)
+};
+
+__device__ __forceinline__ void compute_warps_barrier(int nthreads) {
+    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
+
 template <class C, bool PAT>
 __global__ void __launch_bounds__(C::NT + 32, 1)
 conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, const float* __restrict__ bias,
                       const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, Geo3 geo, int relu, int S,
-                      int stage_bytes, int* status) {
-    constexpr int G = C::G, CW = C::CW, GPW = C::GPW, KC = C::KC, NW = C::NW;
+                      int stage_bytes, int* status, const int32_t* __restrict__ cta_ptr, const Seg3* __restrict__ segs,
+                      f32x2* partial, int* counters) {
+    constexpr int G = C::G, CW = C::CW, GPW = C::GPW, KC = C::KC, NW = C::NW, RPL = C::RPL;
     constexpr int GP = (G + 1) / 2;
+    static_assert(!PAT || RPL == 1, "the tap lists address one output row per lane");
+    constexpr int ACC2 = GPW * RPL * CW * GP;                            // packed partial sums per thread
     extern __shared__ __align__(128) unsigned char smem[];
     const int xs_bytes = KC * geo.plane * 4;                       // one stage: KC planes, then the weight block
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
     uint64_t* empty = full + S;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + S);
+    volatile int* last_flag = abort_flag + 1;
     float* zrow = reinterpret_cast<float*>(empty + S) + 4;         // geo.pitch zeros
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int f0 = blockIdx.x * geo.R;
-    const int tile = blockIdx.y;
     const int NH = geo.N * geo.H, W = geo.W;
-    const int32_t* bp = blk_ptr + (size_t)tile * (geo.nchunks + 1);
+    const int seg_beg = cta_ptr[blockIdx.x], seg_end = cta_ptr[blockIdx.x + 1];
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -394,6 +415,7 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
             mbar_init(empty + s, NW);
         }
         *abort_flag = 0;
+        *last_flag = 0;
         mbar_fence_init();
     }
     for (int i = tid; i < geo.pitch; i += blockDim.x) zrow[i] = 0.0f;
@@ -402,21 +424,26 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
     if (warp == NW) {
         // ---------------- producer warp ----------------
         bool ok = true;
-        int k = 0;
-        for (; k < geo.nchunks && ok; ++k) {
-            const int s = k % S;
-            if (k >= S) ok = mbar_wait(empty + s, ((k / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
-            if (!ok) break;
-            if (lane == 0) {
-                const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
-                unsigned char* st = smem + (size_t)s * stage_bytes;
-                mbar_arrive_expect_tx(full + s, (uint32_t)xs_bytes + (uint32_t)wn * 16u);
-                tensor_g2s_3d(st, &xmap, -4, f0 - 1, k * KC, full + s);
-                bulk_g2s(st + xs_bytes, rec + wbeg, (uint32_t)wn * 16u, full + s);
+        int it = 0;                                                // steps issued by this CTA so far (all segments)
+        for (int si = seg_beg; si < seg_end && ok; ++si) {
+            const Seg3 sg = segs[si];
+            const int32_t* bp = blk_ptr + (size_t)sg.by * (geo.nchunks + 1);
+            const int f0 = sg.bx * geo.R;
+            for (int k = sg.k0; k < sg.k1; ++k, ++it) {
+                const int s = it % S;
+                if (it >= S) ok = mbar_wait(empty + s, ((it / S) & 1) ^ 1, abort_flag, status, SBNN_ERR_TIMEOUT);
+                if (!ok) break;
+                if (lane == 0) {
+                    const int wbeg = bp[k], wn = bp[k + 1] - wbeg;
+                    unsigned char* st = smem + (size_t)s * stage_bytes;
+                    mbar_arrive_expect_tx(full + s, (uint32_t)xs_bytes + (uint32_t)wn * 16u);
+                    tensor_g2s_3d(st, &xmap, -4, f0 - 1, k * KC, full + s);
+                    bulk_g2s(st + xs_bytes, rec + wbeg, (uint32_t)wn * 16u, full + s);
+                }
             }
         }
         if (!ok) {   // gave up: let the copies already issued land before the CTA's shared memory is released
-            for (int j = max(0, k - S); j < k; ++j) {
+            for (int j = max(0, it - S); j < it; ++j) {
                 bool landed = false;
                 for (uint32_t i = 0; i < kWaitLimit && !landed; ++i) landed = mbar_try_wait(full + j % S, (j / S) & 1);
             }
@@ -426,148 +453,242 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
 
     // ---------------- compute warps ----------------
     const int pw = warp % C::NPW, gw = warp / C::NPW;
-    const int lrow = pw * geo.RPW + lane / geo.LPR;
+    const int lrow = (pw * geo.RPW + lane / geo.LPR) * RPL;      // first of the lane's RPL output rows
     const int lx = (lane % geo.LPR) * CW;
-    const int f = f0 + lrow;
-    const int y = f % geo.H;
     // plane row j holds image row f0 - 1 + j; column c holds x = c - 4
-    int rowoff[3];
-    bool rowok[3];
+    int rowoff[RPL + 2];
 #pragma unroll
-    for (int kh = 0; kh < 3; ++kh) {
-        rowoff[kh] = (lrow + kh) * geo.pitch + lx + 3;             // column of x = lx - 1
-        rowok[kh] = (kh == 0) ? (y > 0) : (kh == 2 ? (y < geo.H - 1) : true);
-    }
+    for (int jr = 0; jr < RPL + 2; ++jr) rowoff[jr] = (lrow + jr) * geo.pitch + lx + 3;   // column of x = lx - 1
     const float* zr = zrow + lx + 3;
     const int lanebase = lrow * geo.pitch + lx + 3;                // tap (kh, kw) of a plane: + kh * pitch + kw, then CW inputs
-    const unsigned rowmask = (rowok[0] ? 1u : 0u) | 2u | (rowok[2] ? 4u : 0u);
 
-    f32x2 acc[GPW][CW][GP];
-#pragma unroll
-    for (int q = 0; q < GPW; ++q) {
-        const int g = tile * C::GT + gw * GPW + q;
-#pragma unroll
-        for (int r = 0; r < GP; ++r) {
-            const float b0 = (g < geo.ngroups) ? bias[g * G + 2 * r] : 0.0f;
-            const float b1 = (g < geo.ngroups && 2 * r + 1 < G) ? bias[g * G + 2 * r + 1] : 0.0f;
-#pragma unroll
-            for (int p = 0; p < CW; ++p) acc[q][p][r] = pack2(b0, b1);
-        }
-    }
+    int it = 0;                                                    // steps consumed by this CTA so far (all segments)
+    bool alive = true;                                             // false once a wait has given up; the barriers below are still joined
+    for (int si = seg_beg; si < seg_end; ++si) {
+        const Seg3 sg = segs[si];
+        const bool split = sg.nparts > 1;
+        const int tile = sg.by;
+        const int f = sg.bx * geo.R + lrow;
+        const int y = f % geo.H;
+        // the lane's RPL rows lie in one image (H is a multiple of RPL), so only the rows above the first and below
+        // the last can belong to a neighbouring image
+        const bool ok_first = y > 0, ok_last = y + RPL - 1 < geo.H - 1;
+        const unsigned rowmask = (ok_first ? 1u : 0u) | 2u | (ok_last ? 4u : 0u);
+        (void)rowmask;
 
-    for (int k = 0; k < geo.nchunks; ++k) {
-        const int s = k % S;
-        if (!mbar_wait(full + s, (k / S) & 1, abort_flag, status, SBNN_ERR_TIMEOUT)) return;
-        const float* xs = reinterpret_cast<const float*>(smem + (size_t)s * stage_bytes);
-        const uint4* ws = reinterpret_cast<const uint4*>(smem + (size_t)s * stage_bytes + xs_bytes);
+        f32x2 acc[GPW][RPL][CW][GP];
 #pragma unroll
         for (int q = 0; q < GPW; ++q) {
-            const int2 hd = reinterpret_cast<const int2*>(ws)[gw * GPW + q];
-            const uint4* r = ws + hd.x;
-            if constexpr (PAT) {
-                // Layers packed with kernel patterns (Section 3.3): the stream lists the kept taps of the group's kept
-                // kernels one by one, four to a record (offset of the tap's first input inside the stage with the kernel
-                // row in the top two bits, then the G weights of each), so pruned taps cost nothing and the loop has no
-                // data-dependent branch.  A list is padded to a whole record with taps of weight zero.
-                for (int it = 0; it < hd.y; ++it, r += C::TQUAD) {
-                    const uint4 off4 = r[0];
-                    const unsigned offs[4] = {off4.x, off4.y, off4.z, off4.w};
+            const int g = tile * C::GT + gw * GPW + q;
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const unsigned kh = offs[u] >> 30;
-                        const float* arow = ((rowmask >> kh) & 1u) ? xs + (offs[u] & 0x3FFFFFFFu) + lanebase : zr;
-                        f32x2 a[CW];
+            for (int r = 0; r < GP; ++r) {
+                // a tile in one piece starts from the bias; the parts of a split tile start from zero
+                const float b0 = (!split && g < geo.ngroups) ? bias[g * G + 2 * r] : 0.0f;
+                const float b1 = (!split && g < geo.ngroups && 2 * r + 1 < G) ? bias[g * G + 2 * r + 1] : 0.0f;
 #pragma unroll
-                        for (int i = 0; i < CW; ++i) a[i] = dup2(arow[i]);
-                        const float* wq = reinterpret_cast<const float*>(r + 1) + u * G;
-                        f32x2 w[GP];
-                        if constexpr (G % 4 == 0) {
+                for (int ro = 0; ro < RPL; ++ro)
 #pragma unroll
-                            for (int v = 0; v < G / 4; ++v) {
-                                const ulonglong2 t = reinterpret_cast<const ulonglong2*>(wq)[v];
-                                w[2 * v] = t.x;
-                                w[2 * v + 1] = t.y;
-                            }
-                        } else if constexpr (G == 2) {
-                            w[0] = *reinterpret_cast<const unsigned long long*>(wq);
-                        } else {
-                            w[0] = pack2(wq[0], 0.0f);
-                        }
-#pragma unroll
-                        for (int p = 0; p < CW; ++p)
-#pragma unroll
-                            for (int rr = 0; rr < GP; ++rr) fma2(acc[q][p][rr], a[p], w[rr]);
-                    }
-                }
-            } else {
-            for (int it = 0; it < hd.y; ++it, r += C::UNIT) {
-                const float* plane = xs + r[0].x;
-                const float* wq = reinterpret_cast<const float*>(r + 1);   // [9][G]
-#pragma unroll
-                for (int kh = 0; kh < 3; ++kh) {
-                    const float* arow = rowok[kh] ? plane + rowoff[kh] : zr;
-                    f32x2 a[CW + 2];
-#pragma unroll
-                    for (int i = 0; i < CW + 2; ++i) a[i] = dup2(arow[i]);
-#pragma unroll
-                    for (int kw = 0; kw < 3; ++kw) {
-                        f32x2 w[GP];
-                        if constexpr (G % 4 == 0) {
-#pragma unroll
-                            for (int v = 0; v < G / 4; ++v) {
-                                const ulonglong2 t = reinterpret_cast<const ulonglong2*>(wq + (kh * 3 + kw) * G)[v];
-                                w[2 * v] = t.x;
-                                w[2 * v + 1] = t.y;
-                            }
-                        } else if constexpr (G == 2) {
-                            w[0] = *reinterpret_cast<const unsigned long long*>(wq + (kh * 3 + kw) * 2);
-                        } else {
-                            w[0] = pack2(wq[kh * 3 + kw], 0.0f);
-                        }
-#pragma unroll
-                        for (int p = 0; p < CW; ++p)
-#pragma unroll
-                            for (int rr = 0; rr < GP; ++rr) fma2(acc[q][p][rr], a[p + kw], w[rr]);
-                    }
-                }
-            }
+                    for (int p = 0; p < CW; ++p) acc[q][ro][p][r] = pack2(b0, b1);
             }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty + s);
-    }
 
-    if (f >= NH) return;
+        if (alive) {
+            for (int k = sg.k0; k < sg.k1; ++k, ++it) {
+                const int s = it % S;
+                if (!mbar_wait(full + s, (it / S) & 1, abort_flag, status, SBNN_ERR_TIMEOUT)) {
+                    alive = false;
+                    break;
+                }
+                const float* xs = reinterpret_cast<const float*>(smem + (size_t)s * stage_bytes);
+                const uint4* ws = reinterpret_cast<const uint4*>(smem + (size_t)s * stage_bytes + xs_bytes);
 #pragma unroll
-    for (int q = 0; q < GPW; ++q) {
-        const int g = tile * C::GT + gw * GPW + q;
-        if (g >= geo.ngroups) continue;
+                for (int q = 0; q < GPW; ++q) {
+                    const int2 hd = reinterpret_cast<const int2*>(ws)[gw * GPW + q];
+                    const uint4* r = ws + hd.x;
+                    if constexpr (PAT) {
+                        // Layers packed with kernel patterns (Section 3.3): the stream lists the kept taps of the group's kept
+                        // kernels one by one, four to a record (offset of the tap's first input inside the stage with the kernel
+                        // row in the top two bits, then the G weights of each), so pruned taps cost nothing and the loop has no
+                        // data-dependent branch.  A list is padded to a whole record with taps of weight zero.
+                        for (int j = 0; j < hd.y; ++j, r += C::TQUAD) {
+                            const uint4 off4 = r[0];
+                            const unsigned offs[4] = {off4.x, off4.y, off4.z, off4.w};
 #pragma unroll
-        for (int p = 0; p < CW; ++p) {
-            const int x = lx + p;
-            if (x >= W) continue;
-            float* yp = Y + ((size_t)f * W + x) * geo.Cout + g * G;
-            float v[2 * GP];
+                            for (int u = 0; u < 4; ++u) {
+                                const unsigned kh = offs[u] >> 30;
+                                const float* arow = ((rowmask >> kh) & 1u) ? xs + (offs[u] & 0x3FFFFFFFu) + lanebase : zr;
+                                f32x2 a[CW];
 #pragma unroll
-            for (int rr = 0; rr < GP; ++rr) unpack2(acc[q][p][rr], v[2 * rr], v[2 * rr + 1]);
-            if (relu) {
+                                for (int i = 0; i < CW; ++i) a[i] = dup2(arow[i]);
+                                const float* wq = reinterpret_cast<const float*>(r + 1) + u * G;
+                                f32x2 w[GP];
+                                if constexpr (G % 4 == 0) {
 #pragma unroll
-                for (int rr = 0; rr < 2 * GP; ++rr) v[rr] = fmaxf(v[rr], 0.0f);
+                                    for (int v = 0; v < G / 4; ++v) {
+                                        const ulonglong2 t = reinterpret_cast<const ulonglong2*>(wq)[v];
+                                        w[2 * v] = t.x;
+                                        w[2 * v + 1] = t.y;
+                                    }
+                                } else if constexpr (G == 2) {
+                                    w[0] = *reinterpret_cast<const unsigned long long*>(wq);
+                                } else {
+                                    w[0] = pack2(wq[0], 0.0f);
+                                }
+#pragma unroll
+                                for (int p = 0; p < CW; ++p)
+#pragma unroll
+                                    for (int rr = 0; rr < GP; ++rr) fma2(acc[q][0][p][rr], a[p], w[rr]);
+                            }
+                        }
+                    } else {
+                    for (int j = 0; j < hd.y; ++j, r += C::UNIT) {
+                        const float* plane = xs + r[0].x;
+                        const float* wq = reinterpret_cast<const float*>(r + 1);   // [9][G]
+                        f32x2 w[3][3][GP];                                          // tap row kh is fetched with input row kh
+#pragma unroll
+                        for (int jr = 0; jr < RPL + 2; ++jr) {
+                            const bool ok = jr == 0 ? ok_first : (jr == RPL + 1 ? ok_last : true);
+                            const float* arow = ok ? plane + rowoff[jr] : zr;
+                            f32x2 a[CW + 2];
+#pragma unroll
+                            for (int i = 0; i < CW + 2; ++i) a[i] = dup2(arow[i]);
+                            if (jr < 3) {
+#pragma unroll
+                                for (int kw = 0; kw < 3; ++kw) {
+                                    if constexpr (G % 4 == 0) {
+#pragma unroll
+                                        for (int v = 0; v < G / 4; ++v) {
+                                            const ulonglong2 t = reinterpret_cast<const ulonglong2*>(wq + (jr * 3 + kw) * G)[v];
+                                            w[jr < 3 ? jr : 0][kw][2 * v] = t.x;
+                                            w[jr < 3 ? jr : 0][kw][2 * v + 1] = t.y;
+                                        }
+                                    } else if constexpr (G == 2) {
+                                        w[jr < 3 ? jr : 0][kw][0] = *reinterpret_cast<const unsigned long long*>(wq + (jr * 3 + kw) * 2);
+                                    } else {
+                                        w[jr < 3 ? jr : 0][kw][0] = pack2(wq[jr * 3 + kw], 0.0f);
+                                    }
+                                }
+                            }
+                            // input row jr is tap row kh = jr - ro of output row ro
+#pragma unroll
+                            for (int ro = 0; ro < RPL; ++ro) {
+                                const int kh = jr - ro;
+                                if (kh < 0 || kh > 2) continue;
+#pragma unroll
+                                for (int kw = 0; kw < 3; ++kw)
+#pragma unroll
+                                    for (int p = 0; p < CW; ++p)
+#pragma unroll
+                                        for (int rr = 0; rr < GP; ++rr) fma2(acc[q][ro][p][rr], a[p + kw], w[kh][kw][rr]);
+                            }
+                        }
+                    }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty + s);
             }
-            if constexpr (G >= 4) {
+        }
+
+        if (split) {
+            // partial sums of this part -> its slot, [packed sum][thread]
+            f32x2* mine = partial + (size_t)(sg.slot + sg.part) * (ACC2 * C::NT) + tid;
+            if (alive) {
 #pragma unroll
-                for (int vv = 0; vv < G / 4; ++vv)
-                    reinterpret_cast<float4*>(yp)[vv] = make_float4(v[4 * vv], v[4 * vv + 1], v[4 * vv + 2], v[4 * vv + 3]);
-            } else if constexpr (G == 2) {
-                *reinterpret_cast<float2*>(yp) = make_float2(v[0], v[1]);
-            } else {
-                yp[0] = v[0];
+                for (int q = 0; q < GPW; ++q)
+#pragma unroll
+                    for (int ro = 0; ro < RPL; ++ro)
+#pragma unroll
+                        for (int p = 0; p < CW; ++p)
+#pragma unroll
+                            for (int rr = 0; rr < GP; ++rr)
+                                mine[(size_t)(((q * RPL + ro) * CW + p) * GP + rr) * C::NT] = acc[q][ro][p][rr];
+            }
+            __threadfence();
+            compute_warps_barrier(C::NT);
+            if (tid == 0) *last_flag = (!*abort_flag && atomicAdd(counters + sg.counter, 1) == sg.nparts - 1) ? 1 : 0;
+            compute_warps_barrier(C::NT);
+            const bool last = *last_flag != 0;
+            if (!last || !alive) continue;
+            __threadfence();
+            const f32x2* first = partial + (size_t)sg.slot * (ACC2 * C::NT) + tid;
+#pragma unroll
+            for (int q = 0; q < GPW; ++q) {
+                const int g = tile * C::GT + gw * GPW + q;
+#pragma unroll
+                for (int rr = 0; rr < GP; ++rr) {
+                    const float b0 = (g < geo.ngroups) ? bias[g * G + 2 * rr] : 0.0f;
+                    const float b1 = (g < geo.ngroups && 2 * rr + 1 < G) ? bias[g * G + 2 * rr + 1] : 0.0f;
+#pragma unroll
+                    for (int ro = 0; ro < RPL; ++ro)
+#pragma unroll
+                    for (int p = 0; p < CW; ++p) {
+                        const f32x2* src = first + (size_t)(((q * RPL + ro) * CW + p) * GP + rr) * C::NT;
+                        float s0, s1;
+                        unpack2(__ldcg(src), s0, s1);
+                        for (int j = 1; j < sg.nparts; ++j) {
+                            float t0, t1;
+                            unpack2(__ldcg(src + (size_t)j * (ACC2 * C::NT)), t0, t1);
+                            s0 += t0;
+                            s1 += t1;
+                        }
+                        acc[q][ro][p][rr] = pack2(s0 + b0, s1 + b1);
+                    }
+                }
+            }
+        } else if (!alive) {
+            continue;
+        }
+
+#pragma unroll
+        for (int q = 0; q < GPW; ++q) {
+            const int g = tile * C::GT + gw * GPW + q;
+            if (g >= geo.ngroups) continue;
+#pragma unroll
+            for (int ro = 0; ro < RPL; ++ro)
+#pragma unroll
+            for (int p = 0; p < CW; ++p) {
+                const int x = lx + p;
+                if (x >= W || f + ro >= NH) continue;
+                float* yp = Y + ((size_t)(f + ro) * W + x) * geo.Cout + g * G;
+                float v[2 * GP];
+#pragma unroll
+                for (int rr = 0; rr < GP; ++rr) unpack2(acc[q][ro][p][rr], v[2 * rr], v[2 * rr + 1]);
+                if (relu) {
+#pragma unroll
+                    for (int rr = 0; rr < 2 * GP; ++rr) v[rr] = fmaxf(v[rr], 0.0f);
+                }
+                if constexpr (G >= 4) {
+#pragma unroll
+                    for (int vv = 0; vv < G / 4; ++vv)
+                        reinterpret_cast<float4*>(yp)[vv] = make_float4(v[4 * vv], v[4 * vv + 1], v[4 * vv + 2], v[4 * vv + 3]);
+                } else if constexpr (G == 2) {
+                    *reinterpret_cast<float2*>(yp) = make_float2(v[0], v[1]);
+                } else {
+                    yp[0] = v[0];
+                }
             }
         }
     }
 }
 
 // ---- host side -------------------------------------------------------------------------------
+
+// Number of SMs of the current device (one persistent CTA each).
+int sm_count3() {
+    static std::mutex mu;
+    static std::map<int, int> n;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = n.find(dev);
+    if (it == n.end()) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        it = n.emplace(dev, v).first;
+    }
+    return it->second;
+}
 
 int pow2_ceil(int v) {
     int p = 1;
@@ -639,6 +760,7 @@ sbnn_status build_stream3(const sbnn_packed* p, int GT, int KC, int plane, Strea
     }
     Stream3x3 s;
     s.ntiles = ntiles; s.nchunks = nchunks; s.max_blk = max_blk;
+    s.blk_host = blk;
     SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&s.rec), std::max<size_t>(rec.size() * 4, 16)));
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s.blk_ptr), blk.size() * 4);
     if (e == cudaSuccess && !rec.empty()) e = cudaMemcpy(s.rec, rec.data(), rec.size() * 4, cudaMemcpyHostToDevice);
@@ -649,7 +771,7 @@ sbnn_status build_stream3(const sbnn_packed* p, int GT, int KC, int plane, Strea
         cudaGetLastError();
         return fail(SBNN_ERR_CUDA, "uploading the 3x3 weight stream: %s", cudaGetErrorString(e));
     }
-    *out = s;
+    *out = std::move(s);
     return SBNN_OK;
 }
 
@@ -703,6 +825,7 @@ sbnn_status build_stream3_taps(const sbnn_packed* p, int GT, int KC, int plane, 
     }
     Stream3x3 s;
     s.ntiles = ntiles; s.nchunks = nchunks; s.max_blk = max_blk;
+    s.blk_host = blk;
     SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&s.rec), std::max<size_t>(rec.size() * 4, 16)));
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s.blk_ptr), blk.size() * 4);
     if (e == cudaSuccess && !rec.empty()) e = cudaMemcpy(s.rec, rec.data(), rec.size() * 4, cudaMemcpyHostToDevice);
@@ -713,7 +836,79 @@ sbnn_status build_stream3_taps(const sbnn_packed* p, int GT, int KC, int plane, 
         cudaGetLastError();
         return fail(SBNN_ERR_CUDA, "uploading the 3x3 tap stream: %s", cudaGetErrorString(e));
     }
-    *out = s;
+    *out = std::move(s);
+    return SBNN_OK;
+}
+
+// Deals the channel steps of a launch (row tiles x group tiles x steps, row tiles fastest) to `ncta` persistent CTAs
+// in shares of equal weight: a step weighs its weight block (16-byte words: the kept kernels or taps it multiplies) plus
+// a constant for what every step costs (barrier round trip, list headers).  A share is cut into segments at tile
+// borders; tiles that end up in several shares get partial-sum slots and an arrival counter.
+sbnn_status build_plan3(const Stream3x3& s, int nrow, int ncta_max, Plan3x3* out) {
+    const int n = s.nchunks;
+    const long long T = (long long)nrow * s.ntiles, steps = T * n;
+    const int ncta = (int)std::max<long long>(1, std::min<long long>(ncta_max, steps));
+    constexpr long long kStepCost = 6;
+    long long total = 0;
+    for (int by = 0; by < s.ntiles; ++by) {
+        total += ((long long)(s.blk_host[(size_t)by * (n + 1) + n] - s.blk_host[(size_t)by * (n + 1)]) + kStepCost * n) * nrow;
+    }
+    std::vector<int32_t> cta_ptr(ncta + 1, 0);
+    std::vector<Seg3> segs;
+    try {
+        long long cum = 0;
+        int cur_cta = 0;
+        for (int by = 0; by < s.ntiles; ++by) {
+            const int32_t* bp = s.blk_host.data() + (size_t)by * (n + 1);
+            for (int bx = 0; bx < nrow; ++bx) {
+                int part = 0;
+                int k = 0;
+                while (k < n) {
+                    // the CTA that owns the step starting at cumulative weight `cum`
+                    int c = total > 0 ? (int)std::min<long long>(ncta - 1, (__int128)cum * ncta / total) : 0;
+                    if (c < cur_cta) c = cur_cta;
+                    while (cur_cta < c) cta_ptr[++cur_cta] = (int32_t)segs.size();
+                    // this CTA's share ends at weight (c + 1) * total / ncta: take steps while they start below it
+                    const long long lim = (long long)(((__int128)(c + 1) * total + ncta - 1) / ncta);
+                    const int k0 = k;
+                    while (k < n && (k == k0 || cum < lim)) {
+                        cum += (long long)(bp[k + 1] - bp[k]) + kStepCost;
+                        ++k;
+                    }
+                    const Seg3 sg = {bx, by, k0, k, part++, 0, 0, 0};
+                    segs.push_back(sg);
+                }
+                // the tile's segments are the last `part` entries
+                for (int j = 0; j < part; ++j) segs[segs.size() - 1 - j].nparts = part;
+            }
+        }
+        while (cur_cta < ncta) cta_ptr[++cur_cta] = (int32_t)segs.size();
+    } catch (const std::bad_alloc&) {
+        return fail(SBNN_ERR_ALLOC, "out of host memory planning the 3x3 launch");
+    }
+    Plan3x3 pl;
+    pl.ncta = ncta;
+    for (size_t i = 0; i < segs.size(); ++i) {
+        if (segs[i].nparts > 1 && segs[i].part == 0) {
+            for (int j = 0; j < segs[i].nparts; ++j) {
+                segs[i + j].slot = pl.nslots;
+                segs[i + j].counter = pl.ncounters;
+            }
+            pl.nslots += segs[i].nparts;
+            pl.ncounters += 1;
+        }
+    }
+    SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&pl.cta_ptr), cta_ptr.size() * 4));
+    cudaError_t e = cudaMalloc(&pl.segs, std::max<size_t>(segs.size() * sizeof(Seg3), 32));
+    if (e == cudaSuccess) e = cudaMemcpy(pl.cta_ptr, cta_ptr.data(), cta_ptr.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !segs.empty()) e = cudaMemcpy(pl.segs, segs.data(), segs.size() * sizeof(Seg3), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(pl.cta_ptr);
+        cudaFree(pl.segs);
+        cudaGetLastError();
+        return fail(SBNN_ERR_CUDA, "uploading the 3x3 launch plan: %s", cudaGetErrorString(e));
+    }
+    *out = pl;
     return SBNN_OK;
 }
 
@@ -736,19 +931,20 @@ sbnn_status launch3(const sbnn_packed* p, const float* x, float* y, int N, int H
     if (smem > 227 * 1024) return fail(SBNN_ERR_UNSUPPORTED, "3x3 tile for W=%d needs %zu bytes of shared memory", W, smem);
 
     // the stream's plane offsets depend on the plane size, hence on (W, tile shape)
-    Stream3x3 s;
+    const Stream3x3* sp = nullptr;
     {
         std::lock_guard<std::mutex> lk(p->mu);
         const int key = (plane << 8) | (C::GT << 4) | (C::KC / 4);
         auto it = p->streams3x3.find(key);
         if (it == p->streams3x3.end()) {
-            sbnn_status r = build_stream3(p, C::GT, C::KC, plane, &s);
+            Stream3x3 built;
+            sbnn_status r = build_stream3(p, C::GT, C::KC, plane, &built);
             if (r != SBNN_OK) return r;
-            p->streams3x3[key] = s;
-        } else {
-            s = it->second;
+            it = p->streams3x3.emplace(key, std::move(built)).first;
         }
+        sp = &it->second;   // map nodes stay where they are until the layer is freed
     }
+    const Stream3x3& s = *sp;
     if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
     sbnn_status ra = set_max_dyn_smem(reinterpret_cast<const void*>(&conv3x3_gs_kernel<C>), (int)smem);
     if (ra != SBNN_OK) return ra;
@@ -762,13 +958,13 @@ sbnn_status launch3(const sbnn_packed* p, const float* x, float* y, int N, int H
 
 // Pitch for the channel-major variant: a multiple of 4 (16-byte aligned row pieces), >= LPR*CW + 5, and such
 // that the first reads of the 32 lanes fall into 32 distinct banks if possible.
-int pick_pitch4(int LPR, int CW) {
+int pick_pitch4(int LPR, int CW, int RPL = 1) {
     const int lo = (LPR * CW + 5 + 3) / 4 * 4;
     for (int p = lo; p < lo + 128; p += 4) {
         unsigned used = 0;
         bool ok = true;
         for (int l = 0; l < 32 && ok; ++l) {
-            const int b = ((l / LPR) * p + (l % LPR) * CW) & 31;
+            const int b = ((l / LPR) * RPL * p + (l % LPR) * CW) & 31;
             ok = !((used >> b) & 1u);
             used |= 1u << b;
         }
@@ -795,19 +991,20 @@ sbnn_status launch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y,
     const size_t smem = (size_t)2 * C::KC * plane * 4 + (size_t)2 * C::WS_U4 * 16;
     const long long pieces = (long long)(g.R + 2) * (W / 4);
     if (smem > 227 * 1024 || pieces > 2LL * C::NT || (long long)N * H * W * 1 > 0x7fffffffLL / 2) return SBNN_OK;
-    Stream3x3 s;
+    const Stream3x3* sp = nullptr;
     {
         std::lock_guard<std::mutex> lk(p->mu);
         const int key = (plane << 8) | (C::GT << 4) | (C::KC / 4);
         auto it = p->streams3x3.find(key);
         if (it == p->streams3x3.end()) {
-            sbnn_status r = build_stream3(p, C::GT, C::KC, plane, &s);
+            Stream3x3 built;
+            sbnn_status r = build_stream3(p, C::GT, C::KC, plane, &built);
             if (r != SBNN_OK) return r;
-            p->streams3x3[key] = s;
-        } else {
-            s = it->second;
+            it = p->streams3x3.emplace(key, std::move(built)).first;
         }
+        sp = &it->second;   // map nodes stay where they are until the layer is freed
     }
+    const Stream3x3& s = *sp;
     if (s.max_blk > C::WS_U4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, C::WS_U4);
     sbnn_status ra = set_max_dyn_smem(reinterpret_cast<const void*>(&conv3x3_gs_cm_kernel<C>), (int)smem);
     if (ra != SBNN_OK) return ra;
@@ -826,15 +1023,16 @@ sbnn_status launch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y,
 // Launches the copy-engine variant; *done = false (and SBNN_OK) if the shape does not fit it.
 template <class C>
 sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
-                        cudaStream_t st, bool* done) {
+                        cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
     *done = false;
     Geo3 g;
     g.N = N; g.H = H; g.W = W; g.Cin = p->Cin; g.Cout = p->Cout; g.ngroups = p->ngroups;
     g.LPR = lanes_per_row(W, C::CW);
     g.RPW = 32 / g.LPR;
-    g.R = C::NPW * g.RPW;
-    g.pitch = pick_pitch4(g.LPR, C::CW);
+    g.R = C::NPW * g.RPW * C::RPL;
+    g.pitch = pick_pitch4(g.LPR, C::CW, C::RPL);
     g.plane = (g.R + 2) * g.pitch;                                 // the copied box: no padding between planes
+    if (H % C::RPL) return SBNN_OK;                                // a lane's rows must lie in one image
     g.nchunks = (p->Cin + C::KC - 1) / C::KC;
     g.dpp_row = g.dpp_x = 0;
     if (g.pitch > 256 || g.R + 2 > 256 || W % 4 || ldx % 4) return SBNN_OK;
@@ -847,21 +1045,38 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     if ((size_t)S * stage_bytes + tail > 227 * 1024) S = 2;
     const size_t smem = (size_t)S * stage_bytes + tail;
     if (smem > 227 * 1024) return SBNN_OK;
-    Stream3x3 s;
+    const long long NH = (long long)N * H;
+    const int nrow = (int)((NH + g.R - 1) / g.R);
+    const Stream3x3* sp = nullptr;
+    Plan3x3 plan;
     {
         std::lock_guard<std::mutex> lk(p->mu);
         const int key = (g.plane << 8) | (C::GT << 4) | (C::KC / 4) | (pat ? (1 << 30) : 0);
         auto it = p->streams3x3.find(key);
         if (it == p->streams3x3.end()) {
-            sbnn_status r = pat ? build_stream3_taps(p, C::GT, C::KC, g.plane, g.pitch, &s) : build_stream3(p, C::GT, C::KC, g.plane, &s);
+            Stream3x3 built;
+            sbnn_status r = pat ? build_stream3_taps(p, C::GT, C::KC, g.plane, g.pitch, &built) : build_stream3(p, C::GT, C::KC, g.plane, &built);
             if (r != SBNN_OK) return r;
-            p->streams3x3[key] = s;
-        } else {
-            s = it->second;
+            it = p->streams3x3.emplace(key, std::move(built)).first;
         }
+        sp = &it->second;   // map nodes stay where they are until the layer is freed
+        const int ncta = sm_count3();
+        const long long pkey = ((long long)key << 32) | ((long long)(nrow & 0xFFFFF) << 12) | (long long)(ncta & 0xFFF);
+        auto ip = p->plans3x3.find(pkey);
+        if (ip == p->plans3x3.end()) {
+            Plan3x3 built;
+            sbnn_status r = build_plan3(*sp, nrow, ncta, &built);
+            if (r != SBNN_OK) return r;
+            ip = p->plans3x3.emplace(pkey, built).first;
+        }
+        plan = ip->second;
     }
+    const Stream3x3& s = *sp;
     if (s.max_blk > ws_u4) return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 weight block %d exceeds buffer %d", s.max_blk, ws_u4);
-    sbnn_status r = set_max_dyn_smem(pat ? reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C, true>)
+    constexpr bool kTapLists = C::RPL == 1;                        // instances with several rows per lane have no tap-list form
+    if (pat && !kTapLists) return SBNN_OK;
+    using CP = K3<C::G, C::CW, C::GPW, C::NPW, C::NGW, C::KC, 1>;  // == C wherever the tap-list kernel is launched
+    sbnn_status r = set_max_dyn_smem(pat ? reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<CP, true>)
                                          : reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C, false>), (int)smem);
     if (r != SBNN_OK) return r;
     int* status = nullptr;
@@ -870,17 +1085,27 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
         *done = true;
         return SBNN_OK;
     }
-    const long long NH = (long long)N * H;
+    // partial sums of the split tiles and their arrival counters, behind the planes of X in the scratch buffer
+    constexpr size_t slot_bytes = (size_t)C::GPW * C::RPL * C::CW * ((C::G + 1) / 2) * C::NT * sizeof(f32x2);
+    const size_t counters_off = (plan.nslots * slot_bytes + 255) / 256 * 256;
+    if (counters_off + (size_t)plan.ncounters * 4 > extra_bytes)
+        return fail(SBNN_ERR_UNSUPPORTED, "internal: 3x3 launch plan needs %zu bytes of scratch, %zu reserved",
+                    counters_off + (size_t)plan.ncounters * 4, extra_bytes);
+    f32x2* partial = reinterpret_cast<f32x2*>(extra);
+    int* counters = reinterpret_cast<int*>(extra + counters_off);
+    if (plan.ncounters) SBNN_CUDA_TRY(cudaMemsetAsync(counters, 0, (size_t)plan.ncounters * 4, st));
     Map3 xmap;
     const unsigned long long dims[3] = {(unsigned long long)W, (unsigned long long)NH, (unsigned long long)p->Cin};
     const unsigned long long strides[2] = {(unsigned long long)W * 4, (unsigned long long)ldx * 4};
     const unsigned box[3] = {(unsigned)g.pitch, (unsigned)(g.R + 2), (unsigned)C::KC};
     if ((r = encode_tiled_map(&xmap, xt, 4, 3, dims, strides, box)) != SBNN_OK) return r;
-    dim3 grid((unsigned)((NH + g.R - 1) / g.R), s.ntiles);
+    const Seg3* segs = static_cast<const Seg3*>(plan.segs);
     if (pat)
-        conv3x3_gs_tma_kernel<C, true><<<grid, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status);
+        conv3x3_gs_tma_kernel<CP, true><<<plan.ncta, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status,
+                                                                            plan.cta_ptr, segs, partial, counters);
     else
-        conv3x3_gs_tma_kernel<C, false><<<grid, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status);
+        conv3x3_gs_tma_kernel<C, false><<<plan.ncta, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status,
+                                                                             plan.cta_ptr, segs, partial, counters);
     SBNN_CUDA_TRY(cudaGetLastError());
     *done = true;
     return SBNN_OK;
@@ -888,14 +1113,26 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
 
 template <int CW>
 sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
-                          cudaStream_t st, bool* done) {
+                          cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
     switch (p->G) {
-        case 1: return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
-        case 2: return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
-        case 4: return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
-        case 8: return launch3_tma<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
-        default: return launch3_tma<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, y, N, H, W, relu, st, done);
+        case 1: return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+        case 2: return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+        case 4:
+            // two output rows per lane where the image height allows it (whole-kernel layers; the tap lists keep one)
+            if (H % 2 == 0 && p->tap_mask.empty())
+                return launch3_tma<K3<4, CW, 1, 3, 4, 8, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+        case 8: return launch3_tma<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+        default: return launch3_tma<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
     }
+}
+
+// Scratch the copy-engine kernel may need beyond the planes of X: every CTA border splits at most one tile, so there are
+// at most 2 * CTAs partial-sum slots (NT threads x GPW * CW * G sums: at most 448 * 8 * CW floats in every instance
+// above) and as many counters.
+size_t tma_extra_bytes(int cw) {
+    const size_t sms = (size_t)sm_count3();
+    return 2 * sms * (size_t)448 * 8 * cw * sizeof(float) + 256 + 2 * sms * sizeof(int);
 }
 
 template <int CW>
@@ -939,6 +1176,11 @@ void free_streams_3x3(sbnn_packed* p) {
         cudaFree(kv.second.blk_ptr);
     }
     p->streams3x3.clear();
+    for (auto& kv : p->plans3x3) {
+        cudaFree(kv.second.cta_ptr);
+        cudaFree(kv.second.segs);
+    }
+    p->plans3x3.clear();
 }
 
 }  // namespace sbnn
@@ -966,11 +1208,13 @@ extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev,
         // fast path: planes of the input ([Cin][ld]) in the per-device scratch buffer, then the cp.async kernel
         const int M = N * H * W, ld = (M + 3) / 4 * 4;
         float* xt = nullptr;
-        if ((st = scratch_workspace((size_t)w->Cin * ld * sizeof(float), s, &xt)) != SBNN_OK) return st;
+        const size_t xt_bytes = ((size_t)w->Cin * ld * sizeof(float) + 255) / 256 * 256, extra_bytes = tma_extra_bytes(cw);
+        if ((st = scratch_workspace(xt_bytes + extra_bytes, s, &xt)) != SBNN_OK) return st;
         if (!prepare_only() && (st = launch_transpose(x_dev, w->Cin, xt, ld, M, w->Cin, s)) != SBNN_OK) return st;
+        unsigned char* extra = reinterpret_cast<unsigned char*>(xt) + xt_bytes;
         bool done = false;
-        st = cw == 7 ? dispatch3_tma<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
-                     : dispatch3_tma<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);
+        st = cw == 7 ? dispatch3_tma<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
+                     : dispatch3_tma<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
         if (st != SBNN_OK || done) return st;
         st = cw == 7 ? dispatch3_cm<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
                      : dispatch3_cm<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);
