@@ -448,6 +448,24 @@ SBNN_API sbnn_status sbnn_selftest_fma_rate(int iterations, double* flop_out, vo
  * index of the device copy (the host copy and the private layouts stay as they are) and returns the previous value.
  */
 SBNN_API sbnn_status sbnn_debug_check_packed(const sbnn_packed* w, void* cuda_stream);
+
+/*
+ * Debug aid (host arithmetic only, needs no GPU; the paper has no counterpart): the work plan of the pipelined 3x3
+ * kernel behind sbnn_conv3x3_gs.  That kernel runs `ncta` persistent CTAs; the channel steps of all tiles
+ * (group tile `by` outermost, then row tile `bx`, then step k) are laid end to end and cut into `ncta` consecutive
+ * shares of equal weight, where step k of group tile `by` weighs block_ptr[by][k+1] - block_ptr[by][k] (the 16-byte
+ * words of weights it multiplies) plus a constant.  block_ptr is [ntiles][nchunks + 1], host, non-decreasing per tile.
+ * Output: cta_ptr_out [ncta + 1] (host): CTA c owns segments cta_ptr_out[c] .. cta_ptr_out[c+1]-1; segs_out (host,
+ * room for seg_capacity segments of 8 ints): {bx, by, k0, k1, part, nparts, slot, counter} -- steps [k0, k1) of tile
+ * (bx, by); a tile cut into nparts > 1 segments gets nparts consecutive partial-sum slots from `slot` and one arrival
+ * counter (each part stores its sums, the part that arrives last adds them in part order and finishes the tile).
+ * *nsegs = segments produced; *nslots, *ncounters (may be NULL) = slots and counters the plan needs.
+ * Errors: SBNN_ERR_NULL, SBNN_ERR_SHAPE (non-positive sizes, decreasing block_ptr, seg_capacity too small: *nsegs is
+ * still set), SBNN_ERR_ALLOC.
+ */
+SBNN_API sbnn_status sbnn_debug_plan_conv3x3(const int32_t* block_ptr, int ntiles, int nchunks, int nrow, int ncta,
+                                             int32_t* cta_ptr_out, int32_t* segs_out, int seg_capacity, int* nsegs,
+                                             int* nslots, int* ncounters);
 SBNN_API sbnn_status sbnn_debug_poke_device_index(sbnn_packed* w, long long unit, int value, int* previous);
 
 /*

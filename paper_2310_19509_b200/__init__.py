@@ -35,6 +35,7 @@ from .binding import (  # noqa: F401
     selftest_fma_rate,
     debug_set_packed_device,
     debug_check_packed,
+    debug_plan_conv3x3,
     debug_poke_device_index,
     selftest_wait_timeout,
     status_str,

@@ -74,6 +74,7 @@ def lib():
         "sbnn_debug_set_packed_device": [P, I, P],
         "sbnn_debug_check_packed": [P, P],
         "sbnn_debug_poke_device_index": [P, C.c_longlong, I, P],
+        "sbnn_debug_plan_conv3x3": [P, I, I, I, I, P, P, I, P, P, P],
     }
     for name, args in sig.items():
         f = getattr(L, name)
@@ -274,6 +275,20 @@ def debug_set_packed_device(w: Packed, device) -> int:
 def debug_check_packed(w: Packed, stream=None):
     """Enqueue the device-side consistency check of a packed layer (result through get_async_status)."""
     _check(lib().sbnn_debug_check_packed(w.handle, _stream(stream)))
+
+
+def debug_plan_conv3x3(block_ptr, nrow, ncta):
+    """Work plan of the pipelined 3x3 kernel for a block table [ntiles][nchunks + 1] (int32 numpy, host): returns
+    (cta_ptr [ncta + 1], segs [nsegs][8] = bx, by, k0, k1, part, nparts, slot, counter, nslots, ncounters)."""
+    bp = np.ascontiguousarray(block_ptr, dtype=np.int32)
+    ntiles, nchunks = bp.shape[0], bp.shape[1] - 1
+    cap = ntiles * nrow + 2 * ncta + 8
+    cta_ptr = np.zeros(ncta + 1, dtype=np.int32)
+    segs = np.zeros((cap, 8), dtype=np.int32)
+    nsegs, nslots, ncounters = C.c_int(), C.c_int(), C.c_int()
+    _check(lib().sbnn_debug_plan_conv3x3(bp.ctypes.data, ntiles, nchunks, int(nrow), int(ncta), cta_ptr.ctypes.data,
+                                         segs.ctypes.data, cap, C.byref(nsegs), C.byref(nslots), C.byref(ncounters)))
+    return cta_ptr, segs[:nsegs.value].copy(), nslots.value, ncounters.value
 
 
 def debug_poke_device_index(w: Packed, unit, value) -> int:

@@ -840,68 +840,83 @@ sbnn_status build_stream3_taps(const sbnn_packed* p, int GT, int KC, int plane, 
     return SBNN_OK;
 }
 
-// Deals the channel steps of a launch (row tiles x group tiles x steps, row tiles fastest) to `ncta` persistent CTAs
-// in shares of equal weight: a step weighs its weight block (16-byte words: the kept kernels or taps it multiplies) plus
+// Deals the channel steps of a launch (group tiles x row tiles x steps, steps fastest) to `ncta` persistent CTAs in
+// shares of equal weight: a step weighs its weight block (16-byte words: the kept kernels or taps it multiplies) plus
 // a constant for what every step costs (barrier round trip, list headers).  A share is cut into segments at tile
-// borders; tiles that end up in several shares get partial-sum slots and an arrival counter.
-sbnn_status build_plan3(const Stream3x3& s, int nrow, int ncta_max, Plan3x3* out) {
-    const int n = s.nchunks;
-    const long long T = (long long)nrow * s.ntiles, steps = T * n;
+// borders; tiles that end up in several shares get partial-sum slots and an arrival counter.  `blk` is the stream's
+// block table ([ntiles][nchunks + 1] offsets).  Host arithmetic only.
+struct Plan3Host {
+    std::vector<int32_t> cta_ptr;
+    std::vector<Seg3> segs;
+    int ncta = 0, nslots = 0, ncounters = 0;
+};
+void plan3_host(const int32_t* blk, int ntiles, int nchunks, int nrow, int ncta_max, Plan3Host* out) {
+    const int n = nchunks;
+    const long long T = (long long)nrow * ntiles, steps = T * n;
     const int ncta = (int)std::max<long long>(1, std::min<long long>(ncta_max, steps));
     constexpr long long kStepCost = 6;
     long long total = 0;
-    for (int by = 0; by < s.ntiles; ++by) {
-        total += ((long long)(s.blk_host[(size_t)by * (n + 1) + n] - s.blk_host[(size_t)by * (n + 1)]) + kStepCost * n) * nrow;
-    }
-    std::vector<int32_t> cta_ptr(ncta + 1, 0);
-    std::vector<Seg3> segs;
-    try {
-        long long cum = 0;
-        int cur_cta = 0;
-        for (int by = 0; by < s.ntiles; ++by) {
-            const int32_t* bp = s.blk_host.data() + (size_t)by * (n + 1);
-            for (int bx = 0; bx < nrow; ++bx) {
-                int part = 0;
-                int k = 0;
-                while (k < n) {
-                    // the CTA that owns the step starting at cumulative weight `cum`
-                    int c = total > 0 ? (int)std::min<long long>(ncta - 1, (__int128)cum * ncta / total) : 0;
-                    if (c < cur_cta) c = cur_cta;
-                    while (cur_cta < c) cta_ptr[++cur_cta] = (int32_t)segs.size();
-                    // this CTA's share ends at weight (c + 1) * total / ncta: take steps while they start below it
-                    const long long lim = (long long)(((__int128)(c + 1) * total + ncta - 1) / ncta);
-                    const int k0 = k;
-                    while (k < n && (k == k0 || cum < lim)) {
-                        cum += (long long)(bp[k + 1] - bp[k]) + kStepCost;
-                        ++k;
-                    }
-                    const Seg3 sg = {bx, by, k0, k, part++, 0, 0, 0};
-                    segs.push_back(sg);
+    for (int by = 0; by < ntiles; ++by)
+        total += ((long long)(blk[(size_t)by * (n + 1) + n] - blk[(size_t)by * (n + 1)]) + kStepCost * n) * nrow;
+    std::vector<int32_t>& cta_ptr = out->cta_ptr;
+    std::vector<Seg3>& segs = out->segs;
+    cta_ptr.assign(ncta + 1, 0);
+    segs.clear();
+    long long cum = 0;
+    int cur_cta = 0;
+    for (int by = 0; by < ntiles; ++by) {
+        const int32_t* bp = blk + (size_t)by * (n + 1);
+        for (int bx = 0; bx < nrow; ++bx) {
+            int part = 0;
+            int k = 0;
+            while (k < n) {
+                // the CTA that owns the step starting at cumulative weight `cum`
+                int c = total > 0 ? (int)std::min<long long>(ncta - 1, (long long)((__int128)cum * ncta / total)) : 0;
+                if (c < cur_cta) c = cur_cta;
+                while (cur_cta < c) cta_ptr[++cur_cta] = (int32_t)segs.size();
+                // this CTA's share ends at weight (c + 1) * total / ncta: take steps while they start below it
+                const long long lim = (long long)(((__int128)(c + 1) * total + ncta - 1) / ncta);
+                const int k0 = k;
+                while (k < n && (k == k0 || cum < lim)) {
+                    cum += (long long)(bp[k + 1] - bp[k]) + kStepCost;
+                    ++k;
                 }
-                // the tile's segments are the last `part` entries
-                for (int j = 0; j < part; ++j) segs[segs.size() - 1 - j].nparts = part;
+                const Seg3 sg = {bx, by, k0, k, part++, 0, 0, 0};
+                segs.push_back(sg);
             }
+            for (int j = 0; j < part; ++j) segs[segs.size() - 1 - j].nparts = part;   // the tile's segments are the last `part` entries
         }
-        while (cur_cta < ncta) cta_ptr[++cur_cta] = (int32_t)segs.size();
+    }
+    while (cur_cta < ncta) cta_ptr[++cur_cta] = (int32_t)segs.size();
+    out->ncta = ncta;
+    out->nslots = out->ncounters = 0;
+    for (size_t i = 0; i < segs.size(); ++i) {
+        if (segs[i].nparts > 1 && segs[i].part == 0) {
+            for (int j = 0; j < segs[i].nparts; ++j) {
+                segs[i + j].slot = out->nslots;
+                segs[i + j].counter = out->ncounters;
+            }
+            out->nslots += segs[i].nparts;
+            out->ncounters += 1;
+        }
+    }
+}
+
+sbnn_status build_plan3(const Stream3x3& s, int nrow, int ncta_max, Plan3x3* out) {
+    Plan3Host h;
+    try {
+        plan3_host(s.blk_host.data(), s.ntiles, s.nchunks, nrow, ncta_max, &h);
     } catch (const std::bad_alloc&) {
         return fail(SBNN_ERR_ALLOC, "out of host memory planning the 3x3 launch");
     }
     Plan3x3 pl;
-    pl.ncta = ncta;
-    for (size_t i = 0; i < segs.size(); ++i) {
-        if (segs[i].nparts > 1 && segs[i].part == 0) {
-            for (int j = 0; j < segs[i].nparts; ++j) {
-                segs[i + j].slot = pl.nslots;
-                segs[i + j].counter = pl.ncounters;
-            }
-            pl.nslots += segs[i].nparts;
-            pl.ncounters += 1;
-        }
-    }
-    SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&pl.cta_ptr), cta_ptr.size() * 4));
-    cudaError_t e = cudaMalloc(&pl.segs, std::max<size_t>(segs.size() * sizeof(Seg3), 32));
-    if (e == cudaSuccess) e = cudaMemcpy(pl.cta_ptr, cta_ptr.data(), cta_ptr.size() * 4, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess && !segs.empty()) e = cudaMemcpy(pl.segs, segs.data(), segs.size() * sizeof(Seg3), cudaMemcpyHostToDevice);
+    pl.ncta = h.ncta;
+    pl.nslots = h.nslots;
+    pl.ncounters = h.ncounters;
+    SBNN_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&pl.cta_ptr), h.cta_ptr.size() * 4));
+    cudaError_t e = cudaMalloc(&pl.segs, std::max<size_t>(h.segs.size() * sizeof(Seg3), 32));
+    if (e == cudaSuccess) e = cudaMemcpy(pl.cta_ptr, h.cta_ptr.data(), h.cta_ptr.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !h.segs.empty()) e = cudaMemcpy(pl.segs, h.segs.data(), h.segs.size() * sizeof(Seg3), cudaMemcpyHostToDevice);
     if (e != cudaSuccess) {
         cudaFree(pl.cta_ptr);
         cudaFree(pl.segs);
@@ -1114,13 +1129,17 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
 template <int CW>
 sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
                           cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
+    // two output rows per lane where the image height allows it (whole-kernel layers; the tap lists keep one)
+    const bool two_rows = H % 2 == 0 && p->tap_mask.empty();
     switch (p->G) {
-        case 1: return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
-        case 2: return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+        case 1:
+            if (two_rows) return launch3_tma<K3<1, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+        case 2:
+            if (two_rows) return launch3_tma<K3<2, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
         case 4:
-            // two output rows per lane where the image height allows it (whole-kernel layers; the tap lists keep one)
-            if (H % 2 == 0 && p->tap_mask.empty())
-                return launch3_tma<K3<4, CW, 1, 3, 4, 8, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+            if (two_rows) return launch3_tma<K3<4, CW, 1, 3, 4, 8, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
             return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
         case 8: return launch3_tma<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
         default: return launch3_tma<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
@@ -1222,4 +1241,31 @@ extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev,
     }
     return cw == 7 ? dispatch3<7>(w, x_dev, y_dev, N, H, W, flags & SBNN_RELU, s)
                    : dispatch3<8>(w, x_dev, y_dev, N, H, W, flags & SBNN_RELU, s);
+}
+
+extern "C" sbnn_status sbnn_debug_plan_conv3x3(const int32_t* block_ptr, int ntiles, int nchunks, int nrow, int ncta,
+                                               int32_t* cta_ptr_out, int32_t* segs_out, int seg_capacity, int* nsegs,
+                                               int* nslots, int* ncounters) {
+    clear_error();
+    if (!block_ptr || !cta_ptr_out || !segs_out || !nsegs) return fail(SBNN_ERR_NULL, "block_ptr, cta_ptr_out, segs_out and nsegs must not be NULL");
+    if (ntiles < 1 || nchunks < 1 || nrow < 1 || ncta < 1 || seg_capacity < 0) return fail(SBNN_ERR_SHAPE, "ntiles, nchunks, nrow and ncta must be positive");
+    for (int t = 0; t < ntiles; ++t)
+        for (int k = 0; k < nchunks; ++k)
+            if (block_ptr[(size_t)t * (nchunks + 1) + k + 1] < block_ptr[(size_t)t * (nchunks + 1) + k])
+                return fail(SBNN_ERR_SHAPE, "block_ptr must not decrease inside a tile");
+    Plan3Host h;
+    try {
+        plan3_host(block_ptr, ntiles, nchunks, nrow, ncta, &h);
+    } catch (const std::bad_alloc&) {
+        return fail(SBNN_ERR_ALLOC, "out of host memory planning the 3x3 launch");
+    }
+    *nsegs = (int)h.segs.size();
+    if (nslots) *nslots = h.nslots;
+    if (ncounters) *ncounters = h.ncounters;
+    if ((int)h.segs.size() > seg_capacity) return fail(SBNN_ERR_SHAPE, "%zu segments do not fit seg_capacity=%d", h.segs.size(), seg_capacity);
+    for (int c = 0; c <= h.ncta; ++c) cta_ptr_out[c] = h.cta_ptr[c];
+    for (int c = h.ncta + 1; c <= ncta; ++c) cta_ptr_out[c] = h.cta_ptr[h.ncta];
+    static_assert(sizeof(Seg3) == 8 * sizeof(int32_t), "Seg3 is eight ints");
+    if (!h.segs.empty()) memcpy(segs_out, h.segs.data(), h.segs.size() * sizeof(Seg3));
+    return SBNN_OK;
 }

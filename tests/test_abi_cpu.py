@@ -453,3 +453,64 @@ def test_paper_style_4x4_blocks_are_recognised_and_stored_with_one_index_per_blo
     p1.save(path)
     assert struct.unpack_from("<8i", open(path, "rb").read(), 8)[7] == 0
     p1.free()
+
+
+@pytest.mark.parametrize("ntiles,nchunks,nrow,ncta", [(16, 32, 16, 148), (16, 32, 19, 148), (3, 3, 1, 148), (1, 1, 1, 148),
+                                                      (11, 32, 19, 132), (5, 7, 100, 4), (2, 40, 3, 7), (4, 9, 2, 1)])
+def test_conv3x3_work_plan_covers_every_step_once_in_balanced_shares(ntiles, nchunks, nrow, ncta):
+    """The persistent 3x3 kernel's plan (host arithmetic, through the C interface): the segments, read in CTA order,
+    enumerate every (group tile, row tile, step) exactly once and in order; a CTA's weight differs from an equal share
+    by less than one step; split tiles number their parts and own consecutive slots and one counter each."""
+    rng = np.random.default_rng(ntiles * 1000 + nchunks)
+    words = rng.integers(0, 60, size=(ntiles, nchunks)).astype(np.int64)
+    words[rng.random(words.shape) < 0.1] = 0                       # steps in which the tile keeps nothing
+    bp = np.zeros((ntiles, nchunks + 1), dtype=np.int32)
+    bp[:, 1:] = np.cumsum(words, axis=1)
+    bp += (np.arange(ntiles, dtype=np.int32) * 5000)[:, None]       # tiles follow one another in the stream
+    cta_ptr, segs, nslots, ncounters = sbnn.debug_plan_conv3x3(bp, nrow, ncta)
+    steps = ntiles * nrow * nchunks
+    ncta_eff = min(ncta, steps)
+    assert cta_ptr[0] == 0 and np.all(np.diff(cta_ptr) >= 0) and cta_ptr[-1] == len(segs)
+    # coverage and order
+    pos = 0                                                         # next step expected, in (by, bx, k) order
+    for bx, by, k0, k1, part, nparts, slot, counter in segs:
+        assert k1 > k0
+        assert pos == (by * nrow + bx) * nchunks + k0
+        assert (part == 0) == (k0 == 0)
+        pos += k1 - k0
+    assert pos == steps
+    # parts, slots, counters
+    by_tile = {}
+    for i, sg in enumerate(segs):
+        by_tile.setdefault((sg[1], sg[0]), []).append(sg)
+    seen_slots, seen_counters = set(), set()
+    for parts in by_tile.values():
+        n = len(parts)
+        assert [int(sg[4]) for sg in parts] == list(range(n)) and all(sg[5] == n for sg in parts)
+        assert parts[-1][3] == nchunks
+        if n > 1:
+            assert len({int(sg[6]) for sg in parts}) == 1 and len({int(sg[7]) for sg in parts}) == 1
+            slots = set(range(int(parts[0][6]), int(parts[0][6]) + n))
+            assert not (slots & seen_slots) and int(parts[0][7]) not in seen_counters
+            seen_slots |= slots
+            seen_counters.add(int(parts[0][7]))
+    assert seen_slots == set(range(nslots)) and seen_counters == set(range(ncounters))
+    assert nslots <= 2 * ncta_eff
+    # balance: weight of a step = its words + 6
+    weight = words + 6
+    total = int(weight.sum()) * nrow
+    share = total / ncta_eff
+    heaviest = int(weight.max())
+    for c in range(ncta_eff):
+        wc = sum(int(weight[sg[1], sg[2]:sg[3]].sum()) for sg in segs[cta_ptr[c]:cta_ptr[c + 1]])
+        assert abs(wc - share) < heaviest + 1, (c, wc, share)
+    # CTAs beyond the number of steps own nothing
+    assert np.all(cta_ptr[ncta_eff:] == len(segs))
+
+
+def test_conv3x3_work_plan_errors():
+    bp = np.array([[0, 4, 2]], dtype=np.int32)                      # decreasing
+    with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_SHAPE"):
+        sbnn.debug_plan_conv3x3(bp, 1, 4)
+    with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_SHAPE"):
+        sbnn.debug_plan_conv3x3(np.array([[0, 4, 8]], dtype=np.int32), 0, 4)

@@ -461,6 +461,29 @@ def test_3x3_shapes_and_groups(g, hw):
         assert_within(y, ref, s, what=f"3x3 G={g} {hw} relu={relu}")
 
 
+@pytest.mark.parametrize("g,n,h,w,cin,cout", [(4, 40, 14, 28, 64, 64), (4, 9, 7, 28, 40, 96), (8, 12, 14, 28, 64, 128),
+                                               (2, 30, 8, 56, 32, 24), (1, 20, 10, 28, 24, 40), (16, 6, 28, 28, 48, 64),
+                                               (4, 200, 14, 28, 16, 32)])
+def test_3x3_tiles_split_between_persistent_ctas(g, n, h, w, cin, cout):
+    """The pipelined 3x3 kernel deals the channel steps of all tiles to one CTA per SM in equal shares.  Shapes with
+    a few steps per CTA (every tile cut into several parts whose partial sums the last arrival adds), with about as
+    many tiles as CTAs (tiles cut in two) and with many more tiles than CTAs (most tiles whole); even heights run two
+    output rows per lane (G <= 4), odd heights and wider groups one.  Every output against the oracle."""
+    d = WL.single_conv_inputs(n, h, w, cin, cout, 3, g, 50, seed=21, w_sigma=0.05)
+    for relu in (True, False):
+        y = run_3x3(d, sbnn.SBNN_RELU if relu else 0)
+        ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
+        assert_within(y, ref, s, what=f"3x3 split tiles G={g} n={n} {h}x{w} {cin}->{cout} relu={relu}")
+
+
+def test_3x3_same_result_on_every_run():
+    """Split tiles are added in part order whichever part arrives last: two runs agree bit for bit."""
+    d = WL.single_conv_inputs(40, 14, 28, 64, 64, 3, 4, 50, seed=22, w_sigma=0.05)
+    y0 = run_3x3(d)
+    for _ in range(3):
+        assert np.array_equal(run_3x3(d), y0)
+
+
 @pytest.mark.parametrize("g,kept_taps", [(4, 4), (2, 4), (8, 6), (1, 1)])
 def test_3x3_kernel_patterns(g, kept_taps):
     """Kernels pruned tap by tap (centre + kept_taps - 1 others, one pattern per group and input channel, packed by
