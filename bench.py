@@ -239,7 +239,8 @@ def time_layers_in_chain(sbnn, torch, net, layers, batch, xd, reps):
             runs.append(ev0.elapsed_time(ev1) * 1e-3 / reps)
         prefix.append(float(np.median(runs)))
         del g
-    return [max(prefix[0], 0.0)] + [max(prefix[l] - prefix[l - 1], 0.0) for l in range(1, len(layers))]
+    # (a difference can come out at or below zero when timing noise exceeds a very short layer: floor of 10 ns)
+    return [max(prefix[0], 1e-8)] + [max(prefix[l] - prefix[l - 1], 1e-8) for l in range(1, len(layers))]
 
 
 def sweep_oracle_lines():
