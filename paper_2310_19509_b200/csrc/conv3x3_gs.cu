@@ -23,6 +23,7 @@
 
 #include "common.h"
 #include "pipeline.cuh"
+#include "shares.h"
 
 namespace sbnn {
 namespace {
@@ -840,66 +841,33 @@ sbnn_status build_stream3_taps(const sbnn_packed* p, int GT, int KC, int plane, 
     return SBNN_OK;
 }
 
-// Deals the channel steps of a launch (group tiles x row tiles x steps, steps fastest) to `ncta` persistent CTAs in
-// shares of equal weight: a step weighs its weight block (16-byte words: the kept kernels or taps it multiplies) plus
-// a constant for what every step costs (barrier round trip, list headers).  A share is cut into segments at tile
-// borders; tiles that end up in several shares get partial-sum slots and an arrival counter.  `blk` is the stream's
-// block table ([ntiles][nchunks + 1] offsets).  Host arithmetic only.
+// The launch's work plan (shares.h): the tile sequence is group tile (outermost), row tile; a step weighs its weight
+// block (16-byte words: the kept kernels or taps it multiplies) plus a constant for what every step costs (barrier
+// round trip, list headers).  `blk` is the stream's block table ([ntiles][nchunks + 1] offsets).  Host arithmetic only.
 struct Plan3Host {
     std::vector<int32_t> cta_ptr;
     std::vector<Seg3> segs;
     int ncta = 0, nslots = 0, ncounters = 0;
 };
 void plan3_host(const int32_t* blk, int ntiles, int nchunks, int nrow, int ncta_max, Plan3Host* out) {
-    const int n = nchunks;
-    const long long T = (long long)nrow * ntiles, steps = T * n;
-    const int ncta = (int)std::max<long long>(1, std::min<long long>(ncta_max, steps));
     constexpr long long kStepCost = 6;
-    long long total = 0;
-    for (int by = 0; by < ntiles; ++by)
-        total += ((long long)(blk[(size_t)by * (n + 1) + n] - blk[(size_t)by * (n + 1)]) + kStepCost * n) * nrow;
-    std::vector<int32_t>& cta_ptr = out->cta_ptr;
-    std::vector<Seg3>& segs = out->segs;
-    cta_ptr.assign(ncta + 1, 0);
-    segs.clear();
-    long long cum = 0;
-    int cur_cta = 0;
-    for (int by = 0; by < ntiles; ++by) {
-        const int32_t* bp = blk + (size_t)by * (n + 1);
-        for (int bx = 0; bx < nrow; ++bx) {
-            int part = 0;
-            int k = 0;
-            while (k < n) {
-                // the CTA that owns the step starting at cumulative weight `cum`
-                int c = total > 0 ? (int)std::min<long long>(ncta - 1, (long long)((__int128)cum * ncta / total)) : 0;
-                if (c < cur_cta) c = cur_cta;
-                while (cur_cta < c) cta_ptr[++cur_cta] = (int32_t)segs.size();
-                // this CTA's share ends at weight (c + 1) * total / ncta: take steps while they start below it
-                const long long lim = (long long)(((__int128)(c + 1) * total + ncta - 1) / ncta);
-                const int k0 = k;
-                while (k < n && (k == k0 || cum < lim)) {
-                    cum += (long long)(bp[k + 1] - bp[k]) + kStepCost;
-                    ++k;
-                }
-                const Seg3 sg = {bx, by, k0, k, part++, 0, 0, 0};
-                segs.push_back(sg);
-            }
-            for (int j = 0; j < part; ++j) segs[segs.size() - 1 - j].nparts = part;   // the tile's segments are the last `part` entries
-        }
+    SharePlan sp;
+    // the launch's tile sequence: group tile by = tile / nrow outermost, row tile bx = tile % nrow
+    plan_shares((long long)ntiles * nrow, nchunks,
+                [&](long long tile, int k) {
+                    const int32_t* bp = blk + (size_t)(tile / nrow) * (nchunks + 1);
+                    return (long long)(bp[k + 1] - bp[k]) + kStepCost;
+                },
+                ncta_max, &sp);
+    out->cta_ptr = std::move(sp.cta_ptr);
+    out->segs.resize(sp.segs.size());
+    for (size_t i = 0; i < sp.segs.size(); ++i) {
+        const ShareSeg& g = sp.segs[i];
+        out->segs[i] = Seg3{g.tile % nrow, g.tile / nrow, g.k0, g.k1, g.part, g.nparts, g.slot, g.counter};
     }
-    while (cur_cta < ncta) cta_ptr[++cur_cta] = (int32_t)segs.size();
-    out->ncta = ncta;
-    out->nslots = out->ncounters = 0;
-    for (size_t i = 0; i < segs.size(); ++i) {
-        if (segs[i].nparts > 1 && segs[i].part == 0) {
-            for (int j = 0; j < segs[i].nparts; ++j) {
-                segs[i + j].slot = out->nslots;
-                segs[i + j].counter = out->ncounters;
-            }
-            out->nslots += segs[i].nparts;
-            out->ncounters += 1;
-        }
-    }
+    out->ncta = sp.ncta;
+    out->nslots = sp.nslots;
+    out->ncounters = sp.ncounters;
 }
 
 sbnn_status build_plan3(const Stream3x3& s, int nrow, int ncta_max, Plan3x3* out) {
