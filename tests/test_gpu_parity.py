@@ -463,12 +463,13 @@ def test_3x3_shapes_and_groups(g, hw):
 
 @pytest.mark.parametrize("g,n,h,w,cin,cout", [(4, 40, 14, 28, 64, 64), (4, 9, 7, 28, 40, 96), (8, 12, 14, 28, 64, 128),
                                                (2, 30, 8, 56, 32, 24), (1, 20, 10, 28, 24, 40), (16, 6, 28, 28, 48, 64),
-                                               (4, 200, 14, 28, 16, 32)])
+                                               (4, 200, 14, 28, 16, 32), (4, 20, 14, 28, 40, 72), (4, 3, 56, 56, 24, 120)])
 def test_3x3_tiles_split_between_persistent_ctas(g, n, h, w, cin, cout):
     """The pipelined 3x3 kernel deals the channel steps of all tiles to one CTA per SM in equal shares.  Shapes with
     a few steps per CTA (every tile cut into several parts whose partial sums the last arrival adds), with about as
     many tiles as CTAs (tiles cut in two) and with many more tiles than CTAs (most tiles whole); even heights run two
-    output rows per lane (G <= 4), odd heights and wider groups one.  Every output against the oracle."""
+    output rows per lane (G <= 4; both tile shapes of G = 4: 3 x 4 warps with 8-channel steps, 2 x 6 warps with 16-channel
+    steps where the group count suits tiles of six), odd heights and wider groups one.  Every output against the oracle."""
     d = WL.single_conv_inputs(n, h, w, cin, cout, 3, g, 50, seed=21, w_sigma=0.05)
     for relu in (True, False):
         y = run_3x3(d, sbnn.SBNN_RELU if relu else 0)
