@@ -348,6 +348,16 @@ def single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, reps):
             rec["us_channel_major"] = round(tc * 1e6, 1)
             rec["frac_channel_major"] = round(max(t_alu, t_hbm) / tc, 3)
             del xt, yt
+        if k == 3 and w % 4 == 0:
+            # the 3x3 layer in the kernel's own layout (channel-major in and out): no conversion pass
+            ld = (m + 3) // 4 * 4
+            xt, yt = torch.empty((cin, ld), device="cuda"), torch.empty((cout, ld), device="cuda")
+            sbnn.to_channel_major(xd, xt, m, cin, ld)
+            tc = _time_fn(torch, lambda: sbnn.conv3x3_gs_cm(p, xt, ld, yt, ld, n, h, w, flags | sbnn.SBNN_OUT_CM), reps, flush)
+            sbnn.get_async_status()
+            rec["us_channel_major"] = round(tc * 1e6, 1)
+            rec["frac_channel_major"] = round(max(t_alu, t_hbm) / tc, 3)
+            del xt, yt
         key = (m, cin, cout, k)
         if key not in dense:
             dense[key] = dense_library_us(torch, m, cin, cout, k, (n, h, w), max(3, reps // 2), flush)

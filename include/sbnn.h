@@ -244,6 +244,21 @@ SBNN_API sbnn_status sbnn_to_channel_major(const float* x_dev, float* xt_dev, in
 SBNN_API sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev, float* y_dev,
                                      int N, int H, int W, int flags, void* cuda_stream);
 
+/*
+ * Channel-major variant of the 3x3 convolution (same arithmetic): the activations are given as xt_dev [Cin][ldx] with
+ * the M = N*H*W pixels of a channel contiguous in (n, y, x) order (ldx >= M, a multiple of 4; the padding need not be
+ * initialised) -- the layout sbnn_conv1x1_gs_cm reads and, with SBNN_OUT_CM, writes, so 1x1 and 3x3 layers chain
+ * without a conversion pass.  This is the layout the pipelined 3x3 kernel stages from; sbnn_conv3x3_gs converts to it first.
+ *   output: y_dev [M][ldy] (pixel-major rows of ldy >= Cout floats, ldy a multiple of 4), or, with SBNN_OUT_CM,
+ *   [Cout][ldy] with ldy >= M.
+ *   flags: SBNN_RELU, SBNN_OUT_CM.
+ * W a multiple of 4 and at most 256, Cin a multiple of 4, else SBNN_ERR_UNSUPPORTED.  The partial sums of tiles that
+ * are shared between CTAs live in the per-device scratch buffer (see sbnn_conv1x1_gs_cm for its rules); the first call
+ * with a new width builds a private re-layout of the weights and a work plan (allocates and copies synchronously).
+ */
+SBNN_API sbnn_status sbnn_conv3x3_gs_cm(const sbnn_packed* w, const float* xt_dev, int ldx, float* y_dev, int ldy,
+                                        int N, int H, int W, int flags, void* cuda_stream);
+
 /* ------------------------------------------------------------------------------------------------
  * Dense supporting layers of MobileNet-v1 (Section 3.2 names the operators; they stay dense here).
  * ------------------------------------------------------------------------------------------------ */

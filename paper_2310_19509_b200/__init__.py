@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     conv1x1_gs_tuned,
     conv3x3_dense,
     conv3x3_gs,
+    conv3x3_gs_cm,
     dwconv3x3,
     dwconv3x3_cm,
     dwconv3x3_conv1x1_gs_cm,

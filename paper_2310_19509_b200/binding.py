@@ -50,6 +50,7 @@ def lib():
         "sbnn_conv1x1_gs": [P, P, P, I, I, I, I, P],
         "sbnn_conv1x1_gs_tuned": [P, P, P, I, I, I, I, I, I, I, I, P],
         "sbnn_conv3x3_gs": [P, P, P, I, I, I, I, P],
+        "sbnn_conv3x3_gs_cm": [P, P, I, P, I, I, I, I, I, P],
         "sbnn_conv1x1_gs_cm": [P, P, I, P, I, I, I, I, I, I, I, P],
         "sbnn_to_channel_major": [P, P, I, I, I, P],
         "sbnn_dwconv3x3": [P, P, P, P, I, I, I, I, I, I, P],
@@ -205,6 +206,10 @@ def to_channel_major(x, xt, m, c, ld, stream=None):
 
 def conv3x3_gs(w: Packed, x, y, n, h, wd, flags=SBNN_RELU, stream=None):
     _check(lib().sbnn_conv3x3_gs(w.handle, _ptr(x), _ptr(y), n, h, wd, flags, _stream(stream)))
+
+
+def conv3x3_gs_cm(w: Packed, xt, ldx, y, ldy, n, h, wd, flags=SBNN_RELU, stream=None):
+    _check(lib().sbnn_conv3x3_gs_cm(w.handle, _ptr(xt), ldx, _ptr(y), ldy, n, h, wd, flags, _stream(stream)))
 
 
 def dwconv3x3(w, b, x, y, n, h, wd, c, stride, flags=SBNN_RELU, stream=None):

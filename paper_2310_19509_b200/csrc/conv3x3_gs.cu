@@ -388,12 +388,12 @@ __device__ __forceinline__ void compute_warps_barrier(int nthreads) {
     asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
 }
 
-template <class C, bool PAT>
+template <class C, bool PAT, bool OUT_CM = false>
 __global__ void __launch_bounds__(C::NT + 32, 1)
 conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, const float* __restrict__ bias,
                       const uint4* __restrict__ rec, const int32_t* __restrict__ blk_ptr, Geo3 geo, int relu, int S,
                       int stage_bytes, int* status, const int32_t* __restrict__ cta_ptr, const Seg3* __restrict__ segs,
-                      f32x2* partial, int* counters) {
+                      f32x2* partial, int* counters, int ldy) {
     constexpr int G = C::G, CW = C::CW, GPW = C::GPW, KC = C::KC, NW = C::NW, RPL = C::RPL;
     constexpr int GP = (G + 1) / 2;
     static_assert(!PAT || RPL == 1, "the tap lists address one output row per lane");
@@ -651,7 +651,6 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
             for (int p = 0; p < CW; ++p) {
                 const int x = lx + p;
                 if (x >= W || f + ro >= NH) continue;
-                float* yp = Y + ((size_t)(f + ro) * W + x) * geo.Cout + g * G;
                 float v[2 * GP];
 #pragma unroll
                 for (int rr = 0; rr < GP; ++rr) unpack2(acc[q][ro][p][rr], v[2 * rr], v[2 * rr + 1]);
@@ -659,6 +658,12 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
 #pragma unroll
                     for (int rr = 0; rr < 2 * GP; ++rr) v[rr] = fmaxf(v[rr], 0.0f);
                 }
+                if constexpr (OUT_CM) {                             // [Cout][ldy]: a lane's CW columns are a contiguous run
+#pragma unroll
+                    for (int rr = 0; rr < G; ++rr) Y[(size_t)(g * G + rr) * ldy + (size_t)(f + ro) * W + x] = v[rr];
+                    continue;
+                }
+                float* yp = Y + ((size_t)(f + ro) * W + x) * ldy + g * G;
                 if constexpr (G >= 4) {
 #pragma unroll
                     for (int vv = 0; vv < G / 4; ++vv)
@@ -1005,8 +1010,8 @@ sbnn_status launch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y,
 
 // Launches the copy-engine variant; *done = false (and SBNN_OK) if the shape does not fit it.
 template <class C>
-sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
-                        cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
+sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int ldy, bool out_cm, int N, int H, int W,
+                        int relu, cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
     *done = false;
     Geo3 g;
     g.N = N; g.H = H; g.W = W; g.Cin = p->Cin; g.Cout = p->Cout; g.ngroups = p->ngroups;
@@ -1059,8 +1064,11 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     constexpr bool kTapLists = C::RPL == 1;                        // instances with several rows per lane have no tap-list form
     if (pat && !kTapLists) return SBNN_OK;
     using CP = K3<C::G, C::CW, C::GPW, C::NPW, C::NGW, C::KC, 1>;  // == C wherever the tap-list kernel is launched
-    sbnn_status r = set_max_dyn_smem(pat ? reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<CP, true>)
-                                         : reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C, false>), (int)smem);
+    sbnn_status r = set_max_dyn_smem(pat ? reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<CP, true, false>)
+                                         : reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C, false, false>), (int)smem);
+    if (r == SBNN_OK)
+        r = set_max_dyn_smem(pat ? reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<CP, true, true>)
+                                 : reinterpret_cast<const void*>(&conv3x3_gs_tma_kernel<C, false, true>), (int)smem);
     if (r != SBNN_OK) return r;
     int* status = nullptr;
     if ((r = async_status_word(&status)) != SBNN_OK) return r;
@@ -1083,29 +1091,33 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     const unsigned box[3] = {(unsigned)g.pitch, (unsigned)(g.R + 2), (unsigned)C::KC};
     if ((r = encode_tiled_map(&xmap, xt, 4, 3, dims, strides, box)) != SBNN_OK) return r;
     const Seg3* segs = static_cast<const Seg3*>(plan.segs);
-    if (pat)
-        conv3x3_gs_tma_kernel<CP, true><<<plan.ncta, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status,
-                                                                            plan.cta_ptr, segs, partial, counters);
-    else
-        conv3x3_gs_tma_kernel<C, false><<<plan.ncta, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, stage_bytes, status,
-                                                                             plan.cta_ptr, segs, partial, counters);
+#define SBNN_L3(KCFG, PATF, CMF)                                                                                              \
+    conv3x3_gs_tma_kernel<KCFG, PATF, CMF><<<plan.ncta, C::NT + 32, smem, st>>>(xmap, y, p->d_bias, s.rec, s.blk_ptr, g, relu, S, \
+                                                                               stage_bytes, status, plan.cta_ptr, segs, partial, \
+                                                                               counters, ldy)
+    if (pat) {
+        if (out_cm) SBNN_L3(CP, true, true); else SBNN_L3(CP, true, false);
+    } else {
+        if (out_cm) SBNN_L3(C, false, true); else SBNN_L3(C, false, false);
+    }
+#undef SBNN_L3
     SBNN_CUDA_TRY(cudaGetLastError());
     *done = true;
     return SBNN_OK;
 }
 
 template <int CW>
-sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int N, int H, int W, int relu,
-                          cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
+sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int ldy, bool out_cm, int N, int H, int W,
+                          int relu, cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
     // two output rows per lane where the image height allows it (whole-kernel layers; the tap lists keep one)
     const bool two_rows = H % 2 == 0 && p->tap_mask.empty();
     switch (p->G) {
         case 1:
-            if (two_rows) return launch3_tma<K3<1, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
-            return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+            if (two_rows) return launch3_tma<K3<1, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
         case 2:
-            if (two_rows) return launch3_tma<K3<2, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
-            return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+            if (two_rows) return launch3_tma<K3<2, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
         case 4:
             if (two_rows) {
                 // 2 row warps x 6 group warps with 16-channel steps is about 6 % faster per group than 3 x 4 with
@@ -1113,14 +1125,14 @@ sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float*
                 // mostly empty.  Falls back to 3 x 4 when two stages of the larger tile do not fit.
                 const int ng = p->ngroups;
                 if ((ng + 5) / 6 * 6 * 0.94 < (ng + 3) / 4 * 4) {
-                    sbnn_status r = launch3_tma<K3<4, CW, 1, 2, 6, 16, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+                    sbnn_status r = launch3_tma<K3<4, CW, 1, 2, 6, 16, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
                     if (r != SBNN_OK || *done) return r;
                 }
-                return launch3_tma<K3<4, CW, 1, 3, 4, 8, 2>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+                return launch3_tma<K3<4, CW, 1, 3, 4, 8, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
             }
-            return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
-        case 8: return launch3_tma<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
-        default: return launch3_tma<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, y, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+        case 8: return launch3_tma<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+        default: return launch3_tma<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
     }
 }
 
@@ -1210,8 +1222,8 @@ extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev,
         if (!prepare_only() && (st = launch_transpose(x_dev, w->Cin, xt, ld, M, w->Cin, s)) != SBNN_OK) return st;
         unsigned char* extra = reinterpret_cast<unsigned char*>(xt) + xt_bytes;
         bool done = false;
-        st = cw == 7 ? dispatch3_tma<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
-                     : dispatch3_tma<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
+        st = cw == 7 ? dispatch3_tma<7>(w, xt, ld, y_dev, w->Cout, false, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
+                     : dispatch3_tma<8>(w, xt, ld, y_dev, w->Cout, false, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
         if (st != SBNN_OK || done) return st;
         st = cw == 7 ? dispatch3_cm<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
                      : dispatch3_cm<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);
@@ -1246,4 +1258,37 @@ extern "C" sbnn_status sbnn_debug_plan_conv3x3(const int32_t* block_ptr, int nti
     static_assert(sizeof(Seg3) == 8 * sizeof(int32_t), "Seg3 is eight ints");
     if (!h.segs.empty()) memcpy(segs_out, h.segs.data(), h.segs.size() * sizeof(Seg3));
     return SBNN_OK;
+}
+
+extern "C" sbnn_status sbnn_conv3x3_gs_cm(const sbnn_packed* w, const float* xt_dev, int ldx, float* y_dev, int ldy, int N, int H,
+                                          int W, int flags, void* cuda_stream) {
+    clear_error();
+    if (!w || !xt_dev || !y_dev) return fail(SBNN_ERR_NULL, "packed weights, xt_dev and y_dev must not be NULL");
+    if (w->KH != 3 || w->KW != 3) return fail(SBNN_ERR_SHAPE, "packed layer is %dx%d, expected 3x3", w->KH, w->KW);
+    if (N < 0 || H < 0 || W < 0) return fail(SBNN_ERR_SHAPE, "negative activation shape %dx%dx%d", N, H, W);
+    if ((int64_t)N * H * W > 0x7fffffff) return fail(SBNN_ERR_SHAPE, "N*H*W exceeds 2^31-1");
+    if (flags & ~(SBNN_RELU | SBNN_OUT_CM)) return fail(SBNN_ERR_UNSUPPORTED, "flag bits 0x%x not accepted here", flags);
+    const bool out_cm = (flags & SBNN_OUT_CM) != 0;
+    const long long M = (long long)N * H * W;
+    if (ldx < M || ldx % 4) return fail(SBNN_ERR_SHAPE, "ldx=%d must be >= N*H*W=%lld and a multiple of 4", ldx, M);
+    if (out_cm ? (ldy < M) : (ldy < w->Cout || ldy % 4))
+        return fail(SBNN_ERR_SHAPE, "ldy=%d does not fit the output layout", ldy);
+    if (!aligned16(xt_dev) || !aligned16(y_dev)) return fail(SBNN_ERR_ALIGN, "xt_dev and y_dev must be 16-byte aligned");
+    if (w->Cin % 4) return fail(SBNN_ERR_UNSUPPORTED, "Cin=%d is not a multiple of 4", w->Cin);
+    if (M == 0) return SBNN_OK;
+    const int cw = choose_cw(W);
+    if (!cw || W % 4) return fail(SBNN_ERR_UNSUPPORTED, "W=%d: the channel-major 3x3 kernel takes widths divisible by 4, at most 256", W);
+    sbnn_status st = check_packed_device(w);
+    if (st != SBNN_OK) return st;
+    if ((st = check_device()) != SBNN_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    float* scratch = nullptr;
+    const size_t extra_bytes = tma_extra_bytes(cw);
+    if ((st = scratch_workspace(extra_bytes, s, &scratch)) != SBNN_OK) return st;
+    bool done = false;
+    unsigned char* extra = reinterpret_cast<unsigned char*>(scratch);
+    st = cw == 7 ? dispatch3_tma<7>(w, xt_dev, ldx, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
+                 : dispatch3_tma<8>(w, xt_dev, ldx, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
+    if (st != SBNN_OK || done) return st;
+    return fail(SBNN_ERR_UNSUPPORTED, "the pipelined 3x3 kernel does not take this shape (rows of %d pixels)", W);
 }

@@ -477,6 +477,46 @@ def test_3x3_tiles_split_between_persistent_ctas(g, n, h, w, cin, cout):
         assert_within(y, ref, s, what=f"3x3 split tiles G={g} n={n} {h}x{w} {cin}->{cout} relu={relu}")
 
 
+@pytest.mark.parametrize("g,n,h,w,cin,cout", [(4, 3, 28, 28, 256, 256), (4, 5, 14, 28, 40, 72), (8, 4, 7, 28, 32, 64),
+                                               (2, 3, 8, 56, 24, 20), (16, 2, 6, 100, 20, 48), (1, 2, 10, 12, 8, 7)])
+def test_3x3_channel_major_entry(g, n, h, w, cin, cout):
+    """sbnn_conv3x3_gs_cm: activations given as channel-major planes (the layout the pipelined kernel stages from, no
+    conversion pass), output pixel-major or, with SBNN_OUT_CM, channel-major with a padded leading dimension whose
+    padding must stay untouched.  Every output against the oracle; both agree bit for bit with each other."""
+    d = WL.single_conv_inputs(n, h, w, cin, cout, 3, g, 50, seed=31, w_sigma=0.05)
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], g)
+    m = n * h * w
+    ld = (m + 3) // 4 * 4 + 8
+    xt = torch.full((cin, ld), float("nan"), device="cuda")
+    sbnn.to_channel_major(dev(d["x"]), xt, m, cin, ld)
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    ldy = (cout + 3) // 4 * 4
+    y_pm = torch.full((m, ldy), float("nan"), device="cuda")
+    sbnn.conv3x3_gs_cm(p, xt, ld, y_pm, ldy, n, h, w, sbnn.SBNN_RELU)
+    sbnn.get_async_status()
+    got = y_pm[:, :cout].cpu().numpy().reshape(n, h, w, cout)
+    assert_within(got, ref, s, what=f"3x3 channel-major in, pixel-major out G={g}")
+    assert torch.isnan(y_pm[:, cout:]).all()
+    y_cm = torch.full((cout, ld), float("nan"), device="cuda")
+    sbnn.conv3x3_gs_cm(p, xt, ld, y_cm, ld, n, h, w, sbnn.SBNN_RELU | sbnn.SBNN_OUT_CM)
+    sbnn.get_async_status()
+    assert torch.isnan(y_cm[:, m:]).all()
+    assert torch.equal(y_cm[:, :m].t().contiguous(), y_pm[:, :cout].contiguous())
+    p.free()
+
+
+def test_3x3_channel_major_entry_refuses_what_it_cannot_run():
+    d = WL.single_conv_inputs(1, 6, 6, 8, 8, 3, 4, 50, seed=32)
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    xt = torch.zeros((8, 40), device="cuda")
+    y = torch.zeros((36, 8), device="cuda")
+    with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_UNSUPPORTED"):      # W = 6 is not a multiple of 4
+        sbnn.conv3x3_gs_cm(p, xt, 40, y, 8, 1, 6, 6, sbnn.SBNN_RELU)
+    with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_SHAPE"):            # ldx < M
+        sbnn.conv3x3_gs_cm(p, xt, 32, y, 8, 1, 6, 6, sbnn.SBNN_RELU)
+    p.free()
+
+
 def test_3x3_same_result_on_every_run():
     """Split tiles are added in part order whichever part arrives last: two runs agree bit for bit."""
     d = WL.single_conv_inputs(40, 14, 28, 64, 64, 3, 4, 50, seed=22, w_sigma=0.05)
