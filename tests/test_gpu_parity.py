@@ -505,6 +505,33 @@ def test_3x3_channel_major_entry(g, n, h, w, cin, cout):
     p.free()
 
 
+def test_bottleneck_block_chained_in_channel_major_layout():
+    """1x1 (256 -> 64) -> 3x3 (64 -> 64) -> 1x1 (64 -> 256), all group-sparse (G = 4, 50 %), chained on the device in the
+    channel-major layout with no conversion between the layers.  Each layer is checked against the oracle applied to
+    the activations the previous GPU layer produced (so a layer's tolerance is its own, not a propagated one)."""
+    n, h, w = 6, 28, 28
+    m = n * h * w
+    ld = (m + 3) // 4 * 4
+    shapes = [(256, 64, 1), (64, 64, 3), (64, 256, 1)]
+    layers = [WL.single_conv_inputs(n, h, w, ci, co, k, 4, 50, seed=40 + i, w_sigma=0.05, layer=i) for i, (ci, co, k) in enumerate(shapes)]
+    packed = [sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4) for d in layers]
+    xt = torch.full((256, ld), float("nan"), device="cuda")
+    sbnn.to_channel_major(dev(layers[0]["x"]), xt, m, 256, ld)
+    acts = [xt] + [torch.full((co, ld), float("nan"), device="cuda") for _, co, _ in shapes]
+    fl = sbnn.SBNN_RELU | sbnn.SBNN_OUT_CM
+    sbnn.conv1x1_gs_cm(packed[0], acts[0], ld, acts[1], ld, m, fl)
+    sbnn.conv3x3_gs_cm(packed[1], acts[1], ld, acts[2], ld, n, h, w, fl)
+    sbnn.conv1x1_gs_cm(packed[2], acts[2], ld, acts[3], ld, m, fl)
+    sbnn.get_async_status()
+    host = [a[:, :m].t().contiguous().cpu().numpy() for a in acts]       # [m][C] each
+    for i, (d, (ci, co, k)) in enumerate(zip(layers, shapes)):
+        xin = host[i].reshape(n, h, w, ci)
+        ref, s = R.conv2d(xin, d["w"], d["mask"], d["bias"], relu=True)
+        assert_within(host[i + 1].reshape(n, h, w, co), ref, s, what=f"bottleneck layer {i} ({k}x{k}, {ci} -> {co})")
+    for p in packed:
+        p.free()
+
+
 def test_3x3_channel_major_entry_refuses_what_it_cannot_run():
     d = WL.single_conv_inputs(1, 6, 6, 8, 8, 3, 4, 50, seed=32)
     p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
