@@ -898,6 +898,30 @@ def test_prepare_then_calls_only_enqueue_and_capture_refuses_to_grow_the_scratch
     p.free()
 
 
+def test_3x3_prepared_call_is_captured_and_replayed():
+    """After sbnn_prepare for the shape (weight stream, work plan, scratch), a 3x3 call on a new width is recorded into a
+    CUDA graph (conversion pass, clearing of the arrival counters, the persistent kernel) without allocating, and two
+    replays give the oracle's result both times (the counters are cleared inside the graph)."""
+    d = WL.single_conv_inputs(7, 12, 44, 24, 40, 3, 4, 50, seed=23, w_sigma=0.05)
+    n, h, w, _ = d["x"].shape
+    p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
+    sbnn.prepare(p, n, h, w)
+    xd = dev(d["x"])
+    out = Guarded((n, h, w, 40))
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        sbnn.conv3x3_gs(p, xd, out.t, n, h, w, sbnn.SBNN_RELU, stream=torch.cuda.current_stream())
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=True)
+    for _ in range(2):
+        out.t.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        sbnn.get_async_status()
+        assert_within(out.numpy("captured 3x3"), ref, s, what="3x3 graph replay after sbnn_prepare")
+    p.free()
+
+
 def test_few_pixel_kernel_on_a_layer_without_kept_units():
     """Every unit pruned: the few-pixel kernel's look-ahead fetch has no unit to read; the output is act(bias)."""
     d = WL.single_conv_inputs(1, 3, 5, 40, 24, 1, 4, 100, seed=10)
