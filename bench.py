@@ -318,20 +318,24 @@ def single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, reps):
     from sbnn_inputs import workloads as WL
     out, dense = [], {}
 
-    def one(name, d, k, flags, mode):
+    def one(name, d, k, flags, mode, tap_mask=None):
         x = d["x"]
         n, h, w, cin = x.shape
         cout, g = d["w"].shape[0], d["g"]
         m = n * h * w
-        p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], g)
+        if tap_mask is not None:     # kernels pruned tap by tap on top of the unit mask (packed with their patterns)
+            p = sbnn.pack_weights(d["w"], tap_mask, d["bias"], g, tap_patterns=True)
+        else:
+            p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], g)
         xd = torch.from_numpy(x).cuda()
         yd = torch.empty((n, h, w, cout), device="cuda")
         fn = (lambda: sbnn.conv3x3_gs(p, xd, yd, n, h, w, flags)) if k == 3 else (lambda: sbnn.conv1x1_gs(p, xd, yd, n, h, w, flags))
         t = _time_fn(torch, fn, reps, flush)
         sbnn.get_async_status()
         units = int(d["unit_mask"].sum())
-        flops = 2.0 * m * g * k * k * units
-        byts = 4.0 * (m * (cin + cout) + units * (1 + g * k * k) + cout + cout // g + 1)
+        taps = k * k if tap_mask is None else int(tap_mask.sum()) / float(g * units)   # kept taps per kept kernel
+        flops = 2.0 * m * g * taps * units
+        byts = 4.0 * (m * (cin + cout) + units * (1 + g * taps) + cout + cout // g + 1)
         peak = bf16_tflops if mode == "bf16_tc" else FP32_PEAK_TFLOPS
         t_alu, t_hbm = flops / (peak * 1e12), byts / (hbm_gbs * 1e9)
         rec = {"case": name, "mode": mode, "G": g, "sparsity_pct": d["sparsity_pct"], "us": round(t * 1e6, 1),
@@ -348,7 +352,9 @@ def single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, reps):
             rec["us_channel_major"] = round(tc * 1e6, 1)
             rec["frac_channel_major"] = round(max(t_alu, t_hbm) / tc, 3)
             del xt, yt
-        if k == 3 and w % 4 == 0:
+        if tap_mask is not None:
+            rec["kept_taps_per_kernel"] = round(taps, 2)
+        if k == 3 and w % 4 == 0 and tap_mask is None:
             # the 3x3 layer in the kernel's own layout (channel-major in and out): no conversion pass
             ld = (m + 3) // 4 * 4
             xt, yt = torch.empty((cin, ld), device="cuda"), torch.empty((cout, ld), device="cuda")
@@ -367,7 +373,11 @@ def single_layer_lines(sbnn, torch, flush, hbm_gbs, bf16_tflops, reps):
         del xd, yd
 
     one("config1", WL.config1(), 1, sbnn.SBNN_RELU, "fp32")
-    one("config4", WL.config4(), 3, sbnn.SBNN_RELU, "fp32")
+    d4 = WL.config4()
+    one("config4", d4, 3, sbnn.SBNN_RELU, "fp32")
+    from sbnn_inputs import tap_pattern_mask
+    one("config4_patterns_4_of_9_taps", d4, 3, sbnn.SBNN_RELU, "fp32", tap_mask=tap_pattern_mask(0, 19, d4["unit_mask"], 4, 4))
+    del d4
     cases = [(g, sp) for g in (4, 8) for sp in (0, 30, 50, 70, 90)]
     for (g, sp), d in zip(cases, WL.config5_family(cases)):
         one(f"config5_G{g}_s{sp}", d, 1, sbnn.SBNN_RELU, "fp32")

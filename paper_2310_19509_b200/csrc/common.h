@@ -120,6 +120,7 @@ struct sbnn_packed {
     std::vector<int32_t> group_ptr, idx;
     std::vector<float> val, bias;
     std::vector<uint16_t> tap_mask;   // per kept unit, bit t = tap t kept; empty unless packed with tap patterns
+    mutable long long kept_taps = -1; // taps kept over all units of a pattern layer (counted on first use, under mu)
     int gi = 1;                       // 4 if every group's kept channels are aligned runs of 4 (the paper's 4 x 4 blocks), else 1
     std::vector<int32_t> block_idx;   // gi == 4: first channel of every run, [nnz / 4]
     // device side (valid when device >= 0)

@@ -696,6 +696,20 @@ int sm_count3() {
     return it->second;
 }
 
+// True if a layer packed with kernel patterns should run the tap-list kernel: a listed tap costs about 60 us per "every
+// kept kernel, one tap" on config 4's shape, the whole-kernel loop with two output rows per lane about 35 us per tap
+// including the pruned ones (their stored weights are zeros), so lists pay below about five kept taps per kernel.
+bool use_tap_lists(const sbnn_packed* p) {
+    if (p->tap_mask.empty()) return false;
+    std::lock_guard<std::mutex> lk(p->mu);
+    if (p->kept_taps < 0) {
+        long long n = 0;
+        for (uint16_t m : p->tap_mask) n += __builtin_popcount(m);
+        p->kept_taps = n;
+    }
+    return (double)p->kept_taps < 4.8 * (double)p->tap_mask.size();
+}
+
 int pow2_ceil(int v) {
     int p = 1;
     while (p < v) p <<= 1;
@@ -1024,7 +1038,7 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     g.nchunks = (p->Cin + C::KC - 1) / C::KC;
     g.dpp_row = g.dpp_x = 0;
     if (g.pitch > 256 || g.R + 2 > 256 || W % 4 || ldx % 4) return SBNN_OK;
-    const bool pat = !p->tap_mask.empty();   // packed with kernel patterns: the kernel walks a list of kept taps
+    const bool pat = use_tap_lists(p);       // packed with kernel patterns: the kernel walks a list of kept taps
     if (pat && (long long)C::KC * g.plane + 2LL * g.pitch + 2 >= (1LL << 30)) return SBNN_OK;
     const int ws_u4 = pat ? C::WS_U4_TAPS : C::WS_U4;
     const int stage_bytes = (C::KC * g.plane * 4 + ws_u4 * 16 + 127) / 128 * 128;
@@ -1110,7 +1124,7 @@ template <int CW>
 sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int ldy, bool out_cm, int N, int H, int W,
                           int relu, cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
     // two output rows per lane where the image height allows it (whole-kernel layers; the tap lists keep one)
-    const bool two_rows = H % 2 == 0 && p->tap_mask.empty();
+    const bool two_rows = H % 2 == 0 && !use_tap_lists(p);
     switch (p->G) {
         case 1:
             if (two_rows) return launch3_tma<K3<1, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);

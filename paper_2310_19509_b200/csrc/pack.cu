@@ -440,6 +440,13 @@ extern "C" sbnn_status sbnn_packed_load(const char* path, sbnn_packed** out) {
         delete p;
         return st;
     }
+    // The weights of pruned taps are zeros, as the packer writes them: kernels that run a whole 3x3 kernel multiply them.
+    if (has_taps) {
+        for (int64_t u = 0; u < nnz; ++u)
+            for (int t = 0; t < taps; ++t)
+                if (!((p->tap_mask[u] >> t) & 1u))
+                    for (int r = 0; r < p->G; ++r) p->val[((size_t)u * taps + t) * p->G + r] = 0.0f;
+    }
     return finish_packed(p, out);
 }
 
