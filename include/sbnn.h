@@ -148,7 +148,8 @@ SBNN_API sbnn_status sbnn_packed_free(sbnn_packed* p);
  *   uint16       tap_mask[nnz_units]            only if has_tap_mask
  *   uint64       FNV-1a (64 bit) of all preceding bytes
  * Loading checks the magic, the version, the checksum and the structure (prefix sums, ascending in-range indices,
- * non-empty tap masks) and returns SBNN_ERR_IO for a file that cannot be read, is truncated or corrupt,
+ * non-empty tap masks), sets the stored weights of pruned taps to zero (as the packer writes them: kernels that run a
+ * whole 3x3 kernel multiply every stored tap), and returns SBNN_ERR_IO for a file that cannot be read, is truncated or corrupt,
  * SBNN_ERR_UNSUPPORTED for another version and SBNN_ERR_SHAPE for inconsistent contents; *out is NULL then.
  */
 SBNN_API sbnn_status sbnn_packed_save(const sbnn_packed* p, const char* path);

@@ -514,3 +514,40 @@ def test_conv3x3_work_plan_errors():
         sbnn.debug_plan_conv3x3(bp, 1, 4)
     with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_SHAPE"):
         sbnn.debug_plan_conv3x3(np.array([[0, 4, 8]], dtype=np.int32), 0, 4)
+
+
+def test_loading_a_pattern_layer_zeroes_the_weights_of_pruned_taps(tmp_path):
+    """A file whose value block holds something at a pruned tap (written by another tool) loads with zeros there:
+    the whole-kernel 3x3 loops multiply every stored tap, so the stored value of a pruned tap must be zero."""
+    import struct
+    rng = np.random.default_rng(41)
+    g, cin, cout = 2, 10, 6
+    w = rng.standard_normal((cout, 3, 3, cin)).astype(np.float32)
+    um = group_mask_layer_global(2, 3, cout // g, cin, 40)
+    m = tap_pattern_mask(2, 19, um, g, 4)
+    p = sbnn.pack_weights(w, m, None, g, tap_patterns=True)
+    path = str(tmp_path / "layer.sbnn")
+    p.save(path)
+    want = p.view()
+    p.free()
+    f = _read_packed_file(path)
+    raw = bytearray(open(path, "rb").read())
+    nnz = len(f["idx"])
+    val_off = 48 + 4 * (cout // g + 1) + 4 * nnz
+    poked = 0
+    for u in range(nnz):
+        for t in range(9):
+            if not (int(f["taps"][u]) >> t) & 1:
+                struct.pack_into("<f", raw, val_off + 4 * ((u * 9 + t) * g), 7.5)   # first filter of the group, pruned tap
+                poked += 1
+    assert poked > 0
+    h = 1469598103934665603
+    for byte in raw[:-8]:
+        h = ((h ^ byte) * 1099511628211) & 0xFFFFFFFFFFFFFFFF
+    struct.pack_into("<Q", raw, len(raw) - 8, h)
+    bad = str(tmp_path / "poked.sbnn")
+    open(bad, "wb").write(bytes(raw))
+    q = sbnn.load_packed(bad)
+    got = q.view()
+    assert np.array_equal(got["val"], want["val"]) and np.array_equal(got["tap_mask"], want["tap_mask"])
+    q.free()
