@@ -239,8 +239,8 @@ SBNN_API sbnn_status sbnn_to_channel_major(const float* x_dev, float* xt_dev, in
  * X taken as zero outside the image.  Shapes as above with KH = KW = 3.  SBNN_BF16_TC is not accepted.
  * W <= 256 and Cin a multiple of 4, else SBNN_ERR_UNSUPPORTED.  The first call with a new image width
  * builds a private re-layout of the weights (allocates and copies synchronously); later calls only enqueue.
- * For widths divisible by 4 the input is first copied, channel by channel, into a scratch buffer kept per
- * device (allocated or grown synchronously the first time a size is seen).
+ * The input is first copied, channel by channel (image rows padded to a multiple of 4 floats), into a scratch buffer
+ * kept per device (allocated or grown synchronously the first time a size is seen).
  */
 SBNN_API sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev, float* y_dev,
                                      int N, int H, int W, int flags, void* cuda_stream);

@@ -678,6 +678,27 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
     }
 }
 
+// X [M][C] (pixel-major, M = rows * W) -> planes Xt [C][rows][Wp] with the image rows padded to Wp >= W floats (a
+// multiple of 4, so that a row starts on a 16-byte boundary as the tiled copy requires): 32 x 32 tiles through
+// padded shared memory.  The Wp - W floats behind a row are never read (the copy treats x >= W as outside the tensor).
+__global__ void __launch_bounds__(256)
+to_padded_planes_kernel(const float* __restrict__ x, float* __restrict__ xt, int M, int C, int W, int Wp, long long ld) {
+    __shared__ float t[32][33];
+    const int m0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty + 8 * i, c = c0 + tx;
+        if (m < M && c < C) t[ty + 8 * i][tx] = x[(size_t)m * C + c];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = c0 + ty + 8 * i, m = m0 + tx;
+        if (m < M && c < C) xt[(size_t)c * ld + (size_t)(m / W) * Wp + (m % W)] = t[tx][ty + 8 * i];
+    }
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 // Number of SMs of the current device (one persistent CTA each).
@@ -1024,8 +1045,8 @@ sbnn_status launch3_cm(const sbnn_packed* p, const float* xt, int ldx, float* y,
 
 // Launches the copy-engine variant; *done = false (and SBNN_OK) if the shape does not fit it.
 template <class C>
-sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int ldy, bool out_cm, int N, int H, int W,
-                        int relu, cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
+sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, long long ldx, int row_pitch, float* y, int ldy, bool out_cm, int N,
+                        int H, int W, int relu, cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
     *done = false;
     Geo3 g;
     g.N = N; g.H = H; g.W = W; g.Cin = p->Cin; g.Cout = p->Cout; g.ngroups = p->ngroups;
@@ -1037,7 +1058,7 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     if (H % C::RPL) return SBNN_OK;                                // a lane's rows must lie in one image
     g.nchunks = (p->Cin + C::KC - 1) / C::KC;
     g.dpp_row = g.dpp_x = 0;
-    if (g.pitch > 256 || g.R + 2 > 256 || W % 4 || ldx % 4) return SBNN_OK;
+    if (g.pitch > 256 || g.R + 2 > 256 || row_pitch % 4 || ldx % 4) return SBNN_OK;   // rows and planes start on 16-byte boundaries
     const bool pat = use_tap_lists(p);       // packed with kernel patterns: the kernel walks a list of kept taps
     if (pat && (long long)C::KC * g.plane + 2LL * g.pitch + 2 >= (1LL << 30)) return SBNN_OK;
     const int ws_u4 = pat ? C::WS_U4_TAPS : C::WS_U4;
@@ -1101,7 +1122,7 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
     if (plan.ncounters) SBNN_CUDA_TRY(cudaMemsetAsync(counters, 0, (size_t)plan.ncounters * 4, st));
     Map3 xmap;
     const unsigned long long dims[3] = {(unsigned long long)W, (unsigned long long)NH, (unsigned long long)p->Cin};
-    const unsigned long long strides[2] = {(unsigned long long)W * 4, (unsigned long long)ldx * 4};
+    const unsigned long long strides[2] = {(unsigned long long)row_pitch * 4, (unsigned long long)ldx * 4};
     const unsigned box[3] = {(unsigned)g.pitch, (unsigned)(g.R + 2), (unsigned)C::KC};
     if ((r = encode_tiled_map(&xmap, xt, 4, 3, dims, strides, box)) != SBNN_OK) return r;
     const Seg3* segs = static_cast<const Seg3*>(plan.segs);
@@ -1121,17 +1142,17 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y
 }
 
 template <int CW>
-sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float* y, int ldy, bool out_cm, int N, int H, int W,
-                          int relu, cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
+sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, long long ldx, int row_pitch, float* y, int ldy, bool out_cm, int N,
+                          int H, int W, int relu, cudaStream_t st, unsigned char* extra, size_t extra_bytes, bool* done) {
     // two output rows per lane where the image height allows it (whole-kernel layers; the tap lists keep one)
     const bool two_rows = H % 2 == 0 && !use_tap_lists(p);
     switch (p->G) {
         case 1:
-            if (two_rows) return launch3_tma<K3<1, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
-            return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+            if (two_rows) return launch3_tma<K3<1, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<1, CW, 4, 7, 2, 8>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
         case 2:
-            if (two_rows) return launch3_tma<K3<2, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
-            return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+            if (two_rows) return launch3_tma<K3<2, CW, 2, 3, 4, 8, 2>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<2, CW, 4, 7, 2, 8>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
         case 4:
             if (two_rows) {
                 // 2 row warps x 6 group warps with 16-channel steps is about 6 % faster per group than 3 x 4 with
@@ -1139,14 +1160,14 @@ sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, int ldx, float*
                 // mostly empty.  Falls back to 3 x 4 when two stages of the larger tile do not fit.
                 const int ng = p->ngroups;
                 if ((ng + 5) / 6 * 6 * 0.94 < (ng + 3) / 4 * 4) {
-                    sbnn_status r = launch3_tma<K3<4, CW, 1, 2, 6, 16, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+                    sbnn_status r = launch3_tma<K3<4, CW, 1, 2, 6, 16, 2>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
                     if (r != SBNN_OK || *done) return r;
                 }
-                return launch3_tma<K3<4, CW, 1, 3, 4, 8, 2>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+                return launch3_tma<K3<4, CW, 1, 3, 4, 8, 2>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
             }
-            return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
-        case 8: return launch3_tma<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
-        default: return launch3_tma<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+            return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+        case 8: return launch3_tma<K3<8, CW, 1, 7, 2, 8>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+        default: return launch3_tma<K3<16, CW, 1, 7, 1, 8>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
     }
 }
 
@@ -1227,21 +1248,33 @@ extern "C" sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev,
     if (st != SBNN_OK) return st;
     if ((st = check_device()) != SBNN_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (W % 4 == 0) {
-        // fast path: planes of the input ([Cin][ld]) in the per-device scratch buffer, then the cp.async kernel
-        const int M = N * H * W, ld = (M + 3) / 4 * 4;
+    {
+        // fast path: planes of the input in the per-device scratch buffer ([Cin][N*H][Wp], rows padded to a multiple of
+        // 4 floats), then the copy-engine kernel
+        const int M = N * H * W, Wp = (W + 3) / 4 * 4;
+        const long long ld = (long long)N * H * Wp;
         float* xt = nullptr;
         const size_t xt_bytes = ((size_t)w->Cin * ld * sizeof(float) + 255) / 256 * 256, extra_bytes = tma_extra_bytes(cw);
         if ((st = scratch_workspace(xt_bytes + extra_bytes, s, &xt)) != SBNN_OK) return st;
-        if (!prepare_only() && (st = launch_transpose(x_dev, w->Cin, xt, ld, M, w->Cin, s)) != SBNN_OK) return st;
+        if (!prepare_only()) {
+            if (Wp == W) {
+                if ((st = launch_transpose(x_dev, w->Cin, xt, (int)ld, M, w->Cin, s)) != SBNN_OK) return st;
+            } else {
+                dim3 grid((M + 31) / 32, (w->Cin + 31) / 32);
+                to_padded_planes_kernel<<<grid, 256, 0, s>>>(x_dev, xt, M, w->Cin, W, Wp, ld);
+                SBNN_CUDA_TRY(cudaGetLastError());
+            }
+        }
         unsigned char* extra = reinterpret_cast<unsigned char*>(xt) + xt_bytes;
         bool done = false;
-        st = cw == 7 ? dispatch3_tma<7>(w, xt, ld, y_dev, w->Cout, false, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
-                     : dispatch3_tma<8>(w, xt, ld, y_dev, w->Cout, false, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
+        st = cw == 7 ? dispatch3_tma<7>(w, xt, ld, Wp, y_dev, w->Cout, false, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
+                     : dispatch3_tma<8>(w, xt, ld, Wp, y_dev, w->Cout, false, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
         if (st != SBNN_OK || done) return st;
-        st = cw == 7 ? dispatch3_cm<7>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
-                     : dispatch3_cm<8>(w, xt, ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);
-        if (st != SBNN_OK || done) return st;
+        if (Wp == W && ld <= 0x7fffffffLL) {
+            st = cw == 7 ? dispatch3_cm<7>(w, xt, (int)ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done)
+                         : dispatch3_cm<8>(w, xt, (int)ld, y_dev, N, H, W, flags & SBNN_RELU, s, &done);
+            if (st != SBNN_OK || done) return st;
+        }
     }
     return cw == 7 ? dispatch3<7>(w, x_dev, y_dev, N, H, W, flags & SBNN_RELU, s)
                    : dispatch3<8>(w, x_dev, y_dev, N, H, W, flags & SBNN_RELU, s);
@@ -1301,8 +1334,8 @@ extern "C" sbnn_status sbnn_conv3x3_gs_cm(const sbnn_packed* w, const float* xt_
     if ((st = scratch_workspace(extra_bytes, s, &scratch)) != SBNN_OK) return st;
     bool done = false;
     unsigned char* extra = reinterpret_cast<unsigned char*>(scratch);
-    st = cw == 7 ? dispatch3_tma<7>(w, xt_dev, ldx, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
-                 : dispatch3_tma<8>(w, xt_dev, ldx, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
+    st = cw == 7 ? dispatch3_tma<7>(w, xt_dev, ldx, W, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
+                 : dispatch3_tma<8>(w, xt_dev, ldx, W, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
     if (st != SBNN_OK || done) return st;
     return fail(SBNN_ERR_UNSUPPORTED, "the pipelined 3x3 kernel does not take this shape (rows of %d pixels)", W);
 }
