@@ -959,6 +959,11 @@ TileCfg choose_cfg_cm(const sbnn_packed* p, long long M) {
     // count (warps of a ragged last group tile are idle).  Measured on the 1024 -> 1024 layer with 64-channel steps:
     // 8 warps (2 per scheduler) 1034 us, 12 warps (3 per scheduler) 1039 us, 11 warps 1109 us -- eleven warps cost as
     // much per tile as twelve; three warps on a scheduler hide about 2 % more latency than two.
+    // What a third warp on a scheduler hides of the per-list latencies grows as the lists get shorter: config 5,
+    // 12 against 8 warps (whole launch, so including the 4 % of the 12-warp CTA): 50 % kept units 1033 / 1025 us,
+    // 30 % kept 670 / 684 us, 10 % kept 313 / 352 us.
+    const double kept = (p->ngroups > 0 && p->Cin > 0) ? (double)p->nnz / ((double)p->ngroups * p->Cin) : 1.0;
+    const double hide3 = kept >= 0.5 ? 0.02 : (kept >= 0.3 ? 0.02 + 0.1 * (0.5 - kept) : 0.04 + 0.45 * (0.3 - kept));
     auto launch_cost = [&](const TileCfg& c) {
         const long long ptiles = (M + c.TM() - 1) / c.TM(), gtiles = (p->ngroups + c.GT() - 1) / c.GT();
         const long long sms = std::max(1, sm_count()), total = ptiles * gtiles;
@@ -969,7 +974,7 @@ TileCfg choose_cfg_cm(const sbnn_packed* p, long long M) {
             const int m = std::max(std::max(load[0], load[1]), std::max(load[2], load[3]));
             // (with the producer a 12-warp CTA has 13 warps, which the register file serves like 16: 128 registers a
             // thread instead of the 154 the loop wants, measured 4-6 % slower per tile than the 11-warp CTA)
-            return (m >= 3 ? 0.98 * m : (double)m) * (c.NW == 12 ? 1.04 : 1.0);
+            return (m >= 3 ? (1.0 - hide3) * m : (double)m) * (c.NW == 12 ? 1.04 : 1.0);
         };
         double full_tile = 0.0;                      // cost of one pass over the group tiles of a pixel tile
         for (long long g = 0; g < gtiles; ++g) full_tile += tile_cost(g);
