@@ -963,7 +963,7 @@ TileCfg choose_cfg_cm(const sbnn_packed* p, long long M) {
     // 12 against 8 warps (whole launch, so including the 4 % of the 12-warp CTA): 50 % kept units 1033 / 1025 us,
     // 30 % kept 670 / 684 us, 10 % kept 313 / 352 us.
     const double kept = (p->ngroups > 0 && p->Cin > 0) ? (double)p->nnz / ((double)p->ngroups * p->Cin) : 1.0;
-    const double hide3 = kept >= 0.5 ? 0.02 : (kept >= 0.3 ? 0.02 + 0.1 * (0.5 - kept) : 0.04 + 0.45 * (0.3 - kept));
+    const double hide3 = kept >= 0.5 ? 0.02 : (kept >= 0.3 ? 0.02 + 0.2 * (0.5 - kept) : 0.06 + 0.35 * (0.3 - kept));
     auto launch_cost = [&](const TileCfg& c) {
         const long long ptiles = (M + c.TM() - 1) / c.TM(), gtiles = (p->ngroups + c.GT() - 1) / c.GT();
         const long long sms = std::max(1, sm_count()), total = ptiles * gtiles;
