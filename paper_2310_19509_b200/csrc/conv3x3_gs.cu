@@ -982,18 +982,22 @@ sbnn_status launch3(const sbnn_packed* p, const float* x, float* y, int N, int H
 // Pitch for the channel-major variant: a multiple of 4 (16-byte aligned row pieces), >= LPR*CW + 5, and such
 // that the first reads of the 32 lanes fall into 32 distinct banks if possible.
 int pick_pitch4(int LPR, int CW, int RPL = 1) {
+    // Fewest lanes on the busiest bank; ties go to the smaller pitch.  (With few lanes per row a warp spans many rows,
+    // whose offsets are multiples of the pitch: no multiple of 4 spreads them over 32 banks, but the choice still
+    // matters: a pitch of 16 with two rows per lane puts all 32 lanes on one bank, 20 on four.)
     const int lo = (LPR * CW + 5 + 3) / 4 * 4;
+    int best = lo, best_worst = 33;
     for (int p = lo; p < lo + 128; p += 4) {
-        unsigned used = 0;
-        bool ok = true;
-        for (int l = 0; l < 32 && ok; ++l) {
-            const int b = ((l / LPR) * RPL * p + (l % LPR) * CW) & 31;
-            ok = !((used >> b) & 1u);
-            used |= 1u << b;
+        int count[32] = {0};
+        int worst = 0;
+        for (int l = 0; l < 32; ++l) worst = std::max(worst, ++count[((l / LPR) * RPL * p + (l % LPR) * CW) & 31]);
+        if (worst < best_worst) {
+            best_worst = worst;
+            best = p;
         }
-        if (ok) return p;
+        if (worst == 1) break;
     }
-    return lo;
+    return best;
 }
 
 // Launches the channel-major variant; *done = false (and SBNN_OK) if the shape does not fit it.
