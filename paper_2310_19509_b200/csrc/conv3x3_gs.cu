@@ -612,7 +612,42 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
             const bool last = *last_flag != 0;
             if (!last || !alive) continue;
             __threadfence();
-            const f32x2* first = partial + (size_t)sg.slot * (ACC2 * C::NT) + tid;
+            // Part 0 straight into the accumulators (all loads independent and in flight together), then the other
+            // parts in part order, CW * GP loads at a time, and the bias last.  (One accumulator after the other, each
+            // with its own loop over the parts, was a chain of ACC2 * nparts dependent L2 latencies.)
+            const f32x2* src = partial + (size_t)sg.slot * (ACC2 * C::NT) + tid;
+#pragma unroll
+            for (int q = 0; q < GPW; ++q)
+#pragma unroll
+                for (int ro = 0; ro < RPL; ++ro)
+#pragma unroll
+                    for (int p = 0; p < CW; ++p)
+#pragma unroll
+                        for (int rr = 0; rr < GP; ++rr)
+                            acc[q][ro][p][rr] = __ldcg(src + (size_t)(((q * RPL + ro) * CW + p) * GP + rr) * C::NT);
+            for (int j = 1; j < sg.nparts; ++j) {
+                src += (size_t)ACC2 * C::NT;
+#pragma unroll
+                for (int q = 0; q < GPW; ++q)
+#pragma unroll
+                    for (int ro = 0; ro < RPL; ++ro) {
+                        f32x2 t[CW][GP];
+#pragma unroll
+                        for (int p = 0; p < CW; ++p)
+#pragma unroll
+                            for (int rr = 0; rr < GP; ++rr)
+                                t[p][rr] = __ldcg(src + (size_t)(((q * RPL + ro) * CW + p) * GP + rr) * C::NT);
+#pragma unroll
+                        for (int p = 0; p < CW; ++p)
+#pragma unroll
+                            for (int rr = 0; rr < GP; ++rr) {
+                                float s0, s1, t0, t1;
+                                unpack2(acc[q][ro][p][rr], s0, s1);
+                                unpack2(t[p][rr], t0, t1);
+                                acc[q][ro][p][rr] = pack2(s0 + t0, s1 + t1);
+                            }
+                    }
+            }
 #pragma unroll
             for (int q = 0; q < GPW; ++q) {
                 const int g = tile * C::GT + gw * GPW + q;
@@ -623,18 +658,11 @@ conv3x3_gs_tma_kernel(const __grid_constant__ Map3 xmap, float* __restrict__ Y, 
 #pragma unroll
                     for (int ro = 0; ro < RPL; ++ro)
 #pragma unroll
-                    for (int p = 0; p < CW; ++p) {
-                        const f32x2* src = first + (size_t)(((q * RPL + ro) * CW + p) * GP + rr) * C::NT;
-                        float s0, s1;
-                        unpack2(__ldcg(src), s0, s1);
-                        for (int j = 1; j < sg.nparts; ++j) {
-                            float t0, t1;
-                            unpack2(__ldcg(src + (size_t)j * (ACC2 * C::NT)), t0, t1);
-                            s0 += t0;
-                            s1 += t1;
+                        for (int p = 0; p < CW; ++p) {
+                            float s0, s1;
+                            unpack2(acc[q][ro][p][rr], s0, s1);
+                            acc[q][ro][p][rr] = pack2(s0 + b0, s1 + b1);
                         }
-                        acc[q][ro][p][rr] = pack2(s0 + b0, s1 + b1);
-                    }
                 }
             }
         } else if (!alive) {
