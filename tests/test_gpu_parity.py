@@ -544,6 +544,39 @@ def test_3x3_channel_major_entry_refuses_what_it_cannot_run():
     p.free()
 
 
+@pytest.mark.parametrize("seed", list(range(24)))
+def test_3x3_seeded_random_shapes(seed):
+    """Shapes drawn from a seeded generator (widths 1-44 including odd ones, which the library pads to whole 16-byte
+    rows; heights 1-20, odd and even; every group width; empty, sparse and dense masks; Cin a multiple of 4), through
+    the pixel-major entry point, and through the channel-major one where the width allows it.  Every output against the
+    oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    g = int(rng.choice([1, 2, 4, 8, 16]))
+    n, h, w = int(rng.integers(1, 6)), int(rng.integers(1, 21)), int(rng.integers(1, 45))
+    cin = 4 * int(rng.integers(1, 11))
+    cout = g * int(rng.integers(1, 9))
+    sp = int(rng.choice([0, 30, 50, 50, 80, 100]))
+    relu = bool(rng.integers(0, 2))
+    d = WL.single_conv_inputs(n, h, w, cin, cout, 3, g, sp, seed=100 + seed, w_sigma=0.1, mask_mode="layer_global")
+    ref, s = R.conv2d(d["x"], d["w"], d["mask"], d["bias"], relu=relu)
+    what = f"seed {seed}: {n}x{h}x{w}, {cin} -> {cout}, G={g}, {sp} % pruned, relu={relu}"
+    y = run_3x3(d, sbnn.SBNN_RELU if relu else 0)
+    assert_within(y, ref, s, what=what)
+    if w % 4 == 0:
+        p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], g)
+        m = n * h * w
+        ld = (m + 3) // 4 * 4
+        xt = torch.full((cin, ld), float("nan"), device="cuda")
+        sbnn.to_channel_major(dev(d["x"]), xt, m, cin, ld)
+        out = Guarded((cout, ld))
+        sbnn.conv3x3_gs_cm(p, xt, ld, out.t, ld, n, h, w, (sbnn.SBNN_RELU if relu else 0) | sbnn.SBNN_OUT_CM)
+        sbnn.get_async_status()
+        full = out.numpy(what)
+        assert np.all(np.isnan(full[:, m:]))
+        assert_within(full[:, :m].T.reshape(n, h, w, cout), ref, s, what=what + " (channel-major)")
+        p.free()
+
+
 def test_3x3_same_result_on_every_run():
     """Split tiles are added in part order whichever part arrives last: two runs agree bit for bit."""
     d = WL.single_conv_inputs(40, 14, 28, 64, 64, 3, 4, 50, seed=22, w_sigma=0.05)
