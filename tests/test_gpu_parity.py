@@ -585,7 +585,7 @@ def test_3x3_same_result_on_every_run():
         assert np.array_equal(run_3x3(d), y0)
 
 
-@pytest.mark.parametrize("g,kept_taps", [(4, 4), (2, 4), (8, 6), (1, 1)])
+@pytest.mark.parametrize("g,kept_taps", [(4, 4), (2, 4), (8, 6), (8, 3), (16, 2), (1, 1)])
 def test_3x3_kernel_patterns(g, kept_taps):
     """Kernels pruned tap by tap (centre + kept_taps - 1 others, one pattern per group and input channel, packed by
     sbnn_pack_weights_pattern) on top of 50 % removed kernels: same result as the oracle's masked dense convolution."""
