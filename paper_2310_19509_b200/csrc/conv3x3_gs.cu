@@ -1197,6 +1197,12 @@ sbnn_status dispatch3_tma(const sbnn_packed* p, const float* xt, long long ldx, 
                 }
                 return launch3_tma<K3<4, CW, 1, 3, 4, 8, 2>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
             }
+            {
+                // one row per lane (tap lists, odd heights): one group per warp on 3 x 4 warps with 16-channel steps
+                // (four-tap pattern layer of config 4's shape: 263 -> 220 us against two groups per warp on 7 x 2 warps)
+                sbnn_status r = launch3_tma<K3<4, CW, 1, 3, 4, 16>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
+                if (r != SBNN_OK || *done) return r;
+            }
             return launch3_tma<K3<4, CW, 2, 7, 2, 8>>(p, xt, ldx, row_pitch, y, ldy, out_cm, N, H, W, relu, st, extra, extra_bytes, done);
         case 8: {
             // one row per lane (two would need 112 accumulators); 16-channel steps on 12 warps measured 8 % faster than
