@@ -727,6 +727,16 @@ to_padded_planes_kernel(const float* __restrict__ x, float* __restrict__ xt, int
     }
 }
 
+// Planes Xt [C][ldx] (rows of W floats back to back) -> planes [C][rows][Wp] with rows padded to Wp floats.
+__global__ void __launch_bounds__(256)
+pad_plane_rows_kernel(const float* __restrict__ xt, long long ldx, float* __restrict__ xp, long long ldp, long long rows, int W,
+                      int Wp) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;   // element of a plane
+    const int c = blockIdx.y;
+    if (i >= rows * W) return;
+    xp[(size_t)c * ldp + (size_t)(i / W) * Wp + (i % W)] = xt[(size_t)c * ldx + i];
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 // Number of SMs of the current device (one persistent CTA each).
@@ -1372,18 +1382,35 @@ extern "C" sbnn_status sbnn_conv3x3_gs_cm(const sbnn_packed* w, const float* xt_
     if (w->Cin % 4) return fail(SBNN_ERR_UNSUPPORTED, "Cin=%d is not a multiple of 4", w->Cin);
     if (M == 0) return SBNN_OK;
     const int cw = choose_cw(W);
-    if (!cw || W % 4) return fail(SBNN_ERR_UNSUPPORTED, "W=%d: the channel-major 3x3 kernel takes widths divisible by 4, at most 256", W);
+    if (!cw) return fail(SBNN_ERR_UNSUPPORTED, "W=%d: the 3x3 kernel handles rows of at most 256 pixels", W);
+    if (w->Cin > 65535) return fail(SBNN_ERR_SHAPE, "too many input channels");
     sbnn_status st = check_packed_device(w);
     if (st != SBNN_OK) return st;
     if ((st = check_device()) != SBNN_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    // Widths that are not multiples of 4: the rows of the planes do not start on 16-byte boundaries, which the tiled
+    // copy needs, so the planes are first copied into the scratch buffer with padded rows.
+    const int Wp = (W + 3) / 4 * 4;
+    const long long rows = (long long)N * H, ldp = rows * Wp;
+    const size_t pad_bytes = Wp == W ? 0 : ((size_t)w->Cin * ldp * sizeof(float) + 255) / 256 * 256;
     float* scratch = nullptr;
     const size_t extra_bytes = tma_extra_bytes(cw);
-    if ((st = scratch_workspace(extra_bytes, s, &scratch)) != SBNN_OK) return st;
+    if ((st = scratch_workspace(pad_bytes + extra_bytes, s, &scratch)) != SBNN_OK) return st;
+    const float* planes = xt_dev;
+    long long ldplanes = ldx;
+    if (Wp != W) {
+        if (!prepare_only()) {
+            dim3 grid((unsigned)((M + 255) / 256), (unsigned)w->Cin);
+            pad_plane_rows_kernel<<<grid, 256, 0, s>>>(xt_dev, ldx, scratch, ldp, rows, W, Wp);
+            SBNN_CUDA_TRY(cudaGetLastError());
+        }
+        planes = scratch;
+        ldplanes = ldp;
+    }
     bool done = false;
-    unsigned char* extra = reinterpret_cast<unsigned char*>(scratch);
-    st = cw == 7 ? dispatch3_tma<7>(w, xt_dev, ldx, W, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
-                 : dispatch3_tma<8>(w, xt_dev, ldx, W, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
+    unsigned char* extra = reinterpret_cast<unsigned char*>(scratch) + pad_bytes;
+    st = cw == 7 ? dispatch3_tma<7>(w, planes, ldplanes, Wp, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
+                 : dispatch3_tma<8>(w, planes, ldplanes, Wp, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
     if (st != SBNN_OK || done) return st;
     return fail(SBNN_ERR_UNSUPPORTED, "the pipelined 3x3 kernel does not take this shape (rows of %d pixels)", W);
 }

@@ -478,7 +478,8 @@ def test_3x3_tiles_split_between_persistent_ctas(g, n, h, w, cin, cout):
 
 
 @pytest.mark.parametrize("g,n,h,w,cin,cout", [(4, 3, 28, 28, 256, 256), (4, 5, 14, 28, 40, 72), (8, 4, 7, 28, 32, 64),
-                                               (2, 3, 8, 56, 24, 20), (16, 2, 6, 100, 20, 48), (1, 2, 10, 12, 8, 7)])
+                                               (2, 3, 8, 56, 24, 20), (16, 2, 6, 100, 20, 48), (1, 2, 10, 12, 8, 7),
+                                               (4, 6, 14, 14, 64, 48), (8, 9, 7, 7, 32, 40), (4, 2, 5, 13, 12, 8)])
 def test_3x3_channel_major_entry(g, n, h, w, cin, cout):
     """sbnn_conv3x3_gs_cm: activations given as channel-major planes (the layout the pipelined kernel stages from, no
     conversion pass), output pixel-major or, with SBNN_OUT_CM, channel-major with a padded leading dimension whose
@@ -537,8 +538,8 @@ def test_3x3_channel_major_entry_refuses_what_it_cannot_run():
     p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], 4)
     xt = torch.zeros((8, 40), device="cuda")
     y = torch.zeros((36, 8), device="cuda")
-    with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_UNSUPPORTED"):      # W = 6 is not a multiple of 4
-        sbnn.conv3x3_gs_cm(p, xt, 40, y, 8, 1, 6, 6, sbnn.SBNN_RELU)
+    with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_SHAPE"):            # ldy < Cout
+        sbnn.conv3x3_gs_cm(p, xt, 40, y, 4, 1, 6, 6, sbnn.SBNN_RELU)
     with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_SHAPE"):            # ldx < M
         sbnn.conv3x3_gs_cm(p, xt, 32, y, 8, 1, 6, 6, sbnn.SBNN_RELU)
     p.free()
@@ -548,8 +549,7 @@ def test_3x3_channel_major_entry_refuses_what_it_cannot_run():
 def test_3x3_seeded_random_shapes(seed):
     """Shapes drawn from a seeded generator (widths 1-44 including odd ones, which the library pads to whole 16-byte
     rows; heights 1-20, odd and even; every group width; empty, sparse and dense masks; Cin a multiple of 4), through
-    the pixel-major entry point, and through the channel-major one where the width allows it.  Every output against the
-    oracle."""
+    the pixel-major entry point and through the channel-major one.  Every output against the oracle."""
     rng = np.random.default_rng(1000 + seed)
     g = int(rng.choice([1, 2, 4, 8, 16]))
     n, h, w = int(rng.integers(1, 6)), int(rng.integers(1, 21)), int(rng.integers(1, 45))
@@ -562,7 +562,7 @@ def test_3x3_seeded_random_shapes(seed):
     what = f"seed {seed}: {n}x{h}x{w}, {cin} -> {cout}, G={g}, {sp} % pruned, relu={relu}"
     y = run_3x3(d, sbnn.SBNN_RELU if relu else 0)
     assert_within(y, ref, s, what=what)
-    if w % 4 == 0:
+    if True:                                                    # every width: odd ones are padded into the scratch buffer
         p = sbnn.pack_weights(d["w"], d["mask"], d["bias"], g)
         m = n * h * w
         ld = (m + 3) // 4 * 4
