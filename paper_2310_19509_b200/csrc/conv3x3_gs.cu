@@ -1107,7 +1107,7 @@ sbnn_status launch3_tma(const sbnn_packed* p, const float* xt, long long ldx, in
     const int stage_bytes = (C::KC * g.plane * 4 + ws_u4 * 16 + 127) / 128 * 128;
     const size_t tail = (size_t)2 * 3 * 8 + 16 + (size_t)g.pitch * 4;
     int S = 3;
-    if ((size_t)S * stage_bytes + tail > 227 * 1024) S = 2;
+    while (S > 1 && (size_t)S * stage_bytes + tail > 227 * 1024) --S;   // (one stage: copy and arithmetic take turns; narrow maps with many rows per warp)
     const size_t smem = (size_t)S * stage_bytes + tail;
     if (smem > 227 * 1024) return SBNN_OK;
     const long long NH = (long long)N * H;

@@ -463,7 +463,8 @@ def test_3x3_shapes_and_groups(g, hw):
 
 @pytest.mark.parametrize("g,n,h,w,cin,cout", [(4, 40, 14, 28, 64, 64), (4, 9, 7, 28, 40, 96), (8, 12, 14, 28, 64, 128),
                                                (2, 30, 8, 56, 32, 24), (1, 20, 10, 28, 24, 40), (16, 6, 28, 28, 48, 64),
-                                               (4, 200, 14, 28, 16, 32), (4, 20, 14, 28, 40, 72), (4, 3, 56, 56, 24, 120)])
+                                               (4, 200, 14, 28, 16, 32), (4, 20, 14, 28, 40, 72), (4, 3, 56, 56, 24, 120),
+                                               (16, 20, 16, 8, 16, 32)])   # (8-wide map, 224 rows per CTA: one stage only)
 def test_3x3_tiles_split_between_persistent_ctas(g, n, h, w, cin, cout):
     """The pipelined 3x3 kernel deals the channel steps of all tiles to one CTA per SM in equal shares.  Shapes with
     a few steps per CTA (every tile cut into several parts whose partial sums the last arrival adds), with about as
@@ -479,7 +480,7 @@ def test_3x3_tiles_split_between_persistent_ctas(g, n, h, w, cin, cout):
 
 @pytest.mark.parametrize("g,n,h,w,cin,cout", [(4, 3, 28, 28, 256, 256), (4, 5, 14, 28, 40, 72), (8, 4, 7, 28, 32, 64),
                                                (2, 3, 8, 56, 24, 20), (16, 2, 6, 100, 20, 48), (1, 2, 10, 12, 8, 7),
-                                               (4, 6, 14, 14, 64, 48), (8, 9, 7, 7, 32, 40), (4, 2, 5, 13, 12, 8)])
+                                               (4, 6, 14, 14, 64, 48), (8, 9, 7, 7, 32, 40), (4, 2, 5, 13, 12, 8), (16, 20, 16, 8, 16, 32)])
 def test_3x3_channel_major_entry(g, n, h, w, cin, cout):
     """sbnn_conv3x3_gs_cm: activations given as channel-major planes (the layout the pipelined kernel stages from, no
     conversion pass), output pixel-major or, with SBNN_OUT_CM, channel-major with a padded leading dimension whose
