@@ -253,7 +253,7 @@ SBNN_API sbnn_status sbnn_conv3x3_gs(const sbnn_packed* w, const float* x_dev, f
  *   output: y_dev [M][ldy] (pixel-major rows of ldy >= Cout floats, ldy a multiple of 4), or, with SBNN_OUT_CM,
  *   [Cout][ldy] with ldy >= M.
  *   flags: SBNN_RELU, SBNN_OUT_CM.
- * W at most 250, Cin a multiple of 4, else SBNN_ERR_UNSUPPORTED.  For widths that are not multiples of 4 the planes are
+ * W at most 224 (a staged plane row is at most 256 floats), Cin a multiple of 4, else SBNN_ERR_UNSUPPORTED.  For widths that are not multiples of 4 the planes are
  * first copied into the per-device scratch buffer with their rows padded to whole 16-byte units (one extra pass).  The
  * partial sums of tiles that are shared between CTAs live in the per-device scratch buffer (see sbnn_conv1x1_gs_cm for its rules); the first call
  * with a new width builds a private re-layout of the weights and a work plan (allocates and copies synchronously).

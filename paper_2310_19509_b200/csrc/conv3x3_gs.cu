@@ -1412,5 +1412,5 @@ extern "C" sbnn_status sbnn_conv3x3_gs_cm(const sbnn_packed* w, const float* xt_
     st = cw == 7 ? dispatch3_tma<7>(w, planes, ldplanes, Wp, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done)
                  : dispatch3_tma<8>(w, planes, ldplanes, Wp, y_dev, ldy, out_cm, N, H, W, flags & SBNN_RELU, s, extra, extra_bytes, &done);
     if (st != SBNN_OK || done) return st;
-    return fail(SBNN_ERR_UNSUPPORTED, "the pipelined 3x3 kernel does not take this shape (rows of %d pixels)", W);
+    return fail(SBNN_ERR_UNSUPPORTED, "the pipelined 3x3 kernel does not take this shape (rows of %d pixels; it stages rows of at most 224)", W);
 }

@@ -543,6 +543,9 @@ def test_3x3_channel_major_entry_refuses_what_it_cannot_run():
         sbnn.conv3x3_gs_cm(p, xt, 40, y, 4, 1, 6, 6, sbnn.SBNN_RELU)
     with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_SHAPE"):            # ldx < M
         sbnn.conv3x3_gs_cm(p, xt, 32, y, 8, 1, 6, 6, sbnn.SBNN_RELU)
+    wide_x, wide_y = torch.zeros((8, 240), device="cuda"), torch.zeros((240, 8), device="cuda")
+    with pytest.raises(sbnn.SbnnError, match="SBNN_ERR_UNSUPPORTED"):      # rows of 240 pixels are wider than a staged plane row
+        sbnn.conv3x3_gs_cm(p, wide_x, 240, wide_y, 8, 1, 1, 240, sbnn.SBNN_RELU)
     p.free()
 
 
