@@ -146,3 +146,45 @@ def test_mobilenet_batch64_every_pointwise_layer_alone_at_full_size():
         bad = np.abs(got - ref) > TOL * s
         assert not bad.any(), f"{L['name']}: {bad.sum()} of {bad.size} outputs outside tolerance"
     net.free()
+
+
+@pytest.mark.parametrize("batch,sparsity", [(64, 50), (64, 70), (1, 30)])
+def test_mobilenet_chain_every_layer_within_its_own_tolerance(batch, sparsity):
+    """The chain as forward launches it (programmatic dependent launches, the tile shapes of this batch size), layer by
+    layer: the activations after layer l come from forward_prefix(l); for the first and the last image the oracle
+    applies layer l to the GPU's own activations after layer l - 1 and the result must agree within that layer's
+    tolerance 1e-5 * S.  Unlike the bound propagated through 29 layers, which grows by an order of magnitude per
+    layer, this catches an error of a few ulps in any one launch, and a kernel that started before its predecessor's
+    output was complete."""
+    x, layers = mobilenet_v1_inputs(batch, sparsity, 4, seed=0)
+    net = build_net(layers, batch)
+    xd = dev(x)
+    imgs = sorted({0, batch - 1})
+    prev = {img: np.ascontiguousarray(x[img:img + 1]) for img in imgs}      # input of the next layer, as the GPU has it
+    worst = 0.0
+    for li, L in enumerate(layers):
+        hin, cin, hout, cout = sbnn.mobilenet_v1_layer_shape(li)
+        hw = hout * hout
+        if L["kind"] == "fc":
+            out = Guarded((batch, cout))
+        else:
+            ld = (batch * hw + 3) // 4 * 4
+            out = Guarded((cout, ld))
+        net.forward_prefix(xd, out.t, batch, li)
+        sbnn.get_async_status()
+        got_all = out.numpy(L["name"])
+        for img in imgs:
+            rec = R.mobilenet_v1_forward(prev[img], [L])[0]
+            ref, s = rec["ref"], rec["S"]
+            if L["kind"] == "fc":
+                got = got_all[img].reshape(ref.shape)
+            else:
+                got = got_all[:, img * hw:(img + 1) * hw].T.reshape(ref.shape)
+            assert np.all(np.isfinite(got)), f"{L['name']}, image {img}"
+            err = np.abs(got.astype(np.float64) - ref)
+            lim = TOL * s + np.abs(ref) * 2.0 ** -23                        # + the fp32 rounding of the stored result
+            assert np.all(err <= lim), f"{L['name']}, image {img}: worst ratio {np.max(err / np.maximum(lim, 1e-300))}"
+            worst = max(worst, float(np.max(err / np.maximum(lim, 1e-300))))
+            prev[img] = np.ascontiguousarray(got, dtype=np.float32)
+    assert worst < 1.0
+    net.free()
